@@ -1,0 +1,206 @@
+/*
+ * CPU oracle for the AutoJudge verify-and-judge step.  TEST INFRASTRUCTURE ONLY.
+ *
+ * This file is the plain definition of what one speculation cycle's verification
+ * computes, written as slow fp64 loops.  It exists to check the CUDA library and to
+ * be timed as a reported CPU baseline.  It shares no code, header, table or helper
+ * with the CUDA path and must never be called from it; only the tests, the smoke
+ * check and the benchmark's cpu-baseline / reference arms may load it.
+ *
+ * What is computed, per sequence b (sequences are independent), with K draft tokens
+ * and K+1 rows of hidden states (row 0 encodes the last accepted token, row i+1
+ * encodes draft token i):
+ *
+ *   1. logit[j][v] = sum_k h_target[b][j][k] * W[k][v]             (LM head: the target
+ *      model's "forward ... outputs next token logits", Section 3.1)
+ *   2. y[j] = argmax_v logit[j][v]                                 (greedy target token;
+ *      Section 2 footnote on greedy verification, Algorithm 1 ".argmax(-1)")
+ *   3. position i mismatches when draft_tok[i] != y[i]             (the set I(x), Section 3.1)
+ *   4. at a mismatch the classifier is consulted: z = b + w . [h_draft[i+1] ; h_target[i+1]],
+ *      p = sigmoid(z) = P(important); the mismatch is forgiven iff p < tau
+ *      (Section 3.2 design choices 1-3, "Classifier model & training"; Section 3.3 Inference)
+ *   5. accept_len = number of leading positions that match or are forgiven; the first
+ *      unforgiven mismatch and everything after it are rejected (Section 2), and
+ *      next_tok = y[accept_len] (the target's own token there; y[K] if all K pass).
+ *
+ * Readings where the paper is silent: lowest index wins argmax ties; p < tau is strict;
+ * tau <= 0 never forgives and tau >= 1 always forgives; feature order is [draft ; target];
+ * the comparison p < tau is taken on p rounded to fp32 (the precision the kernel decides in).
+ *
+ * All inputs are converted exactly to double; every sum is accumulated in double.
+ *
+ * parity pins: see tests/test_oracle_pins.py (library matmul special case, one-hot
+ * closed forms, tau extremes, monotonicity, brute force over pass patterns, closed-form
+ * expectation of accept_len).  No function here is "parity unpinned".
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+enum { AJO_BF16 = 0, AJO_F32 = 1 };
+enum { AJO_W_VD = 0, AJO_W_DV = 1 };
+
+/* exact widening of one stored element to double */
+static double elem_to_double(const void *base, size_t idx, int dtype)
+{
+    if (dtype == AJO_BF16) {
+        uint32_t bits = ((uint32_t)((const uint16_t *)base)[idx]) << 16;
+        float f;
+        memcpy(&f, &bits, sizeof f);
+        return (double)f;
+    }
+    return (double)((const float *)base)[idx];
+}
+
+int ajo_num_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/*
+ * Step 1 for R rows: logits[r][v] = sum_k h[r][k] * W[k][v], r < R, v < V.
+ * h: R x d row-major; W: [V,d] row-major (w_layout 0) or [d,V] row-major (w_layout 1).
+ * logits: R x V doubles, caller-allocated.
+ */
+int ajo_logits(const void *h, const void *W, int dtype, int w_layout,
+               int R, int d, int V, double *logits)
+{
+    if (!h || !W || !logits || R < 0 || d < 1 || V < 1) return 1;
+    double *hd = (double *)malloc((size_t)(R > 0 ? R : 1) * d * sizeof(double));
+    if (!hd) return 2;
+    for (size_t i = 0; i < (size_t)R * d; i++) hd[i] = elem_to_double(h, i, dtype);
+
+    int failed = 0;
+#pragma omp parallel
+    {
+        double *wcol = (double *)malloc((size_t)d * sizeof(double));
+        if (!wcol) {
+#pragma omp atomic write
+            failed = 1;
+        }
+#pragma omp barrier
+        if (!failed) {
+#pragma omp for schedule(static)
+            for (int v = 0; v < V; v++) {
+                for (int k = 0; k < d; k++) {
+                    size_t idx = (w_layout == AJO_W_VD) ? (size_t)v * d + k : (size_t)k * V + v;
+                    wcol[k] = elem_to_double(W, idx, dtype);
+                }
+                for (int r = 0; r < R; r++) {
+                    const double *hr = hd + (size_t)r * d;
+                    double s = 0.0;
+                    /* summation order is free: every term is exact in double and the
+                       rounding error of any order is far below the comparison tolerances */
+#pragma omp simd reduction(+ : s)
+                    for (int k = 0; k < d; k++) s += hr[k] * wcol[k];
+                    logits[(size_t)r * V + v] = s;
+                }
+            }
+        }
+        free(wcol);
+    }
+    free(hd);
+    return failed ? 2 : 0;
+}
+
+/*
+ * Step 2 for one row: smallest index attaining the maximum, the maximum, and the
+ * distance to the largest value found at any other index (0 when the maximum is tied).
+ */
+void ajo_argmax(const double *row, int V, int32_t *y, double *top1, double *gap)
+{
+    int best = 0;
+    for (int v = 1; v < V; v++)
+        if (row[v] > row[best]) best = v;
+    double second = -INFINITY;
+    for (int v = 0; v < V; v++)
+        if (v != best && row[v] > second) second = row[v];
+    *y = best;
+    *top1 = row[best];
+    *gap = (V > 1) ? row[best] - second : INFINITY;
+}
+
+/*
+ * Step 4 for one position: P(important) from the logistic-regression judge on the
+ * concatenation [h_draft_row ; h_target_row]; judge_w has d_draft + d entries in that order.
+ */
+double ajo_judge_p(const void *h_draft_row, const void *h_target_row, int dtype,
+                   const float *judge_w, float judge_b, int d_draft, int d)
+{
+    double z = (double)judge_b;
+    for (int f = 0; f < d_draft; f++)
+        z += (double)judge_w[f] * elem_to_double(h_draft_row, (size_t)f, dtype);
+    for (int f = 0; f < d; f++)
+        z += (double)judge_w[d_draft + f] * elem_to_double(h_target_row, (size_t)f, dtype);
+    return 1.0 / (1.0 + exp(-z));
+}
+
+/* does the judge forgive a mismatch whose importance probability is p? */
+static int forgiven(double p, float tau)
+{
+    if (tau <= 0.0f) return 0;
+    if (tau >= 1.0f) return 1;
+    return (float)p < tau;
+}
+
+/*
+ * The whole step for B sequences.
+ *   h_target [B][K+1][d], h_draft [B][K+1][d_draft] (NULL iff d_draft == 0), W per w_layout,
+ *   draft_tok [B][K], judge_w [d_draft + d].
+ * Outputs (all caller-allocated, all required):
+ *   accept_len [B], next_tok [B], target_tok [B][K+1], top1 [B][K+1], gap [B][K+1],
+ *   judge_p [B][K]  (p at every mismatching position, NaN where the draft token matched).
+ */
+int ajo_verify(const void *h_target, const void *h_draft, const void *W,
+               const int32_t *draft_tok, const float *judge_w, float judge_b, float tau,
+               int dtype, int w_layout, int B, int K, int d, int d_draft, int V,
+               int32_t *accept_len, int32_t *next_tok, int32_t *target_tok,
+               double *top1, double *gap, double *judge_p)
+{
+    if (!h_target || !W || !draft_tok || !judge_w || B < 1 || K < 1 || d < 1 || V < 1 ||
+        d_draft < 0 || (d_draft > 0 && !h_draft))
+        return 1;
+    size_t esz = (dtype == AJO_BF16) ? 2 : 4;
+    int R = K + 1;
+    double *logits = (double *)malloc((size_t)R * V * sizeof(double));
+    if (!logits) return 2;
+
+    for (int b = 0; b < B; b++) {
+        const char *ht = (const char *)h_target + (size_t)b * R * d * esz;
+        const char *hdr = h_draft ? (const char *)h_draft + (size_t)b * R * d_draft * esz : NULL;
+        int rc = ajo_logits(ht, W, dtype, w_layout, R, d, V, logits);
+        if (rc) { free(logits); return rc; }
+
+        int32_t *y = target_tok + (size_t)b * R;
+        for (int j = 0; j < R; j++)
+            ajo_argmax(logits + (size_t)j * V, V, &y[j], &top1[(size_t)b * R + j], &gap[(size_t)b * R + j]);
+
+        /* p at every mismatch (the device evaluates all mismatches, so all are comparable) */
+        for (int i = 0; i < K; i++) {
+            double p = NAN;
+            if (draft_tok[(size_t)b * K + i] != y[i])
+                p = ajo_judge_p(hdr ? hdr + (size_t)(i + 1) * d_draft * esz : NULL,
+                                ht + (size_t)(i + 1) * d * esz, dtype, judge_w, judge_b, d_draft, d);
+            judge_p[(size_t)b * K + i] = p;
+        }
+
+        /* walk the window in order; stop at the first mismatch the judge does not forgive */
+        int n = 0;
+        while (n < K) {
+            if (draft_tok[(size_t)b * K + n] != y[n] && !forgiven(judge_p[(size_t)b * K + n], tau)) break;
+            n++;
+        }
+        accept_len[b] = n;
+        next_tok[b] = y[n];
+    }
+    free(logits);
+    return 0;
+}

@@ -1,0 +1,310 @@
+"""Pins for the CPU oracle: each test ties it to something other than itself.
+
+- a library routine on the special case where the step *is* that routine (fp64 matmul,
+  first-occurrence argmax);
+- closed forms (one-hot rows turn the projection into a table lookup; unit judge weights
+  turn the classifier into sigmoid(b + one feature));
+- what the paper fixes about the acceptance rule (Section 2: the first mismatch and
+  everything after it are rejected; Section 3.3: the classifier is consulted only where
+  the original rule would reject, a forgiven token is accepted and later tokens are then
+  tested as before; Section 4.3 tables: a larger threshold accepts more);
+- brute force over every match / forgiven / important pattern of a short window;
+- the closed-form expectation of the accepted length under the synthetic generator.
+"""
+import itertools
+import math
+
+import numpy as np
+import pytest
+
+import aj_inputs as gen
+from oracle import aj_oracle as orc
+
+BF16, F32 = gen.BF16, gen.F32
+
+
+def _store(x, dtype):
+    x = np.asarray(x, dtype=np.float32)
+    return gen.f32_to_bf16_bits(x) if dtype == BF16 else x
+
+
+# ---------------------------------------------------------------- projection + argmax
+
+
+@pytest.mark.parametrize("dtype", [BF16, F32])
+@pytest.mark.parametrize("layout", [0, 1])
+@pytest.mark.parametrize("R,d,V", [(1, 8, 5), (5, 96, 333), (17, 256, 1000), (33, 512, 4099)])
+def test_logits_equal_library_matmul(dtype, layout, R, d, V):
+    g = np.random.default_rng(R * 1000 + d + V)
+    h = _store(g.standard_normal((R, d)), dtype)
+    W = _store(g.standard_normal((V, d)) * 0.02, dtype)
+    Wl = W if layout == 0 else np.ascontiguousarray(W.T)
+    got = orc.logits(h, Wl, dtype, layout)
+    want = gen.to_f64(h, dtype) @ gen.to_f64(W, dtype).T
+    assert got.shape == (R, V)
+    np.testing.assert_allclose(got, want, rtol=0, atol=1e-11)
+    for r in range(R):
+        y, top1, gap = orc.argmax(got[r])
+        assert y == int(np.argmax(want[r]))
+        assert top1 == got[r, y]
+        srt = np.sort(got[r])
+        assert gap == pytest.approx(srt[-1] - srt[-2], abs=1e-15)
+
+
+@pytest.mark.parametrize("dtype", [BF16, F32])
+def test_one_hot_rows_read_a_column_of_W(dtype):
+    # h = e_k makes logit[v] = W[k, v] exactly, so y is a lookup in W.  A transposed
+    # operand or a wrong row/column index breaks this on a non-square W.
+    g = np.random.default_rng(7)
+    d, V = 48, 301
+    Wf = g.standard_normal((V, d)).astype(np.float32)
+    W = _store(Wf, dtype)
+    Wv = gen.to_f64(W, dtype)
+    ks = [0, 1, 17, d - 1]
+    h = np.zeros((len(ks), d), np.float32)
+    for r, k in enumerate(ks):
+        h[r, k] = 1.0
+    lg = orc.logits(_store(h, dtype), W, dtype, 0)
+    for r, k in enumerate(ks):
+        np.testing.assert_array_equal(lg[r], Wv[:, k])
+        assert orc.argmax(lg[r])[0] == int(np.argmax(Wv[:, k]))
+
+
+def test_argmax_ties_take_the_lowest_index_and_signed_zeros_tie():
+    assert orc.argmax(np.array([1.0, 3.0, 3.0, 2.0]))[0] == 1
+    assert orc.argmax(np.array([1.0, 3.0, 3.0, 2.0]))[2] == 0.0
+    assert orc.argmax(np.array([-0.0, 0.0, -1.0]))[0] == 0
+    assert orc.argmax(np.array([0.0, -0.0, -1.0]))[0] == 0
+    assert orc.argmax(np.array([-5.0, -2.0, -3.0])) == (1, -2.0, 1.0)
+    assert orc.argmax(np.array([4.0]))[0] == 0
+
+
+def test_projection_invariants():
+    g = np.random.default_rng(11)
+    R, d, V = 6, 64, 257
+    h = _store(g.standard_normal((R, d)), BF16)
+    W = _store(g.standard_normal((V, d)) * 0.02, BF16)
+    base = orc.logits(h, W, BF16)
+    y0 = [orc.argmax(r)[0] for r in base]
+    # permuting vocabulary entries permutes the winner
+    perm = g.permutation(V)
+    lp = orc.logits(h, np.ascontiguousarray(W[perm]), BF16)
+    inv = np.argsort(perm)
+    assert [orc.argmax(r)[0] for r in lp] == [int(inv[y]) for y in y0]
+    # doubling h (exact in bf16) doubles every logit and keeps the winner
+    h2 = _store(gen.bf16_bits_to_f32(h) * 2.0, BF16)
+    l2 = orc.logits(h2, W, BF16)
+    np.testing.assert_array_equal(l2, 2.0 * base)
+    # a duplicated winning column: the lower index is returned
+    for r in range(R):
+        Wd = W.copy()
+        hi = (y0[r] + 40) % V
+        lo_i, hi_i = min(y0[r], hi), max(y0[r], hi)
+        Wd[lo_i] = W[y0[r]]
+        Wd[hi_i] = W[y0[r]]
+        assert orc.argmax(orc.logits(h[r : r + 1], Wd, BF16)[0])[0] == lo_i
+
+
+# ------------------------------------------------------------------------------- judge
+
+
+def _sigmoid(z):
+    return 1.0 / (1.0 + math.exp(-z))
+
+
+@pytest.mark.parametrize("dtype", [BF16, F32])
+def test_judge_closed_forms(dtype):
+    g = np.random.default_rng(3)
+    d, dd = 40, 24
+    ht = _store(g.standard_normal(d), dtype)
+    hd = _store(g.standard_normal(dd), dtype)
+    xt, xd = gen.to_f64(ht, dtype), gen.to_f64(hd, dtype)
+    w0 = np.zeros(d + dd, np.float32)
+    for b in (-2.0, 0.0, 0.75):
+        assert orc.judge_p(hd, ht, dtype, w0, b) == pytest.approx(_sigmoid(b), abs=1e-15)
+    # unit weight on feature f: the first d_draft features are the draft model's, then the target's
+    for f in (0, 5, dd - 1, dd, dd + 7, dd + d - 1):
+        w = w0.copy()
+        w[f] = 1.0
+        x = xd[f] if f < dd else xt[f - dd]
+        assert orc.judge_p(hd, ht, dtype, w, 0.25) == pytest.approx(_sigmoid(0.25 + x), abs=1e-15)
+    # general weights against a float64 dot product; p(z) + p(-z) = 1
+    w = (g.standard_normal(d + dd) * 0.05).astype(np.float32)
+    z = float(w[:dd].astype(np.float64) @ xd + w[dd:].astype(np.float64) @ xt)
+    p = orc.judge_p(hd, ht, dtype, w, 0.0)
+    assert p == pytest.approx(_sigmoid(z), abs=1e-14)
+    assert p + orc.judge_p(hd, ht, dtype, -w, 0.0) == pytest.approx(1.0, abs=1e-14)
+    # target-only features
+    assert orc.judge_p(None, ht, dtype, w[dd:], 0.125) == pytest.approx(
+        _sigmoid(0.125 + float(w[dd:].astype(np.float64) @ xt)), abs=1e-14
+    )
+
+
+# ---------------------------------------------------------- acceptance rule: brute force
+
+
+def _controlled_case(pattern, V=9, d=9, dd=4):
+    """A window whose outcome at each position is chosen by hand.
+
+    pattern[i] in {"m", "f", "i"}: draft token matches / mismatches and is forgiven /
+    mismatches and is important.  W is the identity (V = d), rows of h_target are one-hot,
+    so y[j] is the position of the one; the judge reads draft feature 0 of row i+1.
+    """
+    K = len(pattern)
+    g = np.random.default_rng(sum(3**i * "mfi".index(c) for i, c in enumerate(pattern)) + 100 * K)
+    y = g.integers(0, V, size=K + 1)
+    ht = np.zeros((1, K + 1, d), np.float32)
+    for j in range(K + 1):
+        ht[0, j, y[j]] = 1.0
+    hd = np.zeros((1, K + 1, dd), np.float32)
+    tok = np.empty((1, K), np.int32)
+    for i, c in enumerate(pattern):
+        tok[0, i] = y[i] if c == "m" else (y[i] + 1 + g.integers(0, V - 1)) % V
+        hd[0, i + 1, 0] = {"m": 0.0, "f": -20.0, "i": 20.0}[c]
+    hd[0, 0, 0] = 20.0  # row 0 must never be read by the judge
+    w = np.zeros(dd + d, np.float32)
+    w[0] = 1.0
+    W = np.eye(V, d, dtype=np.float32)
+    return ht, hd, W, tok, w, y
+
+
+def _second_evaluator(passes):
+    """Largest n such that every position before n passes (no early exit)."""
+    K = len(passes)
+    return max(n for n in range(K + 1) if all(passes[:n]))
+
+
+@pytest.mark.parametrize("K", [1, 2, 3, 4])
+def test_every_pattern_of_a_short_window(K):
+    for pattern in itertools.product("mfi", repeat=K):
+        ht, hd, W, tok, w, y = _controlled_case(pattern)
+        r = orc.verify(ht, hd, W, tok, w, 0.0, 0.5, F32)
+        want = _second_evaluator([c != "i" for c in pattern])
+        assert r.accept_len[0] == want, pattern
+        assert r.next_tok[0] == y[want], pattern
+        np.testing.assert_array_equal(r.target_tok[0], y)
+        for i, c in enumerate(pattern):
+            if c == "m":
+                assert math.isnan(r.judge_p[0, i])
+            else:
+                assert r.judge_p[0, i] == pytest.approx(_sigmoid(20.0 if c == "i" else -20.0), abs=1e-12)
+        # never forgiving: plain greedy speculative decoding, stop at the first mismatch
+        r0 = orc.verify(ht, hd, W, tok, w, 0.0, 0.0, F32)
+        assert r0.accept_len[0] == _second_evaluator([c == "m" for c in pattern])
+        # always forgiving: the whole window and the bonus token
+        r1 = orc.verify(ht, hd, W, tok, w, 0.0, 1.0, F32)
+        assert r1.accept_len[0] == K and r1.next_tok[0] == y[K]
+
+
+@pytest.mark.parametrize("block", ["draft", "target"])
+def test_judge_reads_the_row_that_encodes_the_draft_token(block):
+    # one mismatch at position i; only row i+1 carries a large "important" feature, every
+    # other row would forgive.  Reading row i (the state that predicted the token) instead
+    # would accept.  The feature sits either in the draft block or in the target block
+    # (the last target feature has a zero row in W, so it does not disturb the argmax).
+    K, V, d, dd = 5, 7, 8, 3
+    W = np.eye(V, d, dtype=np.float32)
+    for i in range(K):
+        ht = np.zeros((1, K + 1, d), np.float32)
+        y = [(3 * j + 1) % V for j in range(K + 1)]
+        for j in range(K + 1):
+            ht[0, j, y[j]] = 1.0
+        hd = np.full((1, K + 1, dd), -1.0, np.float32)
+        ht[0, :, d - 1] = -1.0
+        feat = (hd, 2, 2) if block == "draft" else (ht, d - 1, dd + d - 1)
+        feat[0][0, i + 1, feat[1]] = 30.0
+        tok = np.array([y[:K]], np.int32)
+        tok[0, i] = (y[i] + 1) % V
+        w = np.zeros(dd + d, np.float32)
+        w[feat[2]] = 1.0
+        r = orc.verify(ht, hd, W, tok, w, 0.0, 0.5, F32)
+        np.testing.assert_array_equal(r.target_tok[0], y)
+        assert r.accept_len[0] == i and r.next_tok[0] == y[i]
+        feat[0][0, i + 1, feat[1]] = -30.0
+        r = orc.verify(ht, hd, W, tok, w, 0.0, 0.5, F32)
+        assert r.accept_len[0] == K
+
+
+# --------------------------------------------- acceptance rule: what the paper fixes
+
+
+def _random_case(cfg):
+    W = gen.make_W(cfg)
+    ht, hd = gen.make_hidden(cfg)
+    w = gen.make_judge(cfg)
+    y = np.stack([[orc.argmax(r)[0] for r in orc.logits(ht[b], W, cfg.dtype)] for b in range(cfg.B)])
+    tok = gen.plant_draft_tokens(cfg, y)
+    return W, ht, hd, w, y, tok
+
+
+@pytest.mark.parametrize("dtype", [BF16, F32])
+def test_threshold_extremes_monotonicity_and_vanilla_bound(dtype):
+    cfg = gen.Config("t", B=40, K=12, d=64, d_draft=32, V=211, dtype=dtype, sigma_w=0.2, match_lo=0.4, match_hi=0.9, seed=5)
+    W, ht, hd, w, y, tok = _random_case(cfg)
+    mism = tok != y[:, : cfg.K]
+    vanilla = np.array([int(np.argmax(np.append(m, True))) for m in mism])
+    prev = None
+    for tau in (0.0, 0.05, 0.2, 0.5, 0.8, 0.95, 1.0):
+        r = orc.verify(ht, hd, W, tok, w, cfg.judge_b, tau, dtype)
+        np.testing.assert_array_equal(r.target_tok, y)
+        assert (r.accept_len >= vanilla).all()
+        assert (r.next_tok == y[np.arange(cfg.B), r.accept_len]).all()
+        assert (np.isnan(r.judge_p) == ~mism).all()
+        if tau == 0.0:
+            np.testing.assert_array_equal(r.accept_len, vanilla)
+        if tau == 1.0:
+            assert (r.accept_len == cfg.K).all()
+        if prev is not None:
+            assert (r.accept_len >= prev).all()
+        prev = r.accept_len
+        # the replay helper agrees with the full evaluation
+        a2, n2 = orc.rewalk(r.target_tok, tok, r.judge_p, tau)
+        np.testing.assert_array_equal(a2, r.accept_len)
+        np.testing.assert_array_equal(n2, r.next_tok)
+    assert 0 < vanilla.mean() < cfg.K  # the case is not degenerate
+
+
+def test_sequences_are_independent_and_the_rejected_tail_is_never_consulted():
+    cfg = gen.Config("t", B=9, K=10, d=32, d_draft=16, V=97, dtype=BF16, sigma_w=0.3, match_lo=0.5, match_hi=0.9, seed=9)
+    W, ht, hd, w, y, tok = _random_case(cfg)
+    full = orc.verify(ht, hd, W, tok, w, 0.0, 0.5, BF16)
+    order = np.random.default_rng(0).permutation(cfg.B)
+    shuf = orc.verify(ht[order], hd[order], W, tok[order], w, 0.0, 0.5, BF16)
+    np.testing.assert_array_equal(shuf.accept_len, full.accept_len[order])
+    np.testing.assert_array_equal(shuf.next_tok, full.next_tok[order])
+    for b in range(cfg.B):
+        one = orc.verify(ht[b : b + 1], hd[b : b + 1], W, tok[b : b + 1], w, 0.0, 0.5, BF16)
+        assert one.accept_len[0] == full.accept_len[b] and one.next_tok[0] == full.next_tok[b]
+        n = int(full.accept_len[b])
+        if n + 2 <= cfg.K:  # junk after the stop changes nothing
+            t2, h2, g2 = tok.copy(), ht.copy(), hd.copy()
+            t2[b, n + 1 :] = 0
+            h2[b, n + 2 :] = gen.f32_to_bf16_bits(np.full((cfg.K - n - 1, cfg.d), 3.0, np.float32))
+            g2[b, n + 2 :] = 0
+            j = orc.verify(h2[b : b + 1], g2[b : b + 1], W, t2[b : b + 1], w, 0.0, 0.5, BF16)
+            assert j.accept_len[0] == n and j.next_tok[0] == full.next_tok[b]
+
+
+# ------------------------------------------ generator + oracle against a closed form
+
+
+def _phi(x):
+    return 0.5 * (1.0 + math.erf(x / math.sqrt(2.0)))
+
+
+@pytest.mark.parametrize("tau", [0.5, 0.7])
+def test_expected_accept_len_matches_closed_form(tau):
+    # With i.i.d. unit-variance features z ~ N(b, sigma_w^2 F), so a mismatch is forgiven
+    # with probability Phi(logit(tau) / sigma_z); a position passes with q = r + (1-r) * that,
+    # and E[accept_len] = sum_{i=1..K} q^i.
+    r_match, K = 0.6, 8
+    cfg = gen.Config("t", B=6000, K=K, d=48, d_draft=16, V=61, dtype=F32, sigma_w=0.1, match_lo=r_match, match_hi=r_match, seed=21)
+    W, ht, hd, w, y, tok = _random_case(cfg)
+    r = orc.verify(ht, hd, W, tok, w, 0.0, tau, F32)
+    sigma_z = float(np.sqrt((w.astype(np.float64) ** 2).sum()))
+    q = r_match + (1 - r_match) * _phi(math.log(tau / (1 - tau)) / sigma_z)
+    want = sum(q**i for i in range(1, K + 1))
+    var = sum((2 * i - 1) * q**i for i in range(1, K + 1)) - want**2  # E[N^2] - E[N]^2
+    se = math.sqrt(var / cfg.B)
+    assert abs(float(r.accept_len.mean()) - want) < 4 * se
+    assert abs(float((tok == y[:, :K]).mean()) - r_match) < 4 * math.sqrt(r_match * (1 - r_match) / (cfg.B * K))

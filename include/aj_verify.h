@@ -1,0 +1,142 @@
+/*
+ * aj_verify — the verify-and-judge step of AutoJudge speculative decoding on one B200 (sm_100a).
+ *
+ * One call verifies, for each of B sequences, a window of K draft tokens against the target
+ * model and reports how many leading draft tokens are kept and which token the target
+ * emits next.  Notation: M = B*(K+1) rows of hidden states; row 0 of a sequence encodes the
+ * last accepted token, row i+1 encodes draft token i; F = d_draft + d judge features.
+ *
+ * What a call computes (the paper's Section 2, greedy verification, relaxed as in Section 3.3):
+ *   logit[b,j,v] = sum_k h_target[b,j,k] * W_lm[k,v]      never written to memory
+ *   y[b,j]       = argmax_v logit[b,j,v]                   lowest index on ties
+ *   mismatch at i when draft_tok[b,i] != y[b,i]            (the set I(x) of Section 3.1)
+ *   at a mismatch only, the classifier of Section 3.2 is evaluated on the hidden states that
+ *   encode the mismatching draft token, draft and target model concatenated:
+ *       p = sigmoid(judge_b + judge_w . [h_draft[b,i+1,:] ; h_target[b,i+1,:]])   = P(important)
+ *   and the mismatch is forgiven iff p < tau (tau <= 0 never forgives, tau >= 1 always does);
+ *   accept_len[b] = number of leading positions that match or are forgiven; the first
+ *   unforgiven mismatch and everything after it are rejected (Section 2);
+ *   next_tok[b]   = y[b, accept_len[b]]  (the bonus token y[b,K] when all K pass).
+ *
+ * Conventions.  Every function returns an aj_status and never throws, aborts or traps the GPU.
+ * All tensors are caller-owned, contiguous, row-major.  "device" pointers are CUDA device
+ * memory on the handle's device; "host" pointers are ordinary (preferably pinned) host memory.
+ * Nothing the caller passes is retained after the enqueued work has run.  aj_verify and
+ * aj_verify_host enqueue work on the given stream and do not synchronise it unless stated.
+ */
+#ifndef AJ_VERIFY_H
+#define AJ_VERIFY_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct aj_handle_s *aj_handle;
+
+typedef enum {
+    AJ_OK = 0,
+    AJ_ERR_INVALID_ARG = 1, /* NULL where required, size out of range, shape differs from the handle's */
+    AJ_ERR_UNSUPPORTED = 2, /* a valid request this build has no kernel for (alignment, layout) */
+    AJ_ERR_WORKSPACE = 3,   /* B or K exceeds what the handle was created for */
+    AJ_ERR_CUDA = 4,        /* a CUDA runtime or driver call failed (no device, out of memory, ...) */
+    AJ_ERR_TIMEOUT = 5,     /* a bounded wait inside a kernel ran out; outputs of that call are invalid */
+    AJ_ERR_NOT_SM100 = 6    /* the device is not compute capability 10.x */
+} aj_status;
+
+typedef enum { AJ_BF16 = 0, AJ_F32 = 1 } aj_dtype; /* storage type of h_target, h_draft and W_lm */
+
+typedef enum {
+    AJ_W_VD = 0, /* W_lm stored row-major [V, d]: one contiguous row per vocabulary entry */
+    AJ_W_DV = 1  /* W_lm stored row-major [d, V] */
+} aj_w_layout;
+
+enum {
+    AJ_FLAG_FORCE_SIMT = 1u,  /* use the plain fp32-accumulate CUDA-core kernel for the projection */
+    AJ_FLAG_TIME_KERNELS = 2u /* record CUDA events around the projection kernel (see aj_last_gemm_ms) */
+};
+
+/*
+ * Create a handle for fixed model dimensions on CUDA device `device`.
+ *   max_B, max_K  largest batch and window a later call may use (1 <= K <= 1024)
+ *   d, d_draft, V target hidden width, draft hidden width (0 = the judge sees target features
+ *                 only, the paper's vLLM variant, Appendix D), vocabulary size
+ *   dtype, layout storage of the hidden states and of W_lm
+ * The handle owns a small device workspace: 8 bytes per row (max_B*(max_K+1)) for the per-row
+ * packed (max, argmax) keys, a status word, and staging buffers for aj_verify_host.  This is the
+ * only place memory is allocated.  AJ_BF16 needs d % 8 == 0 and d_draft % 8 == 0; the tensor-core
+ * path needs AJ_BF16, AJ_W_VD and d % 64 == 0, anything else runs on the CUDA-core kernel.
+ * Errors: AJ_ERR_INVALID_ARG, AJ_ERR_UNSUPPORTED, AJ_ERR_CUDA, AJ_ERR_NOT_SM100.
+ */
+aj_status aj_create(aj_handle *out, int device, int max_B, int max_K, int d, int d_draft, int V,
+                    aj_dtype dtype, aj_w_layout layout, unsigned flags);
+
+/*
+ * One verify-and-judge cycle (Sections 2 and 3.3), device buffers, asynchronous on `cuda_stream`.
+ *   h_target   [B, K+1, d]        device, dtype of the handle, 16-byte aligned
+ *   h_draft    [B, K+1, d_draft]  device, row 0 of each sequence is never read; NULL iff d_draft == 0
+ *   W_lm       d x V              device, layout of the handle, 16-byte aligned
+ *   draft_tok  [B, K] int32       device; ids outside [0,V) are data, they never match
+ *   judge_w    [d_draft + d] f32  device, ordered [draft features ; target features]
+ *   judge_b, tau                  classifier bias and decision threshold, by value
+ *   B, K, d, V                    this call's batch and window; d and V must equal the handle's
+ *   accept_len [B] int32 out      in [0, K]
+ *   next_tok   [B] int32 out      in [0, V)
+ *   target_tok [B, K+1] int32 out optional (NULL ok): y
+ *   top1_val   [B, K+1] f32 out   optional: the winning logit of each row (fp32 accumulate)
+ *   judge_p    [B, K] f32 out     optional: p at every mismatching position, NaN elsewhere
+ *   cuda_stream                   a cudaStream_t (NULL = default stream)
+ * Outputs are valid once the stream has reached the end of the enqueued work.  The return value
+ * covers what the host can see; a kernel-side timeout shows up in aj_last_status.
+ * Calls on one handle share its workspace: calls that overlap on the GPU race.
+ * Errors: AJ_ERR_INVALID_ARG (nothing enqueued), AJ_ERR_WORKSPACE, AJ_ERR_UNSUPPORTED, AJ_ERR_CUDA.
+ */
+aj_status aj_verify(aj_handle h, const void *h_target, const void *h_draft, const void *W_lm,
+                    const int32_t *draft_tok, const float *judge_w, float judge_b, float tau,
+                    int B, int K, int d, int V,
+                    int32_t *accept_len, int32_t *next_tok, int32_t *target_tok,
+                    float *top1_val, float *judge_p, void *cuda_stream);
+
+/*
+ * The same cycle for a caller whose per-cycle tensors live in host memory: h_target, h_draft and
+ * draft_tok are HOST pointers and are copied to the handle's staging buffers; accept_len and
+ * next_tok (and target_tok, if not NULL) are HOST pointers and are copied back.  W_lm and judge_w
+ * are model parameters and stay DEVICE pointers.  The call synchronises `cuda_stream` before it
+ * returns, so the host outputs are valid on return.
+ */
+aj_status aj_verify_host(aj_handle h, const void *h_target_host, const void *h_draft_host,
+                         const void *W_lm, const int32_t *draft_tok_host, const float *judge_w,
+                         float judge_b, float tau, int B, int K, int d, int V,
+                         int32_t *accept_len_host, int32_t *next_tok_host, int32_t *target_tok_host,
+                         void *cuda_stream);
+
+/*
+ * Device-side status of the calls made so far on this handle: AJ_OK, or AJ_ERR_TIMEOUT if a
+ * bounded wait in a kernel gave up.  Synchronises the handle's device; reading clears the word.
+ */
+aj_status aj_last_status(aj_handle h);
+
+/*
+ * With AJ_FLAG_TIME_KERNELS: duration in milliseconds of the projection kernel (the fused
+ * LM-head GEMM + argmax) of the most recent call, from CUDA events recorded on that call's stream
+ * directly around the launch.  Waits for that kernel to finish.  AJ_ERR_INVALID_ARG without the flag.
+ */
+aj_status aj_last_gemm_ms(aj_handle h, float *ms);
+
+/* Number of kernels (and memset nodes) the most recent aj_verify / aj_verify_host call launched. */
+int aj_last_launch_count(aj_handle h);
+
+/* Name of the projection kernel configuration the most recent call used, e.g. "umma_128x256". */
+const char *aj_last_gemm_path(aj_handle h);
+
+/* Free the handle and its workspace.  The caller must have synchronised all work using it. */
+aj_status aj_destroy(aj_handle h);
+
+const char *aj_status_string(aj_status s);
+const char *aj_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AJ_VERIFY_H */

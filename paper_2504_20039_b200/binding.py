@@ -1,0 +1,145 @@
+"""ctypes binding of the aj_verify C-ABI (include/aj_verify.h).
+
+Argument marshalling only: every step of the verify-and-judge cycle runs in the CUDA library.
+There is no CPU fallback; loading fails loudly if the library has not been built.
+torch is used by callers for device memory and streams; this module only needs `data_ptr()`.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libaj_verify.so")
+
+AJ_OK, AJ_ERR_INVALID_ARG, AJ_ERR_UNSUPPORTED, AJ_ERR_WORKSPACE, AJ_ERR_CUDA, AJ_ERR_TIMEOUT, AJ_ERR_NOT_SM100 = range(7)
+AJ_BF16, AJ_F32 = 0, 1
+AJ_W_VD, AJ_W_DV = 0, 1
+AJ_FLAG_FORCE_SIMT, AJ_FLAG_TIME_KERNELS = 1, 2
+
+EXPORTS = (
+    "aj_create", "aj_verify", "aj_verify_host", "aj_last_status", "aj_last_gemm_ms", "aj_last_launch_count",
+    "aj_last_gemm_path", "aj_destroy", "aj_status_string", "aj_version",
+)
+
+_lib = None
+
+
+class AjError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__(f"{what}: {status_string(status)} ({status})")
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded CUDA library; raises if it has not been built (python -m paper_2504_20039_b200.build)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(
+                f"{LIB_PATH} is missing: build the CUDA library first "
+                "(python __graft_entry__.py build, or python paper_2504_20039_b200/build.py)"
+            )
+        L = ctypes.CDLL(LIB_PATH)
+        vp, ci, cf, cu = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_uint
+        L.aj_create.argtypes = [ctypes.POINTER(vp), ci, ci, ci, ci, ci, ci, ci, ci, cu]
+        L.aj_create.restype = ci
+        L.aj_verify.argtypes = [vp, vp, vp, vp, vp, vp, cf, cf, ci, ci, ci, ci, vp, vp, vp, vp, vp, vp]
+        L.aj_verify.restype = ci
+        L.aj_verify_host.argtypes = [vp, vp, vp, vp, vp, vp, cf, cf, ci, ci, ci, ci, vp, vp, vp, vp]
+        L.aj_verify_host.restype = ci
+        L.aj_last_status.argtypes = [vp]
+        L.aj_last_status.restype = ci
+        L.aj_last_gemm_ms.argtypes = [vp, ctypes.POINTER(cf)]
+        L.aj_last_gemm_ms.restype = ci
+        L.aj_last_launch_count.argtypes = [vp]
+        L.aj_last_launch_count.restype = ci
+        L.aj_last_gemm_path.argtypes = [vp]
+        L.aj_last_gemm_path.restype = ctypes.c_char_p
+        L.aj_destroy.argtypes = [vp]
+        L.aj_destroy.restype = ci
+        L.aj_status_string.argtypes = [ci]
+        L.aj_status_string.restype = ctypes.c_char_p
+        L.aj_version.argtypes = []
+        L.aj_version.restype = ctypes.c_char_p
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().aj_status_string(int(status)).decode()
+
+
+def version() -> str:
+    return lib().aj_version().decode()
+
+
+def _ptr(t):
+    """Device or host address of a torch tensor / numpy array / int / None."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    if hasattr(t, "data_ptr"):
+        return t.data_ptr()
+    return t.ctypes.data
+
+
+class Handle:
+    """aj_create / aj_destroy as an object; methods mirror the C entry points."""
+
+    def __init__(self, device: int, max_B: int, max_K: int, d: int, d_draft: int, V: int,
+                 dtype: int = AJ_BF16, layout: int = AJ_W_VD, flags: int = 0):
+        self._h = ctypes.c_void_p()
+        st = lib().aj_create(ctypes.byref(self._h), device, max_B, max_K, d, d_draft, V, dtype, layout, flags)
+        if st != AJ_OK:
+            self._h = ctypes.c_void_p()
+            raise AjError(st, "aj_create")
+        self.d, self.V, self.d_draft = d, V, d_draft
+
+    def verify(self, h_target, h_draft, W_lm, draft_tok, judge_w, judge_b: float, tau: float, B: int, K: int,
+               accept_len, next_tok, target_tok=None, top1_val=None, judge_p=None, stream: int = 0, check: bool = True) -> int:
+        """aj_verify: device tensors in, device tensors out, asynchronous on `stream` (a cudaStream_t as int)."""
+        st = lib().aj_verify(self._h, _ptr(h_target), _ptr(h_draft), _ptr(W_lm), _ptr(draft_tok), _ptr(judge_w),
+                             float(judge_b), float(tau), B, K, self.d, self.V, _ptr(accept_len), _ptr(next_tok),
+                             _ptr(target_tok), _ptr(top1_val), _ptr(judge_p), stream or None)
+        if check and st != AJ_OK:
+            raise AjError(st, "aj_verify")
+        return st
+
+    def verify_host(self, h_target, h_draft, W_lm, draft_tok, judge_w, judge_b: float, tau: float, B: int, K: int,
+                    accept_len, next_tok, target_tok=None, stream: int = 0, check: bool = True) -> int:
+        """aj_verify_host: per-cycle tensors in host memory, W_lm and judge_w on the device; synchronous."""
+        st = lib().aj_verify_host(self._h, _ptr(h_target), _ptr(h_draft), _ptr(W_lm), _ptr(draft_tok), _ptr(judge_w),
+                                  float(judge_b), float(tau), B, K, self.d, self.V, _ptr(accept_len), _ptr(next_tok),
+                                  _ptr(target_tok), stream or None)
+        if check and st != AJ_OK:
+            raise AjError(st, "aj_verify_host")
+        return st
+
+    def last_status(self) -> int:
+        return lib().aj_last_status(self._h)
+
+    def last_gemm_ms(self) -> float:
+        ms = ctypes.c_float()
+        st = lib().aj_last_gemm_ms(self._h, ctypes.byref(ms))
+        if st != AJ_OK:
+            raise AjError(st, "aj_last_gemm_ms")
+        return float(ms.value)
+
+    def last_launch_count(self) -> int:
+        return lib().aj_last_launch_count(self._h)
+
+    def last_gemm_path(self) -> str:
+        return lib().aj_last_gemm_path(self._h).decode()
+
+    def destroy(self) -> None:
+        if self._h:
+            lib().aj_destroy(self._h)
+            self._h = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass

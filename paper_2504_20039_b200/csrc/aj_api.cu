@@ -1,0 +1,344 @@
+// Host side of the C-ABI: argument checks, workspace, tensor maps, stream-ordered launches.
+// One cycle = clear the keys, projection + argmax kernel, judge + scan kernel; no host
+// synchronisation and no allocation inside aj_verify.
+#include "../../include/aj_verify.h"
+#include "aj_internal.cuh"
+
+#include <new>
+
+namespace {
+
+using namespace aj;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct TmapSlot {
+    const void *ptr = nullptr;
+    long long rows = 0;
+    int box_rows = 0;
+    unsigned long long stamp = 0;
+    CUtensorMap map;
+};
+
+constexpr int TMAP_SLOTS = 8;
+
+}  // namespace
+
+struct aj_handle_s {
+    int device = 0;
+    int max_B = 0, max_K = 0, d = 0, d_draft = 0, V = 0;
+    int dtype = 0, layout = 0;
+    unsigned flags = 0;
+    int num_sms = 0;
+    bool umma_ok = false;
+    unsigned long long *keys = nullptr;
+    int *status = nullptr;
+    // staging for aj_verify_host
+    void *st_ht = nullptr, *st_hd = nullptr;
+    int32_t *st_tok = nullptr, *st_acc = nullptr, *st_next = nullptr, *st_tt = nullptr;
+    EncodeTiledFn encode = nullptr;
+    TmapSlot slots[TMAP_SLOTS];
+    unsigned long long stamp = 0;
+    cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+    bool timed = false;
+    int last_launches = 0;
+    const char *last_path = "none";
+};
+
+namespace {
+
+size_t elem_size(int dtype) { return dtype == AJ_BF16 ? 2 : 4; }
+
+class DeviceGuard {
+   public:
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev_) != cudaSuccess) prev_ = -1;
+        if (prev_ != dev) ok_ = cudaSetDevice(dev) == cudaSuccess;
+        changed_ = ok_ && prev_ != dev;
+    }
+    ~DeviceGuard() {
+        if (changed_ && prev_ >= 0) cudaSetDevice(prev_);
+    }
+    bool ok() const { return ok_; }
+
+   private:
+    int prev_ = -1;
+    bool ok_ = true, changed_ = false;
+};
+
+// A tensor map over `rows` rows of `d` bf16 elements, box 64 columns x box_rows rows, 128-byte
+// swizzle; rows past the end read as zero.  Cached per (pointer, rows, box).
+const CUtensorMap *get_tmap(aj_handle h, const void *ptr, long long rows, int box_rows) {
+    TmapSlot *victim = &h->slots[0];
+    for (auto &s : h->slots) {
+        if (s.ptr == ptr && s.rows == rows && s.box_rows == box_rows) {
+            s.stamp = ++h->stamp;
+            return &s.map;
+        }
+        if (s.stamp < victim->stamp) victim = &s;
+    }
+    cuuint64_t dims[2] = {(cuuint64_t)h->d, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)h->d * 2};
+    cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = h->encode(&victim->map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), dims, strides, box,
+                           estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        victim->ptr = nullptr;
+        return nullptr;
+    }
+    victim->ptr = ptr;
+    victim->rows = rows;
+    victim->box_rows = box_rows;
+    victim->stamp = ++h->stamp;
+    return &victim->map;
+}
+
+int choose_bn(int M) { return M <= 128 ? 128 : 256; }
+
+aj_status check_call(aj_handle h, const void *h_target, const void *h_draft, const void *W_lm, const int32_t *draft_tok,
+                     const float *judge_w, int B, int K, int d, int V, const int32_t *accept_len,
+                     const int32_t *next_tok) {
+    if (!h) return AJ_ERR_INVALID_ARG;
+    if (!h_target || !W_lm || !draft_tok || !judge_w || !accept_len || !next_tok) return AJ_ERR_INVALID_ARG;
+    if ((h->d_draft > 0) != (h_draft != nullptr)) return AJ_ERR_INVALID_ARG;
+    if (B < 1 || K < 1 || d != h->d || V != h->V) return AJ_ERR_INVALID_ARG;
+    if (B > h->max_B || K > h->max_K) return AJ_ERR_WORKSPACE;
+    return AJ_OK;
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+}  // namespace
+
+extern "C" {
+
+const char *aj_version(void) { return "aj_verify 0.1 (sm_100a)"; }
+
+const char *aj_status_string(aj_status s) {
+    switch (s) {
+        case AJ_OK: return "ok";
+        case AJ_ERR_INVALID_ARG: return "invalid argument";
+        case AJ_ERR_UNSUPPORTED: return "unsupported configuration";
+        case AJ_ERR_WORKSPACE: return "batch or window exceeds the handle's workspace";
+        case AJ_ERR_CUDA: return "CUDA call failed";
+        case AJ_ERR_TIMEOUT: return "a bounded wait in a kernel ran out";
+        case AJ_ERR_NOT_SM100: return "device is not compute capability 10.x";
+    }
+    return "unknown status";
+}
+
+aj_status aj_create(aj_handle *out, int device, int max_B, int max_K, int d, int d_draft, int V, aj_dtype dtype,
+                    aj_w_layout layout, unsigned flags) {
+    if (!out) return AJ_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (device < 0 || max_B < 1 || max_K < 1 || max_K > 1024 || d < 1 || d_draft < 0 || V < 1) return AJ_ERR_INVALID_ARG;
+    if (dtype != AJ_BF16 && dtype != AJ_F32) return AJ_ERR_INVALID_ARG;
+    if (layout != AJ_W_VD && layout != AJ_W_DV) return AJ_ERR_INVALID_ARG;
+    if (flags & ~(AJ_FLAG_FORCE_SIMT | AJ_FLAG_TIME_KERNELS)) return AJ_ERR_INVALID_ARG;
+    if ((long long)max_B * (max_K + 1) > (1ll << 24)) return AJ_ERR_INVALID_ARG;
+    if (dtype == AJ_BF16 && (d % 8 != 0 || d_draft % 8 != 0)) return AJ_ERR_UNSUPPORTED;
+
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess || device >= count) {
+        cudaGetLastError();
+        return AJ_ERR_CUDA;
+    }
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return AJ_ERR_CUDA;
+    if (prop.major != 10) return AJ_ERR_NOT_SM100;
+    DeviceGuard guard(device);
+    if (!guard.ok()) return AJ_ERR_CUDA;
+
+    aj_handle h = new (std::nothrow) aj_handle_s;
+    if (!h) return AJ_ERR_CUDA;
+    h->device = device;
+    h->max_B = max_B;
+    h->max_K = max_K;
+    h->d = d;
+    h->d_draft = d_draft;
+    h->V = V;
+    h->dtype = dtype;
+    h->layout = layout;
+    h->flags = flags;
+    h->num_sms = prop.multiProcessorCount;
+    h->umma_ok = dtype == AJ_BF16 && layout == AJ_W_VD && d % 64 == 0 && !(flags & AJ_FLAG_FORCE_SIMT);
+
+    const size_t max_M = (size_t)max_B * (max_K + 1);
+    const size_t esz = elem_size(dtype);
+    bool ok = cudaMalloc(&h->keys, max_M * sizeof(unsigned long long)) == cudaSuccess &&
+              cudaMalloc(&h->status, 256) == cudaSuccess && cudaMemset(h->status, 0, 256) == cudaSuccess &&
+              cudaMalloc(&h->st_ht, max_M * d * esz) == cudaSuccess &&
+              (d_draft == 0 || cudaMalloc(&h->st_hd, max_M * d_draft * esz) == cudaSuccess) &&
+              cudaMalloc(&h->st_tok, (size_t)max_B * max_K * 4) == cudaSuccess &&
+              cudaMalloc(&h->st_acc, (size_t)max_B * 4) == cudaSuccess &&
+              cudaMalloc(&h->st_next, (size_t)max_B * 4) == cudaSuccess && cudaMalloc(&h->st_tt, max_M * 4) == cudaSuccess;
+    if (ok && (flags & AJ_FLAG_TIME_KERNELS))
+        ok = cudaEventCreate(&h->ev0) == cudaSuccess && cudaEventCreate(&h->ev1) == cudaSuccess;
+    if (ok && h->umma_ok) {
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        ok = cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &fn, 12000, cudaEnableDefault, &qres) == cudaSuccess &&
+             qres == cudaDriverEntryPointSuccess && fn != nullptr;
+        h->encode = reinterpret_cast<EncodeTiledFn>(fn);
+        if (ok) ok = umma_prepare() == cudaSuccess;
+    }
+    if (!ok) {
+        cudaGetLastError();
+        aj_destroy(h);
+        return AJ_ERR_CUDA;
+    }
+    *out = h;
+    return AJ_OK;
+}
+
+aj_status aj_destroy(aj_handle h) {
+    if (!h) return AJ_ERR_INVALID_ARG;
+    DeviceGuard guard(h->device);
+    cudaFree(h->keys);
+    cudaFree(h->status);
+    cudaFree(h->st_ht);
+    cudaFree(h->st_hd);
+    cudaFree(h->st_tok);
+    cudaFree(h->st_acc);
+    cudaFree(h->st_next);
+    cudaFree(h->st_tt);
+    if (h->ev0) cudaEventDestroy(h->ev0);
+    if (h->ev1) cudaEventDestroy(h->ev1);
+    delete h;
+    return AJ_OK;
+}
+
+aj_status aj_verify(aj_handle h, const void *h_target, const void *h_draft, const void *W_lm, const int32_t *draft_tok,
+                    const float *judge_w, float judge_b, float tau, int B, int K, int d, int V, int32_t *accept_len,
+                    int32_t *next_tok, int32_t *target_tok, float *top1_val, float *judge_p, void *cuda_stream) {
+    aj_status st = check_call(h, h_target, h_draft, W_lm, draft_tok, judge_w, B, K, d, V, accept_len, next_tok);
+    if (st != AJ_OK) return st;
+    if (h->dtype == AJ_BF16 && (!aligned16(h_target) || !aligned16(W_lm) || (h_draft && !aligned16(h_draft))))
+        return AJ_ERR_UNSUPPORTED;
+    DeviceGuard guard(h->device);
+    if (!guard.ok()) return AJ_ERR_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const int M = B * (K + 1);
+    h->last_launches = 0;
+    h->timed = false;
+
+    if (cudaMemsetAsync(h->keys, 0, (size_t)M * sizeof(unsigned long long), stream) != cudaSuccess) return AJ_ERR_CUDA;
+    h->last_launches++;
+
+    GemmArgs g;
+    g.h = h_target;
+    g.W = W_lm;
+    g.M = M;
+    g.d = d;
+    g.V = V;
+    g.dtype = h->dtype;
+    g.w_layout = h->layout;
+    g.keys = h->keys;
+    g.status = h->status;
+
+    const bool time_it = (h->flags & AJ_FLAG_TIME_KERNELS) != 0;
+    if (time_it && cudaEventRecord(h->ev0, stream) != cudaSuccess) return AJ_ERR_CUDA;
+    cudaError_t e;
+    if (h->umma_ok) {
+        UmmaPlan p;
+        p.bn = choose_bn(M);
+        const CUtensorMap *th = get_tmap(h, h_target, M, 128);
+        const CUtensorMap *tw = get_tmap(h, W_lm, V, p.bn);
+        if (!th || !tw) return AJ_ERR_CUDA;
+        p.tmap_h = *th;
+        p.tmap_w = *tw;
+        const int n_m = (M + 127) / 128, n_v = (V + p.bn - 1) / p.bn;
+        const long long tiles = (long long)n_m * n_v;
+        p.grid = (int)(tiles < h->num_sms ? tiles : h->num_sms);
+        e = launch_umma_gemm_argmax(g, p, stream);
+        h->last_path = umma_path_name(p.bn);
+    } else {
+        e = launch_simt_gemm_argmax(g, h->num_sms, stream);
+        h->last_path = "simt";
+    }
+    if (e != cudaSuccess) return AJ_ERR_CUDA;
+    h->last_launches++;
+    if (time_it) {
+        if (cudaEventRecord(h->ev1, stream) != cudaSuccess) return AJ_ERR_CUDA;
+        h->timed = true;
+    }
+
+    JudgeArgs j;
+    j.keys = h->keys;
+    j.h_target = h_target;
+    j.h_draft = h_draft;
+    j.draft_tok = draft_tok;
+    j.judge_w = judge_w;
+    j.judge_b = judge_b;
+    j.tau = tau;
+    j.B = B;
+    j.K = K;
+    j.d = d;
+    j.d_draft = h->d_draft;
+    j.dtype = h->dtype;
+    j.accept_len = accept_len;
+    j.next_tok = next_tok;
+    j.target_tok = target_tok;
+    j.top1_val = top1_val;
+    j.judge_p = judge_p;
+    if (launch_judge_scan(j, stream) != cudaSuccess) return AJ_ERR_CUDA;
+    h->last_launches++;
+    return AJ_OK;
+}
+
+aj_status aj_verify_host(aj_handle h, const void *h_target_host, const void *h_draft_host, const void *W_lm,
+                         const int32_t *draft_tok_host, const float *judge_w, float judge_b, float tau, int B, int K,
+                         int d, int V, int32_t *accept_len_host, int32_t *next_tok_host, int32_t *target_tok_host,
+                         void *cuda_stream) {
+    aj_status st = check_call(h, h_target_host, h_draft_host, W_lm, draft_tok_host, judge_w, B, K, d, V, accept_len_host,
+                              next_tok_host);
+    if (st != AJ_OK) return st;
+    DeviceGuard guard(h->device);
+    if (!guard.ok()) return AJ_ERR_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    const size_t M = (size_t)B * (K + 1), esz = elem_size(h->dtype);
+    bool ok = cudaMemcpyAsync(h->st_ht, h_target_host, M * d * esz, cudaMemcpyHostToDevice, stream) == cudaSuccess &&
+              (h->d_draft == 0 ||
+               cudaMemcpyAsync(h->st_hd, h_draft_host, M * h->d_draft * esz, cudaMemcpyHostToDevice, stream) == cudaSuccess) &&
+              cudaMemcpyAsync(h->st_tok, draft_tok_host, (size_t)B * K * 4, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    if (!ok) return AJ_ERR_CUDA;
+    st = aj_verify(h, h->st_ht, h->d_draft ? h->st_hd : nullptr, W_lm, h->st_tok, judge_w, judge_b, tau, B, K, d, V, h->st_acc,
+                   h->st_next, target_tok_host ? h->st_tt : nullptr, nullptr, nullptr, cuda_stream);
+    if (st != AJ_OK) return st;
+    const int launches = h->last_launches;
+    ok = cudaMemcpyAsync(accept_len_host, h->st_acc, (size_t)B * 4, cudaMemcpyDeviceToHost, stream) == cudaSuccess &&
+         cudaMemcpyAsync(next_tok_host, h->st_next, (size_t)B * 4, cudaMemcpyDeviceToHost, stream) == cudaSuccess &&
+         (!target_tok_host || cudaMemcpyAsync(target_tok_host, h->st_tt, M * 4, cudaMemcpyDeviceToHost, stream) == cudaSuccess) &&
+         cudaStreamSynchronize(stream) == cudaSuccess;
+    h->last_launches = launches;
+    return ok ? AJ_OK : AJ_ERR_CUDA;
+}
+
+aj_status aj_last_status(aj_handle h) {
+    if (!h) return AJ_ERR_INVALID_ARG;
+    DeviceGuard guard(h->device);
+    if (!guard.ok()) return AJ_ERR_CUDA;
+    int word = 0;
+    if (cudaDeviceSynchronize() != cudaSuccess) return AJ_ERR_CUDA;
+    if (cudaMemcpy(&word, h->status, sizeof word, cudaMemcpyDeviceToHost) != cudaSuccess) return AJ_ERR_CUDA;
+    if (word != 0 && cudaMemset(h->status, 0, sizeof word) != cudaSuccess) return AJ_ERR_CUDA;
+    return word == DEV_TIMEOUT ? AJ_ERR_TIMEOUT : (word == 0 ? AJ_OK : AJ_ERR_CUDA);
+}
+
+aj_status aj_last_gemm_ms(aj_handle h, float *ms) {
+    if (!h || !ms || !(h->flags & AJ_FLAG_TIME_KERNELS) || !h->timed) return AJ_ERR_INVALID_ARG;
+    DeviceGuard guard(h->device);
+    if (cudaEventSynchronize(h->ev1) != cudaSuccess) return AJ_ERR_CUDA;
+    if (cudaEventElapsedTime(ms, h->ev0, h->ev1) != cudaSuccess) return AJ_ERR_CUDA;
+    return AJ_OK;
+}
+
+int aj_last_launch_count(aj_handle h) { return h ? h->last_launches : 0; }
+
+const char *aj_last_gemm_path(aj_handle h) { return h ? h->last_path : "none"; }
+
+}  // extern "C"

@@ -1,0 +1,169 @@
+"""Helpers for the GPU parity tests: move seeded inputs to the device, call the C-ABI through
+the binding, and compare with the CPU oracle under the stated tolerances."""
+from __future__ import annotations
+
+from dataclasses import dataclass
+
+import numpy as np
+
+import aj_inputs as gen
+
+# Tolerances (floating point: bf16 or fp32 inputs, fp32 accumulate on the device, fp64 in the oracle)
+TOL_LOGIT = 2e-2   # |winning logit (device) - winning logit (oracle)|
+TOL_P = 1e-4       # |judge probability (device) - (oracle)|
+GAP_EXEMPT = 1e-2  # a row whose top-1/top-2 gap is at most this may legitimately pick the runner-up
+
+
+def to_device(a: np.ndarray, dtype: int, device="cuda:0"):
+    import torch
+
+    if a is None:
+        return None
+    if dtype == gen.BF16 and a.dtype == np.uint16:
+        return torch.from_numpy(a.view(np.int16)).to(device).view(torch.bfloat16)
+    return torch.from_numpy(a).to(device)
+
+
+@dataclass
+class GpuResult:
+    accept_len: np.ndarray
+    next_tok: np.ndarray
+    target_tok: np.ndarray
+    top1: np.ndarray
+    judge_p: np.ndarray
+    path: str
+    launches: int
+
+
+class DeviceCase:
+    """Inputs of one workload resident on the device, plus a handle."""
+
+    def __init__(self, cfg: gen.Config, W, ht, hd, w, layout: int = 0, flags: int = 0, max_B=None, max_K=None):
+        import torch
+
+        import paper_2504_20039_b200 as aj
+
+        self.cfg = cfg
+        self.aj = aj
+        self.torch = torch
+        self.W = W if hasattr(W, "data_ptr") else to_device(W, cfg.dtype)
+        self.ht = to_device(ht, cfg.dtype)
+        self.hd = to_device(hd, cfg.dtype)
+        self.w = to_device(w, gen.F32)
+        self.handle = aj.Handle(0, max_B or cfg.B, max_K or cfg.K, cfg.d, cfg.d_draft, cfg.V, cfg.dtype, layout, flags)
+
+    def run(self, tok: np.ndarray, tau: float, judge_b: float | None = None, B=None, K=None, seqs=slice(None), fill=None) -> GpuResult:
+        torch = self.torch
+        cfg = self.cfg
+        ht = self.ht[seqs]
+        hd = None if self.hd is None else self.hd[seqs]
+        B = ht.shape[0] if B is None else B
+        K = cfg.K if K is None else K
+        tok_d = torch.from_numpy(np.ascontiguousarray(tok, dtype=np.int32)).cuda()
+        i32 = dict(dtype=torch.int32, device="cuda")
+        f32 = dict(dtype=torch.float32, device="cuda")
+        fill_i = -7 if fill is None else fill
+        acc = torch.full((B,), fill_i, **i32)
+        nxt = torch.full((B,), fill_i, **i32)
+        tt = torch.full((B, K + 1), fill_i, **i32)
+        top1 = torch.full((B, K + 1), 12345.0, **f32)
+        jp = torch.full((B, K), 12345.0, **f32)
+        stream = torch.cuda.current_stream().cuda_stream
+        self.handle.verify(ht.contiguous(), None if hd is None else hd.contiguous(), self.W, tok_d, self.w,
+                           cfg.judge_b if judge_b is None else judge_b, tau, B, K, acc, nxt, tt, top1, jp, stream=stream)
+        torch.cuda.synchronize()
+        st = self.handle.last_status()
+        assert st == self.aj.AJ_OK, self.aj.status_string(st)
+        return GpuResult(acc.cpu().numpy(), nxt.cpu().numpy(), tt.cpu().numpy(), top1.cpu().numpy(), jp.cpu().numpy(),
+                         self.handle.last_gemm_path(), self.handle.last_launch_count())
+
+    def close(self):
+        self.handle.destroy()
+
+
+@dataclass
+class ParityReport:
+    rows: int = 0
+    rows_exempt: int = 0
+    seqs: int = 0
+    seqs_exempt: int = 0
+    max_logit_err: float = 0.0
+    max_p_err: float = 0.0
+
+
+def check_parity(orc_res, gpu: GpuResult, tok: np.ndarray, tau: float, seqs=None) -> ParityReport:
+    """Element-by-element comparison of a device result with the oracle's.
+
+    Integer outputs must be bit-exact except where floating point legitimately decides
+    otherwise: a row whose top-1/top-2 gap is at most GAP_EXEMPT may return the runner-up, and
+    a judged position with |p - tau| <= TOL_P may fall on the other side of the threshold.  A
+    sequence is exempt from exactness of accept_len / next_tok only if such a row or position
+    lies at or before the oracle's stop.  Winning logits and probabilities are always compared.
+    `seqs`: indices into the device batch that the oracle rows correspond to (default: all).
+    """
+    rep = ParityReport()
+    idx = np.arange(gpu.accept_len.shape[0]) if seqs is None else np.asarray(seqs)
+    B, R = orc_res.target_tok.shape
+    K = R - 1
+    tok = np.asarray(tok)
+    for r, b in enumerate(idx):
+        y_o, y_g = orc_res.target_tok[r], gpu.target_tok[b]
+        close = orc_res.gap[r] <= GAP_EXEMPT
+        rep.rows += R
+        rep.rows_exempt += int(close.sum())
+        bad = (y_o != y_g) & ~close
+        assert not bad.any(), f"seq {b}: target_tok differs at rows {np.nonzero(bad)[0]} (gaps {orc_res.gap[r][bad]})"
+        err = np.abs(gpu.top1[b].astype(np.float64) - orc_res.top1[r])
+        rep.max_logit_err = max(rep.max_logit_err, float(err.max()))
+        assert err.max() <= TOL_LOGIT, f"seq {b}: winning logit off by {err.max()}"
+        # judge probabilities wherever both sides consulted the judge
+        po, pg = orc_res.judge_p[r], gpu.judge_p[b].astype(np.float64)
+        both = ~np.isnan(po) & ~np.isnan(pg)
+        same_rows = y_o[:K] == y_g[:K]
+        assert (np.isnan(po) == np.isnan(pg))[same_rows].all(), f"seq {b}: judge consulted at different positions"
+        if both.any():
+            perr = np.abs(po[both] - pg[both])
+            rep.max_p_err = max(rep.max_p_err, float(perr.max()))
+            assert perr.max() <= TOL_P, f"seq {b}: judge probability off by {perr.max()}"
+        # accept_len / next_tok
+        n = int(orc_res.accept_len[r])
+        upto = slice(0, n + 1)
+        near_tau = (~np.isnan(po[: min(n + 1, K)])) & (np.abs(po[: min(n + 1, K)] - tau) <= TOL_P) & (0.0 < tau < 1.0)
+        exempt = bool(close[upto].any() or near_tau.any())
+        rep.seqs += 1
+        rep.seqs_exempt += int(exempt)
+        if not exempt:
+            assert gpu.accept_len[b] == n, f"seq {b}: accept_len {gpu.accept_len[b]} != {n}"
+            assert gpu.next_tok[b] == orc_res.next_tok[r], f"seq {b}: next_tok {gpu.next_tok[b]} != {orc_res.next_tok[r]}"
+        # what must hold regardless: the device is consistent with its own tokens
+        assert 0 <= gpu.accept_len[b] <= K
+        assert gpu.next_tok[b] == gpu.target_tok[b, gpu.accept_len[b]]
+    return rep
+
+
+def check_self_consistency(gpu: GpuResult, tok: np.ndarray, tau: float, V: int):
+    """Properties that hold at any size without an oracle (Section 2 / 3.3 of the paper):
+    the accepted length is at least the plain greedy first-mismatch length, equals it when
+    nothing is forgiven, is K when everything is, stops only at a mismatch whose p >= tau,
+    and next_tok is the device's own target token at the stop."""
+    B, K = tok.shape
+    y = gpu.target_tok
+    assert ((y >= 0) & (y < V)).all()
+    mism = tok != y[:, :K]
+    vanilla = np.array([int(np.argmax(np.append(m, True))) for m in mism])
+    acc = gpu.accept_len
+    assert ((acc >= vanilla) & (acc <= K)).all()
+    assert (gpu.next_tok == y[np.arange(B), acc]).all()
+    assert (np.isnan(gpu.judge_p) == ~mism).all()
+    if tau <= 0:
+        assert (acc == vanilla).all()
+    if tau >= 1:
+        assert (acc == K).all()
+    for b in range(B):
+        n = int(acc[b])
+        if 0 < tau < 1:
+            if n < K:
+                assert mism[b, n] and not (gpu.judge_p[b, n] < np.float32(tau))
+            forgiven = mism[b, :n]
+            assert (gpu.judge_p[b, :n][forgiven] < np.float32(tau)).all()
+    return vanilla

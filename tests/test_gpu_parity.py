@@ -99,7 +99,7 @@ SHAPES = [
 @pytest.mark.parametrize("flags", [0, 1], ids=["umma", "simt"])
 def test_cut_down_shapes_bf16(shape, flags):
     name, B, K, d, dd, V = shape
-    cfg = gen.Config(name, B=B, K=K, d=d, d_draft=dd, V=V, sigma_w=0.05, match_lo=0.5, match_hi=0.95, seed=3)
+    cfg = gen.Config(name, B=B, K=K, d=d, d_draft=dd, V=V, sigma_W=0.2, sigma_w=0.05, match_lo=0.5, match_hi=0.95, seed=3)
     reps = _full_parity(cfg, (0.0, 0.3, 0.5, 1.0), flags=flags)
     assert all(r.seqs_exempt <= r.seqs // 2 + 1 for r in reps)
 

@@ -1,0 +1,370 @@
+"""Benchmark of the verify-and-judge step (aj_verify) on B200.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2|c3|c4|sweep] [--impl reference]
+
+A step is one whole cycle (clear keys, LM-head projection + argmax, judge + prefix scan) over one
+batch of seeded synthetic inputs shaped like the paper's Llama-3.x pairs.  The headline workload is
+the batch-1 8B-shaped configuration (B=1, K=16, d=4096, V=128256, bf16), the setting the paper's own
+measurements use (batch size 1); the batched 8B- and 70B-shaped configurations are reported under
+"extra" in the same JSON line.  Metric: verified draft positions per second (B*K per cycle).
+
+Rank layout for N > 1: one process per GPU, every rank verifies its own batch against its own copy
+of W_lm (sequences are independent, there is no data-path collective): weak scaling.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import aj_inputs as gen  # noqa: E402
+
+METRIC = "verified_positions_per_s"
+UNIT = "positions/s"
+L2_BYTES = 126 * 1024 * 1024
+
+
+def workload(name: str) -> gen.Config:
+    return {"c2": gen.C2, "c3": gen.C3, "c4": gen.C4}[name]
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ------------------------------------------------------------------------------------ clocks
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while a timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.rows = []
+        self.proc = None
+        self.thread = None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "20", "-i", str(self.gpu)],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), [x.strip() for x in line.split(",")]))
+
+    def __exit__(self, *exc):
+        if self.proc:
+            time.sleep(0.03)
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=2)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+
+    def summary(self, t0: float, t1: float):
+        rows = [r for t, r in self.rows if t0 <= t <= t1 and len(r) >= 7] or [r for _, r in self.rows if len(r) >= 7]
+        if not rows:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        sm = [float(r[0]) for r in rows]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(r[3 + i].lower().startswith("active") for r in rows)]
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": float(rows[0][1]), "power_w_max": max(float(r[2]) for r in rows),
+                "samples": len(rows), "reasons": reasons}
+
+
+# ------------------------------------------------------------------------------- our GPU arm
+
+
+class GpuWorkload:
+    """One workload resident on the device: rotating copies of W_lm, inputs, outputs, handles."""
+
+    def __init__(self, cfg: gen.Config, device: int, w_copies: int, W_host=None):
+        import torch
+
+        import paper_2504_20039_b200 as aj
+
+        self.torch, self.aj, self.cfg = torch, aj, cfg
+        dev = f"cuda:{device}"
+        bf = lambda a: torch.from_numpy(a.view(np.int16)).to(dev).view(torch.bfloat16)
+        W_host = gen.make_W(cfg) if W_host is None else W_host
+        self.W = [bf(W_host)]
+        for _ in range(w_copies - 1):
+            self.W.append(self.W[0].clone())
+        ht, hd = gen.make_hidden(cfg)
+        self.ht_host, self.hd_host = ht, hd
+        self.ht, self.hd = bf(ht), bf(hd)
+        self.w = torch.from_numpy(gen.make_judge(cfg)).to(dev)
+        i32 = dict(dtype=torch.int32, device=dev)
+        self.acc = torch.empty(cfg.B, **i32)
+        self.nxt = torch.empty(cfg.B, **i32)
+        self.tt = torch.empty((cfg.B, cfg.K + 1), **i32)
+        self.handle = aj.Handle(device, cfg.B, cfg.K, cfg.d, cfg.d_draft, cfg.V, aj.AJ_BF16, aj.AJ_W_VD, 0)
+        self.handle_t = aj.Handle(device, cfg.B, cfg.K, cfg.d, cfg.d_draft, cfg.V, aj.AJ_BF16, aj.AJ_W_VD, aj.AJ_FLAG_TIME_KERNELS)
+        # draft tokens planted against the device's own greedy tokens (a benchmark input, never an oracle input)
+        self.tok = torch.from_numpy(gen.random_draft_tokens(cfg)).to(dev)
+        self.step(self.handle, 0)
+        torch.cuda.synchronize()
+        self.tok_host = gen.plant_draft_tokens(cfg, self.tt.cpu().numpy())
+        self.tok = torch.from_numpy(self.tok_host).to(dev)
+        self.i = 0
+
+    def step(self, handle, i):
+        cfg = self.cfg
+        handle.verify(self.ht, self.hd, self.W[i % len(self.W)], self.tok, self.w, cfg.judge_b, cfg.tau, cfg.B, cfg.K,
+                      self.acc, self.nxt, self.tt, stream=self.torch.cuda.current_stream().cuda_stream)
+
+    def run(self, handle, steps):
+        for _ in range(steps):
+            self.step(handle, self.i)
+            self.i += 1
+
+    def timed(self, handle, steps, barrier):
+        torch = self.torch
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        torch.cuda.synchronize()
+        t0 = time.time()
+        e0.record()
+        self.run(handle, steps)
+        e1.record()
+        torch.cuda.synchronize()
+        t1 = time.time()
+        barrier()
+        return e0.elapsed_time(e1), t0, t1
+
+    def e2e(self, steps, warmup):
+        """The same cycle through aj_verify_host: per-cycle tensors start in pinned host memory."""
+        torch, cfg = self.torch, self.cfg
+        pin = lambda a: torch.from_numpy(a.view(np.int16) if a.dtype == np.uint16 else a).pin_memory()
+        ht, hd, tok = pin(self.ht_host), pin(self.hd_host), pin(self.tok_host)
+        acc = torch.empty(cfg.B, dtype=torch.int32).pin_memory()
+        nxt = torch.empty(cfg.B, dtype=torch.int32).pin_memory()
+        stream = torch.cuda.current_stream().cuda_stream
+        call = lambda i: self.handle.verify_host(ht, hd, self.W[i % len(self.W)], tok, self.w, cfg.judge_b, cfg.tau, cfg.B, cfg.K,
+                                                 acc, nxt, None, stream=stream)
+        for i in range(warmup):
+            call(i)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for i in range(steps):
+            call(i)  # synchronous: returns when accept_len / next_tok are on the host
+        dt = time.perf_counter() - t0
+        h2d = ht.numel() * 2 + hd.numel() * 2 + tok.numel() * 4
+        d2h = 8 * cfg.B
+        return dt / steps, h2d, d2h
+
+    def close(self):
+        self.handle.destroy()
+        self.handle_t.destroy()
+
+
+def roofline_of(cfg: gen.Config, gemm_ms: float, pk):
+    """Roofline of the projection kernel: W streamed once from HBM vs 2*M*d*V flops on the tensor pipe."""
+    flops = 2.0 * cfg.M * cfg.d * cfg.V
+    byts = 2.0 * cfg.d * cfg.V + 2.0 * cfg.M * cfg.d + 8.0 * cfg.M
+    t_hbm = byts / (pk["hbm_gbs"] * 1e9)
+    t_tc = flops / (pk["bf16_tflops"] * 1e12)
+    s = gemm_ms * 1e-3
+    if t_hbm >= t_tc:
+        a = byts / s / 1e9
+        return {"bound": "hbm", "achieved": a, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": a / pk["hbm_gbs"],
+                "traffic": None, "peak_source": f"of {pk['source']}", "kernel_ms": gemm_ms, "algorithmic_bytes": byts}
+    a = flops / s / 1e12
+    return {"bound": "tensor", "achieved": a, "peak": pk["bf16_tflops"], "unit": "TFLOP/s", "frac": a / pk["bf16_tflops"],
+            "frac_of_sustained_peak": a / pk["bf16_tflops_sustained"], "traffic": None, "peak_source": f"of {pk['source']}",
+            "kernel_ms": gemm_ms, "algorithmic_flops": flops}
+
+
+def bench_one(cfg, device, steps, warmup, barrier, reduce_max, pk, w_copies, W_host=None, with_e2e=True):
+    wl = GpuWorkload(cfg, device, w_copies, W_host)
+    try:
+        wl.run(wl.handle, warmup)
+        with ClockSampler(device) as cs:
+            ms, t0, t1 = wl.timed(wl.handle, steps, barrier)
+        clocks = cs.summary(t0, t1)
+        ms = reduce_max(ms)
+        # the same loop again with events around the projection kernel (ring of 512 launches)
+        wl.run(wl.handle_t, min(warmup, 8))
+        wl.handle_t.gemm_ms_stats()
+        prof_steps = min(steps, 512)
+        wl.timed(wl.handle_t, prof_steps, barrier)
+        gemm_mean, gemm_min, n = wl.handle_t.gemm_ms_stats()
+        assert wl.handle.last_status() == wl.aj.AJ_OK and wl.handle_t.last_status() == wl.aj.AJ_OK
+        res = {
+            "ms_per_step": ms / steps, "clocks": clocks, "path": wl.handle.last_gemm_path(),
+            "roofline": roofline_of(cfg, gemm_mean, pk), "gemm_ms_min": gemm_min, "gemm_launches_timed": n,
+            "launches_per_step": wl.handle.last_launch_count(),
+            "mean_accept_len": float(wl.acc.float().mean().item()),
+        }
+        if with_e2e:
+            s, h2d, d2h = wl.e2e(max(10, min(steps, 300)), 5)
+            res["e2e_s_per_step"] = reduce_max(s)
+            res["h2d"], res["d2h"] = h2d, d2h
+        return res
+    finally:
+        wl.close()
+
+
+def cpu_baseline(cfg: gen.Config, W_host=None):
+    """The CPU oracle, as it stands, on a bounded sample of the workload (whole sequences)."""
+    from oracle import aj_oracle as orc
+
+    n_seq = 1  # one whole sequence: (K+1) rows against the full vocabulary
+    sub = gen.scaled(cfg, B=n_seq)
+    W = gen.make_W(cfg) if W_host is None else W_host
+    ht, hd = gen.make_hidden(cfg)
+    ht, hd = ht[:n_seq], hd[:n_seq]
+    w = gen.make_judge(cfg)
+    tok = gen.random_draft_tokens(sub)
+    t0 = time.perf_counter()
+    r = orc.verify(ht, hd, W, tok, w, cfg.judge_b, cfg.tau, cfg.dtype)
+    dt = time.perf_counter() - t0
+    return {"value": n_seq * cfg.K / dt, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle",
+            "sample": f"{n_seq} of {cfg.B} sequences ({cfg.K + 1} rows x V={cfg.V}, d={cfg.d}), {dt:.2f} s, fp64 loops"}, r
+
+
+def reference_arm(args):
+    """--impl reference: the CPU oracle timed on the host cores (there is no other reference program)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import aj_oracle as orc
+
+    cfg = workload(args.workload if args.workload != "sweep" else "c2")
+    steps = args.steps if args.steps is not None else 3
+    warmup = args.warmup if args.warmup is not None else 1
+    W = gen.make_W(cfg)
+    for _ in range(warmup):
+        cpu_baseline(cfg, W)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        base, _ = cpu_baseline(cfg, W)
+    dt = (time.perf_counter() - t0) / steps
+    value = cfg.K / dt  # one sequence per step
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps, "warmup": warmup,
+        "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": {"workload": cfg.name, "B": 1, "K": cfg.K, "d": cfg.d, "d_draft": cfg.d_draft, "V": cfg.V,
+                                       "note": "each step verifies one whole sequence of the workload with the CPU oracle"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle", "sample": base["sample"]},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--workload", default="c2", choices=["c2", "c3", "c4", "sweep"])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-extra", action="store_true", help="skip the batched configurations reported under 'extra'")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return reference_arm(args)
+
+    import torch
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+
+    def reduce_max(x):
+        if dist is None:
+            return float(x)
+        t = torch.tensor([float(x)], device=f"cuda:{local}", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    pk = peaks()
+    head = workload("c2" if args.workload == "sweep" else args.workload)
+    default_steps = {"c2": 4000, "c3": 400, "c4": 200}[head.name[:2]]
+    steps = args.steps if args.steps is not None else default_steps
+    warmup = max(3, args.warmup if args.warmup is not None else 10)
+    copies = 3 if head.d * head.V * 2 < 1.5e9 else 2
+
+    W_host = gen.make_W(head)
+    r = bench_one(head, local, steps, warmup, barrier, reduce_max, pk, copies, W_host)
+    positions = head.B * head.K * world
+    line = {
+        "metric": METRIC, "value": positions / (r["ms_per_step"] * 1e-3), "unit": UNIT, "n_gpus": world, "steps": steps,
+        "warmup": warmup, "ms_per_step": r["ms_per_step"], "us_per_cycle": r["ms_per_step"] * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": head.name, "B": head.B, "K": head.K, "d": head.d, "d_draft": head.d_draft, "V": head.V,
+                   "tau": head.tau, "match_rate": [head.match_lo, head.match_hi], "parallelism": f"replicated W, batch per rank x{world}",
+                   "l2": f"W_lm rotates over {copies} copies of {head.d * head.V * 2 / 1e9:.2f} GB each (inputs larger than the 126 MB L2)",
+                   "gemm_path": r["path"], "mean_accept_len": r["mean_accept_len"]},
+        "clocks": r["clocks"], "roofline": r["roofline"],
+        "e2e": {"value": positions / r["e2e_s_per_step"], "unit": UNIT, "h2d_bytes_per_step": r["h2d"], "d2h_bytes_per_step": r["d2h"],
+                "us_per_cycle": r["e2e_s_per_step"] * 1e6,
+                "note": "aj_verify_host: hidden states and draft tokens from pinned host memory, results read back; W_lm and judge_w are resident parameters"},
+        "gpu_launches": r["launches_per_step"] * steps,
+    }
+
+    extra = []
+    if not args.no_extra:
+        todo = []
+        if args.workload == "sweep":
+            todo = [gen.sweep_config(B, K) for B in gen.SWEEP_B for K in gen.SWEEP_K]
+        elif args.workload == "c2":
+            todo = [gen.C3, gen.C4]
+        for cfg in todo:
+            same_W = cfg.d == head.d and cfg.V == head.V
+            n = max(20, int(0.4 / max(2.0 * cfg.M * cfg.d * cfg.V / 1.2e15, 1.7e-4)))
+            rr = bench_one(cfg, local, n, 5, barrier, reduce_max, pk, 2 if not same_W else copies, W_host if same_W else None, with_e2e=False)
+            extra.append({"workload": cfg.name, "B": cfg.B, "K": cfg.K, "d": cfg.d, "V": cfg.V, "steps": n,
+                          "ms_per_step": rr["ms_per_step"], "value": cfg.B * cfg.K * world / (rr["ms_per_step"] * 1e-3), "unit": UNIT,
+                          "gemm_path": rr["path"], "roofline": rr["roofline"], "clocks": rr["clocks"]})
+    line["extra"] = extra
+
+    if rank == 0 and world == 1 and not args.no_cpu:
+        base, _ = cpu_baseline(head, W_host)
+        line["cpu_baseline"] = base
+    if rank == 0:
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

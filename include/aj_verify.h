@@ -124,7 +124,15 @@ aj_status aj_last_status(aj_handle h);
  */
 aj_status aj_last_gemm_ms(aj_handle h, float *ms);
 
-/* Number of kernels (and memset nodes) the most recent aj_verify / aj_verify_host call launched. */
+/*
+ * With AJ_FLAG_TIME_KERNELS: mean and minimum duration (milliseconds) of the projection kernel
+ * over the calls made since the previous read-out (the most recent 512 at most), and how many
+ * calls that was; then starts a new series.  Waits for those kernels to finish.  min_ms may be NULL.
+ */
+aj_status aj_gemm_ms_stats(aj_handle h, float *mean_ms, float *min_ms, int *count);
+
+/* Number of kernels of this library that the most recent aj_verify / aj_verify_host call launched
+ * (the projection kernel and the judge kernel; the memset that clears the keys is not counted). */
 int aj_last_launch_count(aj_handle h);
 
 /* Name of the projection kernel configuration the most recent call used, e.g. "umma_128x256". */

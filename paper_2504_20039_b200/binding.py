@@ -18,7 +18,7 @@ AJ_W_VD, AJ_W_DV = 0, 1
 AJ_FLAG_FORCE_SIMT, AJ_FLAG_TIME_KERNELS = 1, 2
 
 EXPORTS = (
-    "aj_create", "aj_verify", "aj_verify_host", "aj_last_status", "aj_last_gemm_ms", "aj_last_launch_count",
+    "aj_create", "aj_verify", "aj_verify_host", "aj_last_status", "aj_last_gemm_ms", "aj_gemm_ms_stats", "aj_last_launch_count",
     "aj_last_gemm_path", "aj_destroy", "aj_status_string", "aj_version",
 )
 
@@ -52,6 +52,8 @@ def lib() -> ctypes.CDLL:
         L.aj_last_status.restype = ci
         L.aj_last_gemm_ms.argtypes = [vp, ctypes.POINTER(cf)]
         L.aj_last_gemm_ms.restype = ci
+        L.aj_gemm_ms_stats.argtypes = [vp, ctypes.POINTER(cf), ctypes.POINTER(cf), ctypes.POINTER(ci)]
+        L.aj_gemm_ms_stats.restype = ci
         L.aj_last_launch_count.argtypes = [vp]
         L.aj_last_launch_count.restype = ci
         L.aj_last_gemm_path.argtypes = [vp]
@@ -126,6 +128,14 @@ class Handle:
         if st != AJ_OK:
             raise AjError(st, "aj_last_gemm_ms")
         return float(ms.value)
+
+    def gemm_ms_stats(self):
+        """(mean ms, min ms, calls) of the projection kernel since the previous read-out."""
+        mean, lo, n = ctypes.c_float(), ctypes.c_float(), ctypes.c_int()
+        st = lib().aj_gemm_ms_stats(self._h, ctypes.byref(mean), ctypes.byref(lo), ctypes.byref(n))
+        if st != AJ_OK:
+            raise AjError(st, "aj_gemm_ms_stats")
+        return float(mean.value), float(lo.value), int(n.value)
 
     def last_launch_count(self) -> int:
         return lib().aj_last_launch_count(self._h)

@@ -23,6 +23,7 @@ struct TmapSlot {
 };
 
 constexpr int TMAP_SLOTS = 8;
+constexpr int EVENT_RING = 512;
 
 }  // namespace
 
@@ -41,8 +42,8 @@ struct aj_handle_s {
     EncodeTiledFn encode = nullptr;
     TmapSlot slots[TMAP_SLOTS];
     unsigned long long stamp = 0;
-    cudaEvent_t ev0 = nullptr, ev1 = nullptr;
-    bool timed = false;
+    cudaEvent_t ev0[EVENT_RING] = {}, ev1[EVENT_RING] = {};  // with AJ_FLAG_TIME_KERNELS
+    long long n_timed = 0;                                   // calls recorded since the last read-out
     int last_launches = 0;
     const char *last_path = "none";
 };
@@ -177,7 +178,8 @@ aj_status aj_create(aj_handle *out, int device, int max_B, int max_K, int d, int
               cudaMalloc(&h->st_acc, (size_t)max_B * 4) == cudaSuccess &&
               cudaMalloc(&h->st_next, (size_t)max_B * 4) == cudaSuccess && cudaMalloc(&h->st_tt, max_M * 4) == cudaSuccess;
     if (ok && (flags & AJ_FLAG_TIME_KERNELS))
-        ok = cudaEventCreate(&h->ev0) == cudaSuccess && cudaEventCreate(&h->ev1) == cudaSuccess;
+        for (int i = 0; ok && i < EVENT_RING; i++)
+            ok = cudaEventCreate(&h->ev0[i]) == cudaSuccess && cudaEventCreate(&h->ev1[i]) == cudaSuccess;
     if (ok && h->umma_ok) {
         void *fn = nullptr;
         cudaDriverEntryPointQueryResult qres;
@@ -206,8 +208,10 @@ aj_status aj_destroy(aj_handle h) {
     cudaFree(h->st_acc);
     cudaFree(h->st_next);
     cudaFree(h->st_tt);
-    if (h->ev0) cudaEventDestroy(h->ev0);
-    if (h->ev1) cudaEventDestroy(h->ev1);
+    for (int i = 0; i < EVENT_RING; i++) {
+        if (h->ev0[i]) cudaEventDestroy(h->ev0[i]);
+        if (h->ev1[i]) cudaEventDestroy(h->ev1[i]);
+    }
     delete h;
     return AJ_OK;
 }
@@ -224,10 +228,8 @@ aj_status aj_verify(aj_handle h, const void *h_target, const void *h_draft, cons
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const int M = B * (K + 1);
     h->last_launches = 0;
-    h->timed = false;
 
     if (cudaMemsetAsync(h->keys, 0, (size_t)M * sizeof(unsigned long long), stream) != cudaSuccess) return AJ_ERR_CUDA;
-    h->last_launches++;
 
     GemmArgs g;
     g.h = h_target;
@@ -241,7 +243,8 @@ aj_status aj_verify(aj_handle h, const void *h_target, const void *h_draft, cons
     g.status = h->status;
 
     const bool time_it = (h->flags & AJ_FLAG_TIME_KERNELS) != 0;
-    if (time_it && cudaEventRecord(h->ev0, stream) != cudaSuccess) return AJ_ERR_CUDA;
+    const int slot = (int)(h->n_timed % EVENT_RING);
+    if (time_it && cudaEventRecord(h->ev0[slot], stream) != cudaSuccess) return AJ_ERR_CUDA;
     cudaError_t e;
     if (h->umma_ok) {
         UmmaPlan p;
@@ -263,8 +266,8 @@ aj_status aj_verify(aj_handle h, const void *h_target, const void *h_draft, cons
     if (e != cudaSuccess) return AJ_ERR_CUDA;
     h->last_launches++;
     if (time_it) {
-        if (cudaEventRecord(h->ev1, stream) != cudaSuccess) return AJ_ERR_CUDA;
-        h->timed = true;
+        if (cudaEventRecord(h->ev1[slot], stream) != cudaSuccess) return AJ_ERR_CUDA;
+        h->n_timed++;
     }
 
     JudgeArgs j;
@@ -330,10 +333,32 @@ aj_status aj_last_status(aj_handle h) {
 }
 
 aj_status aj_last_gemm_ms(aj_handle h, float *ms) {
-    if (!h || !ms || !(h->flags & AJ_FLAG_TIME_KERNELS) || !h->timed) return AJ_ERR_INVALID_ARG;
+    if (!h || !ms || !(h->flags & AJ_FLAG_TIME_KERNELS) || h->n_timed == 0) return AJ_ERR_INVALID_ARG;
     DeviceGuard guard(h->device);
-    if (cudaEventSynchronize(h->ev1) != cudaSuccess) return AJ_ERR_CUDA;
-    if (cudaEventElapsedTime(ms, h->ev0, h->ev1) != cudaSuccess) return AJ_ERR_CUDA;
+    const int slot = (int)((h->n_timed - 1) % EVENT_RING);
+    if (cudaEventSynchronize(h->ev1[slot]) != cudaSuccess) return AJ_ERR_CUDA;
+    if (cudaEventElapsedTime(ms, h->ev0[slot], h->ev1[slot]) != cudaSuccess) return AJ_ERR_CUDA;
+    return AJ_OK;
+}
+
+aj_status aj_gemm_ms_stats(aj_handle h, float *mean_ms, float *min_ms, int *count) {
+    if (!h || !mean_ms || !count || !(h->flags & AJ_FLAG_TIME_KERNELS)) return AJ_ERR_INVALID_ARG;
+    DeviceGuard guard(h->device);
+    const long long n = h->n_timed < EVENT_RING ? h->n_timed : EVENT_RING;
+    double sum = 0.0;
+    float lo = 0.0f;
+    for (long long i = 0; i < n; i++) {
+        const int slot = (int)((h->n_timed - 1 - i) % EVENT_RING);
+        float ms = 0.0f;
+        if (cudaEventSynchronize(h->ev1[slot]) != cudaSuccess) return AJ_ERR_CUDA;
+        if (cudaEventElapsedTime(&ms, h->ev0[slot], h->ev1[slot]) != cudaSuccess) return AJ_ERR_CUDA;
+        sum += ms;
+        if (i == 0 || ms < lo) lo = ms;
+    }
+    *mean_ms = n ? (float)(sum / n) : 0.0f;
+    if (min_ms) *min_ms = lo;
+    *count = (int)n;
+    h->n_timed = 0;
     return AJ_OK;
 }
 

@@ -46,7 +46,7 @@ def _full_parity(cfg, taus, flags=0, layout=0, expect_path=None):
             g = case.run(tok, tau)
             if expect_path:
                 assert g.path == expect_path
-            assert g.launches == 3
+            assert g.launches == 2
             reports.append(check_parity(o, g, tok, tau))
             check_self_consistency(g, tok, tau, cfg.V)
         return reports

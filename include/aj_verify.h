@@ -138,6 +138,35 @@ int aj_last_launch_count(aj_handle h);
 /* Name of the projection kernel configuration the most recent call used, e.g. "umma_128x256". */
 const char *aj_last_gemm_path(aj_handle h);
 
+/*
+ * The cycle of aj_verify for callers that cannot allocate device memory.  (The paper has no
+ * counterpart to this entry point; it exists for integration.)
+ *
+ * aj_create calls cudaMalloc for its workspace.  A caller that gave all device memory to its own
+ * pool at start-up, that runs under a per-allocation memory audit, or whose allocator is frozen by
+ * the time it needs a cycle verified cannot use a handle.  This function takes no handle and calls
+ * no cudaMalloc, cudaFree or any allocating routine: its only scratch memory, one 8-byte key per row
+ * of hidden states plus a status word, is a fixed array inside the library's device image, so every
+ * GPU that loads the library holds AJ_STATIC_MAX_ROWS * 8 + 256 bytes (about 256 KB) until exit.
+ *
+ * Arguments are those of aj_create and aj_verify together; the device is the CURRENT CUDA device;
+ * all pointers are device pointers with the layouts aj_verify documents; optional outputs may be
+ * NULL.  dev_status (optional, device, int32) receives 0, or AJ_ERR_TIMEOUT if a bounded wait in a
+ * kernel ran out; read it after the stream has finished.
+ *   B * (K + 1) > AJ_STATIC_MAX_ROWS  ->  AJ_ERR_WORKSPACE, nothing enqueued.
+ * The first call on each device looks up the array's device address (cudaGetSymbolAddress) and
+ * prepares the kernels; make that first call outside any stream capture.  Later calls only enqueue.
+ * All calls on a device share the one array, which keeps the previous call's contents (this call
+ * clears the part it uses, in stream order): two calls whose GPU work overlaps, on different
+ * streams or from different threads, race on it.  Serialise them.
+ */
+#define AJ_STATIC_MAX_ROWS 32768
+aj_status aj_verify_static(const void *h_target, const void *h_draft, const void *W_lm,
+                           const int32_t *draft_tok, const float *judge_w, float judge_b, float tau,
+                           int B, int K, int d, int d_draft, int V, aj_dtype dtype, aj_w_layout layout,
+                           int32_t *accept_len, int32_t *next_tok, int32_t *target_tok,
+                           float *top1_val, float *judge_p, int32_t *dev_status, void *cuda_stream);
+
 /* Free the handle and its workspace.  The caller must have synchronised all work using it. */
 aj_status aj_destroy(aj_handle h);
 

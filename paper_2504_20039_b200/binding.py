@@ -19,7 +19,7 @@ AJ_FLAG_FORCE_SIMT, AJ_FLAG_TIME_KERNELS = 1, 2
 
 EXPORTS = (
     "aj_create", "aj_verify", "aj_verify_host", "aj_last_status", "aj_last_gemm_ms", "aj_gemm_ms_stats", "aj_last_launch_count",
-    "aj_last_gemm_path", "aj_destroy", "aj_status_string", "aj_version",
+    "aj_last_gemm_path", "aj_destroy", "aj_status_string", "aj_version", "aj_verify_static",
 )
 
 _lib = None
@@ -62,6 +62,8 @@ def lib() -> ctypes.CDLL:
         L.aj_destroy.restype = ci
         L.aj_status_string.argtypes = [ci]
         L.aj_status_string.restype = ctypes.c_char_p
+        L.aj_verify_static.argtypes = [vp, vp, vp, vp, vp, cf, cf, ci, ci, ci, ci, ci, ci, ci, vp, vp, vp, vp, vp, vp, vp]
+        L.aj_verify_static.restype = ci
         L.aj_version.argtypes = []
         L.aj_version.restype = ctypes.c_char_p
         _lib = L
@@ -85,6 +87,26 @@ def _ptr(t):
     if hasattr(t, "data_ptr"):
         return t.data_ptr()
     return t.ctypes.data
+
+
+AJ_STATIC_MAX_ROWS = 32768
+
+
+def verify_static(h_target, h_draft, W_lm, draft_tok, judge_w, judge_b: float, tau: float, B: int, K: int, d: int,
+                  d_draft: int, V: int, dtype: int, layout: int, accept_len, next_tok, target_tok=None, top1_val=None,
+                  judge_p=None, dev_status=None, stream: int = 0, check: bool = True) -> int:
+    """aj_verify_static: one cycle on the current device without a handle and without any allocation.
+
+    For callers that cannot call cudaMalloc (all memory already in their own pool, audited or frozen
+    allocators): the scratch lives in a fixed array inside the library.  At most AJ_STATIC_MAX_ROWS
+    rows (B*(K+1)); calls that overlap on the GPU race on that array.
+    """
+    st = lib().aj_verify_static(_ptr(h_target), _ptr(h_draft), _ptr(W_lm), _ptr(draft_tok), _ptr(judge_w), float(judge_b),
+                                float(tau), B, K, d, d_draft, V, dtype, layout, _ptr(accept_len), _ptr(next_tok),
+                                _ptr(target_tok), _ptr(top1_val), _ptr(judge_p), _ptr(dev_status), stream or None)
+    if check and st != AJ_OK:
+        raise AjError(st, "aj_verify_static")
+    return st
 
 
 class Handle:

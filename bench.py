@@ -289,6 +289,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extra", action="store_true", help="skip the batched configurations reported under 'extra'")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline")
+    ap.add_argument("--w-copies", type=int, default=None, help="copies of W_lm to rotate over (default 3, or 2 for the 70B shape)")
     args = ap.parse_args()
     if args.impl == "reference":
         return reference_arm(args)
@@ -321,7 +322,7 @@ def main():
     default_steps = {"c2": 4000, "c3": 400, "c4": 200}[head.name[:2]]
     steps = args.steps if args.steps is not None else default_steps
     warmup = max(3, args.warmup if args.warmup is not None else 10)
-    copies = 3 if head.d * head.V * 2 < 1.5e9 else 2
+    copies = args.w_copies or (3 if head.d * head.V * 2 < 1.5e9 else 2)
 
     W_host = gen.make_W(head)
     r = bench_one(head, local, steps, warmup, barrier, reduce_max, pk, copies, W_host)

@@ -1,6 +1,8 @@
 // Host side of the C-ABI: argument checks, workspace, tensor maps, stream-ordered launches.
-// One cycle = clear the keys, projection + argmax kernel, judge + scan kernel; no host
-// synchronisation and no allocation inside aj_verify.
+// One cycle = projection + argmax kernel, then judge + scan kernel as its programmatic dependent;
+// no host synchronisation and no allocation inside aj_verify.  The per-row keys start at zero
+// (cleared at creation) and the judge kernel clears each key as it reads it, so a cycle needs no
+// separate clearing pass; only after a launch failed half-way are they cleared explicitly.
 #include "../../include/aj_verify.h"
 #include "aj_internal.cuh"
 
@@ -35,6 +37,7 @@ struct aj_handle_s {
     int num_sms = 0;
     bool umma_ok = false;
     unsigned long long *keys = nullptr;
+    bool keys_dirty = false;  // a cycle was started but its judge kernel was not enqueued
     int *status = nullptr;
     // staging for aj_verify_host
     void *st_ht = nullptr, *st_hd = nullptr;
@@ -171,6 +174,7 @@ aj_status aj_create(aj_handle *out, int device, int max_B, int max_K, int d, int
     const size_t max_M = (size_t)max_B * (max_K + 1);
     const size_t esz = elem_size(dtype);
     bool ok = cudaMalloc(&h->keys, max_M * sizeof(unsigned long long)) == cudaSuccess &&
+              cudaMemset(h->keys, 0, max_M * sizeof(unsigned long long)) == cudaSuccess &&
               cudaMalloc(&h->status, 256) == cudaSuccess && cudaMemset(h->status, 0, 256) == cudaSuccess &&
               cudaMalloc(&h->st_ht, max_M * d * esz) == cudaSuccess &&
               (d_draft == 0 || cudaMalloc(&h->st_hd, max_M * d_draft * esz) == cudaSuccess) &&
@@ -229,7 +233,11 @@ aj_status aj_verify(aj_handle h, const void *h_target, const void *h_draft, cons
     const int M = B * (K + 1);
     h->last_launches = 0;
 
-    if (cudaMemsetAsync(h->keys, 0, (size_t)M * sizeof(unsigned long long), stream) != cudaSuccess) return AJ_ERR_CUDA;
+    if (h->keys_dirty) {
+        const size_t all = (size_t)h->max_B * (h->max_K + 1) * sizeof(unsigned long long);
+        if (cudaMemsetAsync(h->keys, 0, all, stream) != cudaSuccess) return AJ_ERR_CUDA;
+    }
+    h->keys_dirty = true;
 
     GemmArgs g;
     g.h = h_target;
@@ -289,6 +297,7 @@ aj_status aj_verify(aj_handle h, const void *h_target, const void *h_draft, cons
     j.top1_val = top1_val;
     j.judge_p = judge_p;
     if (launch_judge_scan(j, stream) != cudaSuccess) return AJ_ERR_CUDA;
+    h->keys_dirty = false;
     h->last_launches++;
     return AJ_OK;
 }
@@ -328,7 +337,10 @@ aj_status aj_last_status(aj_handle h) {
     int word = 0;
     if (cudaDeviceSynchronize() != cudaSuccess) return AJ_ERR_CUDA;
     if (cudaMemcpy(&word, h->status, sizeof word, cudaMemcpyDeviceToHost) != cudaSuccess) return AJ_ERR_CUDA;
-    if (word != 0 && cudaMemset(h->status, 0, sizeof word) != cudaSuccess) return AJ_ERR_CUDA;
+    if (word != 0) {
+        if (cudaMemset(h->status, 0, sizeof word) != cudaSuccess) return AJ_ERR_CUDA;
+        h->keys_dirty = true;  // a cycle that gave up may have left partial keys behind
+    }
     return word == DEV_TIMEOUT ? AJ_ERR_TIMEOUT : (word == 0 ? AJ_OK : AJ_ERR_CUDA);
 }
 

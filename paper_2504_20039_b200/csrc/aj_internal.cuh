@@ -49,7 +49,7 @@ struct GemmArgs {
     int M, d, V;
     int dtype;           // 0 bf16, 1 f32
     int w_layout;        // 0 [V,d], 1 [d,V]
-    unsigned long long *keys;  // [M], must be zero on entry
+    unsigned long long *keys;  // [M], must be zero on entry (the judge kernel clears what it reads)
     int *status;
 };
 
@@ -68,7 +68,7 @@ cudaError_t launch_umma_gemm_argmax(const GemmArgs &a, const UmmaPlan &p, cudaSt
 const char *umma_path_name(int bn);
 
 struct JudgeArgs {
-    const unsigned long long *keys;  // [B*(K+1)]
+    unsigned long long *keys;        // [B*(K+1)]; read, then cleared for the next cycle
     const void *h_target;            // [B, K+1, d]
     const void *h_draft;             // [B, K+1, d_draft] or nullptr
     const int32_t *draft_tok;        // [B, K]

@@ -6,8 +6,14 @@
 //   stop    = first i with mis[i] and not (p[i] < tau)                ballot + ffs over the window
 //   accept_len = stop (K if none), next_tok = y[accept_len]
 //
-// A warp takes one mismatching position at a time: 128-bit loads of the features, fp32
-// accumulate, shuffle reduction.
+// The judge is latency-bound (a few rows of 8-24 KB each), so the work is cut into
+// (position, segment) items: a segment is 1/SEGS of the concatenated feature vector, a warp
+// takes one item at a time and issues all of its 128-bit loads before it uses any of them.
+// Segment sums are added in a fixed order, so p does not depend on scheduling.
+//
+// The kernel is launched as a programmatic dependent of the projection kernel: its blocks may
+// become resident while that kernel still runs and wait at the grid dependency before they
+// read the keys.  Each key is cleared right after it is read, so the next cycle finds zeros.
 #include "aj_internal.cuh"
 
 #include <cuda_bf16.h>
@@ -15,6 +21,9 @@
 namespace aj {
 
 namespace {
+
+constexpr int SEGS = 8;
+constexpr int THREADS = 512;
 
 __device__ inline float dot8_bf16(const uint4 &x, const float4 &w0, const float4 &w1) {
     const __nv_bfloat162 *p = reinterpret_cast<const __nv_bfloat162 *>(&x);
@@ -31,81 +40,156 @@ __device__ inline float dot8_bf16(const uint4 &x, const float4 &w0, const float4
     return s;
 }
 
-// partial dot product of one feature block held by this lane
-__device__ inline float block_dot(const void *x, const float *w, int n, int dtype, int lane) {
-    float s = 0.0f;
-    if (x == nullptr || n <= 0) return s;
-    if (dtype == 0) {
-        const bool vec = (n % 8 == 0) && ((reinterpret_cast<uintptr_t>(x) & 15) == 0) &&
-                         ((reinterpret_cast<uintptr_t>(w) & 15) == 0);
-        if (vec) {
-            const uint4 *xv = reinterpret_cast<const uint4 *>(x);
-            const float4 *wv = reinterpret_cast<const float4 *>(w);
-            for (int c = lane; c < n / 8; c += 32) s += dot8_bf16(__ldg(xv + c), __ldg(wv + 2 * c), __ldg(wv + 2 * c + 1));
-        } else {
-            const __nv_bfloat16 *xs = reinterpret_cast<const __nv_bfloat16 *>(x);
-            for (int f = lane; f < n; f += 32) s = fmaf(__bfloat162float(xs[f]), w[f], s);
-        }
-    } else {
-        const bool vec = (n % 4 == 0) && ((reinterpret_cast<uintptr_t>(x) & 15) == 0) &&
-                         ((reinterpret_cast<uintptr_t>(w) & 15) == 0);
-        if (vec) {
-            const float4 *xv = reinterpret_cast<const float4 *>(x);
-            const float4 *wv = reinterpret_cast<const float4 *>(w);
-            for (int c = lane; c < n / 4; c += 32) {
-                const float4 a = __ldg(xv + c), b = __ldg(wv + c);
-                s = fmaf(a.x, b.x, s);
-                s = fmaf(a.y, b.y, s);
-                s = fmaf(a.z, b.z, s);
-                s = fmaf(a.w, b.w, s);
+__device__ inline float dot4_f32(const float4 &a, const float4 &b) {
+    float s = a.x * b.x;
+    s = fmaf(a.y, b.y, s);
+    s = fmaf(a.z, b.z, s);
+    s = fmaf(a.w, b.w, s);
+    return s;
+}
+
+// This lane's share of chunks [c0, c1) of the concatenated feature vector; a chunk is 16 bytes
+// of features (8 bf16 or 4 f32).  Chunks below `split` come from the draft row, the rest from
+// the target row.  Four chunks are in flight per lane.
+template <bool BF16>
+__device__ inline float segment_dot(const char *xd, const char *xt, const float *w, int split, int c0, int c1, int lane) {
+    constexpr int EPC = BF16 ? 8 : 4;  // elements per chunk
+    float acc = 0.0f;
+    for (int c = c0 + lane; c < c1; c += 128) {
+        uint4 x[4];
+        float4 wa[4], wb[4];
+#pragma unroll
+        for (int u = 0; u < 4; u++) {
+            const int cc = c + 32 * u;
+            if (cc < c1) {
+                const char *src = cc < split ? xd + (size_t)cc * 16 : xt + (size_t)(cc - split) * 16;
+                x[u] = __ldg(reinterpret_cast<const uint4 *>(src));
+                const float4 *wp = reinterpret_cast<const float4 *>(w + (size_t)cc * EPC);
+                wa[u] = __ldg(wp);
+                if (BF16) wb[u] = __ldg(wp + 1);
+            } else {
+                x[u] = make_uint4(0, 0, 0, 0);
+                wa[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                wb[u] = wa[u];
             }
-        } else {
-            const float *xs = reinterpret_cast<const float *>(x);
-            for (int f = lane; f < n; f += 32) s = fmaf(xs[f], w[f], s);
         }
+#pragma unroll
+        for (int u = 0; u < 4; u++) {
+            if (BF16)
+                acc += dot8_bf16(x[u], wa[u], wb[u]);
+            else
+                acc += dot4_f32(*reinterpret_cast<const float4 *>(&x[u]), wa[u]);
+        }
+    }
+    return acc;
+}
+
+// scalar fallback for widths or addresses that do not allow 16-byte loads
+__device__ inline float scalar_dot(const void *x, const float *w, int n, int dtype, int lane) {
+    float s = 0.0f;
+    if (x == nullptr) return s;
+    if (dtype == 0) {
+        const __nv_bfloat16 *xs = reinterpret_cast<const __nv_bfloat16 *>(x);
+        for (int f = lane; f < n; f += 32) s = fmaf(__bfloat162float(xs[f]), w[f], s);
+    } else {
+        const float *xs = reinterpret_cast<const float *>(x);
+        for (int f = lane; f < n; f += 32) s = fmaf(xs[f], w[f], s);
     }
     return s;
 }
 
-__global__ void __launch_bounds__(512) judge_scan_kernel(JudgeArgs a) {
+__global__ void __maxnreg__(96) judge_scan_kernel(JudgeArgs a) {
     extern __shared__ int smem[];
-    int *y_s = smem;               // [K+1]
-    int *rej_s = smem + a.K + 1;   // [K]
-    const int b = blockIdx.x;
     const int K = a.K, R = a.K + 1;
+    int *y_s = smem;                                          // [K+1]
+    int *rej_s = smem + R;                                    // [K]: 1 = mismatch not forgiven
+    int *mis_s = rej_s + K;                                   // [K]
+    float *part_s = reinterpret_cast<float *>(mis_s + K);     // [K][SEGS]
+    const int b = blockIdx.x;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     const size_t esz = a.dtype == 0 ? 2 : 4;
+    const int epc = a.dtype == 0 ? 8 : 4;
 
+    const uintptr_t row_bytes_t = (uintptr_t)a.d * esz, row_bytes_d = (uintptr_t)a.d_draft * esz;
+
+    // ---- before the grid dependency: everything that does not need the projection's result.
+    // Let the next kernel in the stream start its own prologue, stage the draft tokens, and pull
+    // the judge weights (and, for small batches, the candidate feature rows) into L2.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    for (int i = threadIdx.x; i < K; i += blockDim.x) mis_s[i] = a.draft_tok[(size_t)b * K + i];
+    {
+        const char *wbytes = reinterpret_cast<const char *>(a.judge_w);
+        const size_t wlines = ((size_t)(a.d + a.d_draft) * 4 + 127) / 128;
+        for (size_t l = threadIdx.x; l < wlines; l += blockDim.x)
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(wbytes + l * 128));
+        if ((long long)gridDim.x * K <= 256) {
+            const size_t lt = (row_bytes_t + 127) / 128, ld = a.h_draft ? (row_bytes_d + 127) / 128 : 0;
+            const size_t per_row = lt + ld;
+            for (size_t l = threadIdx.x; l < per_row * K; l += blockDim.x) {
+                const size_t row = (size_t)b * R + 1 + l / per_row, o = l % per_row;
+                const char *src = o < lt ? reinterpret_cast<const char *>(a.h_target) + row * row_bytes_t + o * 128
+                                         : reinterpret_cast<const char *>(a.h_draft) + row * row_bytes_d + (o - lt) * 128;
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(src));
+            }
+        }
+    }
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+
+    // ---- the projection kernel has finished and its keys are visible
     for (int j = threadIdx.x; j < R; j += blockDim.x) {
-        const unsigned long long key = a.keys[(size_t)b * R + j];
+        unsigned long long *kp = a.keys + (size_t)b * R + j;
+        const unsigned long long key = *kp;
+        *kp = 0ull;  // leave the workspace clean for the next cycle
         const int y = key_index(key);
         y_s[j] = y;
         if (a.target_tok) a.target_tok[(size_t)b * R + j] = y;
         if (a.top1_val) a.top1_val[(size_t)b * R + j] = key_value(key);
     }
     __syncthreads();
+    for (int i = threadIdx.x; i < K; i += blockDim.x) mis_s[i] = mis_s[i] != y_s[i];  // staged token vs greedy token
+    __syncthreads();
 
-    for (int i = warp; i < K; i += nwarps) {
-        const bool mis = a.draft_tok[(size_t)b * K + i] != y_s[i];  // warp-uniform
-        float p = __int_as_float(0x7fc00000);                      // NaN where the judge is not consulted
-        int rej = 0;
-        if (mis) {
-            const size_t row = (size_t)b * R + (i + 1);  // the hidden states that encode draft token i
-            const char *xd = a.h_draft ? reinterpret_cast<const char *>(a.h_draft) + row * a.d_draft * esz : nullptr;
-            const char *xt = reinterpret_cast<const char *>(a.h_target) + row * a.d * esz;
-            float s = block_dot(xd, a.judge_w, a.d_draft, a.dtype, lane) +
-                      block_dot(xt, a.judge_w + a.d_draft, a.d, a.dtype, lane);
+    const bool vec = (a.d % epc == 0) && (a.d_draft % epc == 0) && (row_bytes_t % 16 == 0) && (row_bytes_d % 16 == 0) &&
+                     ((reinterpret_cast<uintptr_t>(a.h_target) & 15) == 0) &&
+                     ((reinterpret_cast<uintptr_t>(a.h_draft) & 15) == 0) &&
+                     ((reinterpret_cast<uintptr_t>(a.judge_w) & 15) == 0);
+    const int split = a.d_draft / epc;                 // chunks that belong to the draft row
+    const int chunks = (a.d_draft + a.d) / epc;
+    for (int it = warp; it < K * SEGS; it += nwarps) {
+        const int i = it / SEGS, seg = it % SEGS;
+        if (!mis_s[i]) continue;                        // the judge is consulted at mismatches only
+        const size_t row = (size_t)b * R + (i + 1);     // the hidden states that encode draft token i
+        const char *xd = a.h_draft ? reinterpret_cast<const char *>(a.h_draft) + row * row_bytes_d : nullptr;
+        const char *xt = reinterpret_cast<const char *>(a.h_target) + row * row_bytes_t;
+        float s;
+        if (vec) {
+            const int c0 = (int)((long long)chunks * seg / SEGS), c1 = (int)((long long)chunks * (seg + 1) / SEGS);
+            s = a.dtype == 0 ? segment_dot<true>(xd, xt, a.judge_w, split, c0, c1, lane)
+                             : segment_dot<false>(xd, xt, a.judge_w, split, c0, c1, lane);
+        } else {
+            s = seg == 0 ? scalar_dot(xd, a.judge_w, a.d_draft, a.dtype, lane) +
+                               scalar_dot(xt, a.judge_w + a.d_draft, a.d, a.dtype, lane)
+                         : 0.0f;
+        }
 #pragma unroll
-            for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
-            const float z = a.judge_b + s;
+        for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
+        if (lane == 0) part_s[it] = s;
+    }
+    __syncthreads();
+
+    for (int i = threadIdx.x; i < K; i += blockDim.x) {
+        float p = __int_as_float(0x7fc00000);  // NaN where the judge is not consulted
+        int rej = 0;
+        if (mis_s[i]) {
+            float z = a.judge_b;
+#pragma unroll
+            for (int seg = 0; seg < SEGS; seg++) z += part_s[i * SEGS + seg];
             p = 1.0f / (1.0f + expf(-z));
             const bool forgiven = (a.tau <= 0.0f) ? false : (a.tau >= 1.0f) ? true : (p < a.tau);
             rej = forgiven ? 0 : 1;
         }
-        if (lane == 0) {
-            rej_s[i] = rej;
-            if (a.judge_p) a.judge_p[(size_t)b * K + i] = p;
-        }
+        rej_s[i] = rej;
+        if (a.judge_p) a.judge_p[(size_t)b * K + i] = p;
     }
     __syncthreads();
 
@@ -129,10 +213,17 @@ __global__ void __launch_bounds__(512) judge_scan_kernel(JudgeArgs a) {
 }  // namespace
 
 cudaError_t launch_judge_scan(const JudgeArgs &a, cudaStream_t stream) {
-    const int threads = 512;
-    const size_t smem = (size_t)(2 * a.K + 1) * sizeof(int);
-    judge_scan_kernel<<<a.B, threads, smem, stream>>>(a);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)a.B);
+    cfg.blockDim = dim3(THREADS);
+    cfg.dynamicSmemBytes = (size_t)(3 * a.K + 1) * sizeof(int) + (size_t)a.K * SEGS * sizeof(float);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, judge_scan_kernel, a);
 }
 
 }  // namespace aj

@@ -221,6 +221,13 @@ umma_gemm_argmax_kernel(const __grid_constant__ CUtensorMap tmap_h, const __grid
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // This kernel may be launched as a programmatic dependent of whatever precedes it in the
+    // stream, so that the set-up above overlaps that kernel's tail: nothing the caller passed has
+    // been read yet, and nothing is before this wait returns (the previous grid has then finished
+    // and its writes are visible).  Then let this kernel's own dependent, the judge kernel, become
+    // resident; it waits at its grid dependency until this whole grid has finished.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     auto give_up = [&]() {
         *abort_flag = 1;
@@ -376,9 +383,18 @@ cudaError_t launch_one(const GemmArgs &a, const UmmaPlan &p, cudaStream_t stream
     const int n_m = (a.M + BM - 1) / BM;
     const int n_v = (a.V + BN - 1) / BN;
     const int stream_w = (n_m == 1) ? 1 : 0;  // W is read by one CTA only: do not keep it in L2
-    umma_gemm_argmax_kernel<BN><<<p.grid, NUM_THREADS, Cfg<BN>::SMEM_BYTES, stream>>>(
-        p.tmap_h, p.tmap_w, a.M, a.V, a.d, n_m, n_v, stream_w, a.keys, a.status);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)p.grid);
+    cfg.blockDim = dim3(NUM_THREADS);
+    cfg.dynamicSmemBytes = Cfg<BN>::SMEM_BYTES;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, umma_gemm_argmax_kernel<BN>, p.tmap_h, p.tmap_w, a.M, a.V, a.d, n_m, n_v, stream_w,
+                              a.keys, a.status);
 }
 
 }  // namespace

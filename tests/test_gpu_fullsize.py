@@ -1,0 +1,96 @@
+"""GPU parity at the full benchmark sizes, in the launch configuration the benchmark times.
+
+The CPU oracle verifies whole sequences sampled from the batch (all of them for the batch-1
+workload); their draft tokens are planted against the oracle's own greedy tokens.  The other
+sequences of the batch get draft tokens planted against the device's greedy tokens (never an
+oracle input) and are checked through properties that hold at any size.  Set AJ_FULL_ORACLE=1 to
+have the oracle verify every sequence.
+"""
+import os
+
+import numpy as np
+import pytest
+
+import aj_inputs as gen
+from aj_testlib import DeviceCase, check_parity, check_self_consistency
+
+pytestmark = pytest.mark.gpu
+
+_CACHE = {}
+
+
+def _orc():
+    from oracle import aj_oracle as orc
+
+    return orc
+
+
+def _W(cfg):
+    """Host and device copies of the LM head, shared by every workload of the same model shape."""
+    key = (cfg.d, cfg.V, cfg.seed)
+    if key not in _CACHE:
+        _CACHE.clear()  # one LM head on the device at a time
+        from aj_testlib import to_device
+
+        Wh = gen.make_W(cfg)
+        _CACHE[key] = (Wh, to_device(Wh, cfg.dtype))
+    return _CACHE[key]
+
+
+def _sample(cfg, n):
+    if os.environ.get("AJ_FULL_ORACLE") == "1" or n >= cfg.B:
+        return list(range(cfg.B))
+    return sorted(set(np.linspace(0, cfg.B - 1, n).astype(int).tolist()))
+
+
+def _run_workload(cfg, taus, n_sample, expect_path):
+    orc = _orc()
+    Wh, Wd = _W(cfg)
+    ht, hd = gen.make_hidden(cfg)
+    w = gen.make_judge(cfg)
+    seqs = _sample(cfg, n_sample)
+    case = DeviceCase(cfg, Wd, ht, hd, w)
+    try:
+        # pass 1: the device's own greedy tokens, used to plant the sequences the oracle does not see
+        first = case.run(gen.random_draft_tokens(cfg), 0.5)
+        tok = gen.plant_draft_tokens(cfg, first.target_tok)
+        # sampled sequences: greedy tokens from the oracle, draft tokens planted against them
+        o_full = orc.verify(ht[seqs], hd[seqs], Wh, np.zeros((len(seqs), cfg.K), np.int32), w, cfg.judge_b, 0.5, cfg.dtype)
+        tok[seqs] = gen.plant_draft_tokens(cfg, o_full.target_tok, rows=seqs)
+        # one full oracle pass on the planted tokens; other thresholds replay only the accept walk
+        # on the same y and p (the replay is pinned against the full pass in the CPU tests)
+        o = orc.verify(ht[seqs], hd[seqs], Wh, tok[seqs], w, cfg.judge_b, taus[0], cfg.dtype)
+        np.testing.assert_array_equal(o.target_tok, o_full.target_tok)
+        reports = []
+        for tau in taus:
+            if tau != taus[0]:
+                o.accept_len, o.next_tok = orc.rewalk(o.target_tok, tok[seqs], o.judge_p, tau)
+            g = case.run(tok, tau)
+            assert g.path == expect_path and g.launches == 2
+            reports.append(check_parity(o, g, tok[seqs], tau, seqs=seqs))
+            check_self_consistency(g, tok, tau, cfg.V)
+        return reports
+    finally:
+        case.close()
+
+
+def test_c2_8b_batch1_every_row():
+    reps = _run_workload(gen.C2, gen.C2_TAUS, gen.C2.B, "umma_128x128")
+    assert all(r.rows == 17 for r in reps)
+
+
+def test_c3_8b_batched_sampled_sequences():
+    reps = _run_workload(gen.C3, (gen.C3.tau,), 8, "umma_128x256")
+    assert reps[0].seqs >= 8 and reps[0].seqs_exempt <= reps[0].seqs // 2
+
+
+def test_c5_sweep_points_on_the_8b_shape():
+    # smallest, the HBM/tensor crossover, and the largest point of the sweep
+    for B, K, path in [(1, 8, "umma_128x128"), (8, 32, "umma_128x256"), (256, 8, "umma_128x256"), (256, 64, "umma_128x256")]:
+        reps = _run_workload(gen.sweep_config(B, K), (0.5,), 3, path)
+        assert reps[0].seqs >= min(B, 3)
+
+
+def test_c4_70b_sampled_sequences_tau_sweep():
+    reps = _run_workload(gen.C4, gen.C4_TAUS, 4, "umma_128x256")
+    assert len(reps) == 9 and all(r.seqs >= 4 for r in reps)

@@ -54,7 +54,9 @@ typedef enum {
 
 enum {
     AJ_FLAG_FORCE_SIMT = 1u,  /* use the plain fp32-accumulate CUDA-core kernel for the projection */
-    AJ_FLAG_TIME_KERNELS = 2u /* record CUDA events around the projection kernel (see aj_last_gemm_ms) */
+    AJ_FLAG_TIME_KERNELS = 2u, /* record CUDA events around the projection kernel (see aj_last_gemm_ms) */
+    AJ_FLAG_ROW_TILES = 4u     /* tensor-core path with 128-row tiles of h on the UMMA M axis (the earlier
+                                  tiling, kept for comparison) instead of vocabulary-major tiles */
 };
 
 /*

@@ -142,7 +142,7 @@ aj_status aj_create(aj_handle *out, int device, int max_B, int max_K, int d, int
     if (device < 0 || max_B < 1 || max_K < 1 || max_K > 1024 || d < 1 || d_draft < 0 || V < 1) return AJ_ERR_INVALID_ARG;
     if (dtype != AJ_BF16 && dtype != AJ_F32) return AJ_ERR_INVALID_ARG;
     if (layout != AJ_W_VD && layout != AJ_W_DV) return AJ_ERR_INVALID_ARG;
-    if (flags & ~(AJ_FLAG_FORCE_SIMT | AJ_FLAG_TIME_KERNELS)) return AJ_ERR_INVALID_ARG;
+    if (flags & ~(AJ_FLAG_FORCE_SIMT | AJ_FLAG_TIME_KERNELS | AJ_FLAG_ROW_TILES)) return AJ_ERR_INVALID_ARG;
     if ((long long)max_B * (max_K + 1) > (1ll << 24)) return AJ_ERR_INVALID_ARG;
     if (dtype == AJ_BF16 && (d % 8 != 0 || d_draft % 8 != 0)) return AJ_ERR_UNSUPPORTED;
 
@@ -190,7 +190,7 @@ aj_status aj_create(aj_handle *out, int device, int max_B, int max_K, int d, int
         ok = cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &fn, 12000, cudaEnableDefault, &qres) == cudaSuccess &&
              qres == cudaDriverEntryPointSuccess && fn != nullptr;
         h->encode = reinterpret_cast<EncodeTiledFn>(fn);
-        if (ok) ok = umma_prepare() == cudaSuccess;
+        if (ok) ok = umma_prepare() == cudaSuccess && umma_vm_prepare() == cudaSuccess;
     }
     if (!ok) {
         cudaGetLastError();
@@ -254,7 +254,19 @@ aj_status aj_verify(aj_handle h, const void *h_target, const void *h_draft, cons
     const int slot = (int)(h->n_timed % EVENT_RING);
     if (time_it && cudaEventRecord(h->ev0[slot], stream) != cudaSuccess) return AJ_ERR_CUDA;
     cudaError_t e;
-    if (h->umma_ok) {
+    if (h->umma_ok && !(h->flags & AJ_FLAG_ROW_TILES)) {
+        UmmaPlan p;
+        p.bn = vm_choose_bn(M);
+        const CUtensorMap *tw = get_tmap(h, W_lm, V, 128);
+        const CUtensorMap *th = get_tmap(h, h_target, M, p.bn);
+        if (!th || !tw) return AJ_ERR_CUDA;
+        p.tmap_h = *th;
+        p.tmap_w = *tw;
+        const long long tiles = (long long)((M + p.bn - 1) / p.bn) * ((V + 127) / 128);
+        p.grid = (int)(tiles < h->num_sms ? tiles : h->num_sms);
+        e = launch_umma_vm(g, p, stream);
+        h->last_path = umma_vm_path_name(p.bn);
+    } else if (h->umma_ok) {
         UmmaPlan p;
         p.bn = choose_bn(M);
         const CUtensorMap *th = get_tmap(h, h_target, M, 128);

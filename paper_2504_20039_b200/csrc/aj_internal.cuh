@@ -67,6 +67,13 @@ cudaError_t umma_prepare();  // opt-in shared memory attributes; call once per d
 cudaError_t launch_umma_gemm_argmax(const GemmArgs &a, const UmmaPlan &p, cudaStream_t stream);
 const char *umma_path_name(int bn);
 
+// tcgen05 projection + argmax with the vocabulary on the UMMA M axis (the default path).
+// Here tmap_w has a 64 x 128 box and tmap_h a 64 x bn box, bn = vm_choose_bn(M) rows of h per tile.
+int vm_choose_bn(int M);
+cudaError_t umma_vm_prepare();
+cudaError_t launch_umma_vm(const GemmArgs &a, const UmmaPlan &p, cudaStream_t stream);
+const char *umma_vm_path_name(int bn);
+
 struct JudgeArgs {
     unsigned long long *keys;        // [B*(K+1)]; read, then cleared for the next cycle
     const void *h_target;            // [B, K+1, d]

@@ -72,7 +72,7 @@ const DeviceSetup *setup_current_device(aj_status *st) {
         } else if (cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &fn, 12000, cudaEnableDefault, &qres) != cudaSuccess ||
                    qres != cudaDriverEntryPointSuccess || fn == nullptr) {
             s.error = AJ_ERR_CUDA;
-        } else if (umma_prepare() != cudaSuccess) {
+        } else if (umma_vm_prepare() != cudaSuccess) {
             s.error = AJ_ERR_CUDA;
         } else {
             s.scratch = static_cast<unsigned char *>(ptr);
@@ -140,11 +140,11 @@ extern "C" aj_status aj_verify_static(const void *h_target, const void *h_draft,
     cudaError_t e;
     if (dtype == AJ_BF16 && layout == AJ_W_VD && d % 64 == 0) {
         UmmaPlan p;
-        p.bn = M <= 128 ? 128 : 256;
-        if (!encode_rows(s, &p.tmap_h, h_target, d, M, 128) || !encode_rows(s, &p.tmap_w, W_lm, d, V, p.bn)) return AJ_ERR_CUDA;
-        const long long tiles = (long long)((M + 127) / 128) * ((V + p.bn - 1) / p.bn);
+        p.bn = vm_choose_bn(M);
+        if (!encode_rows(s, &p.tmap_w, W_lm, d, V, 128) || !encode_rows(s, &p.tmap_h, h_target, d, M, p.bn)) return AJ_ERR_CUDA;
+        const long long tiles = (long long)((M + p.bn - 1) / p.bn) * ((V + 127) / 128);
         p.grid = (int)(tiles < s->num_sms ? tiles : s->num_sms);
-        e = launch_umma_gemm_argmax(g, p, stream);
+        e = launch_umma_vm(g, p, stream);
     } else {
         e = launch_simt_gemm_argmax(g, s->num_sms, stream);
     }

@@ -75,7 +75,7 @@ def test_golden_workloads(name):
         g = case.run(tok, cfg.tau)
     finally:
         case.close()
-    assert g.path == ("simt" if cfg.dtype == gen.F32 else "umma_128x128")
+    assert g.path == ("simt" if cfg.dtype == gen.F32 else "umma_vm_128x32")
     np.testing.assert_array_equal(g.target_tok, np.array(want["target_tok"]))
     np.testing.assert_array_equal(g.accept_len, np.array(want["accept_len"]))
     np.testing.assert_array_equal(g.next_tok, np.array(want["next_tok"]))
@@ -96,7 +96,7 @@ SHAPES = [
 
 
 @pytest.mark.parametrize("shape", SHAPES, ids=[s[0] for s in SHAPES])
-@pytest.mark.parametrize("flags", [0, 1], ids=["umma", "simt"])
+@pytest.mark.parametrize("flags", [0, 4, 1], ids=["umma_vm", "umma_rows", "simt"])
 def test_cut_down_shapes_bf16(shape, flags):
     name, B, K, d, dd, V = shape
     cfg = gen.Config(name, B=B, K=K, d=d, d_draft=dd, V=V, sigma_W=0.2, sigma_w=0.05, match_lo=0.5, match_hi=0.95, seed=3)
@@ -132,7 +132,7 @@ def test_ties_zeros_and_out_of_range_draft_tokens():
     tok = gen.plant_draft_tokens(cfg, y)
     tok[0, 1] = -5          # ids outside the vocabulary are data: they simply never match
     tok[1, 2] = cfg.V + 9
-    for flags in (0, 1):
+    for flags in (0, 4, 1):
         case = DeviceCase(cfg, W, ht, hd, w, flags=flags)
         try:
             o = orc.verify(ht, hd, W, tok, w, 0.0, 0.5, cfg.dtype)
@@ -146,7 +146,7 @@ def test_ties_zeros_and_out_of_range_draft_tokens():
     # +0 and -0 logits still ties
     Wz = np.zeros_like(W)
     hneg = ht.copy()
-    for flags in (0, 1):
+    for flags in (0, 4, 1):
         case = DeviceCase(cfg, Wz, hneg, hd, w, flags=flags)
         try:
             g = case.run(np.zeros((cfg.B, cfg.K), np.int32), 0.5)
@@ -166,14 +166,15 @@ def test_all_negative_logits_are_not_beaten_by_the_zero_filled_tail():
     w = gen.make_judge(cfg)
     y = _oracle_y(cfg, W, ht)
     tok = gen.plant_draft_tokens(cfg, y)
-    case = DeviceCase(cfg, W, ht, None, w)
-    try:
-        o = orc.verify(ht, None, W, tok, w, 0.0, 0.5, cfg.dtype)
-        g = case.run(tok, 0.5)
-        assert (g.top1 < 0).all()
-        check_parity(o, g, tok, 0.5)
-    finally:
-        case.close()
+    o = orc.verify(ht, None, W, tok, w, 0.0, 0.5, cfg.dtype)
+    for flags in (0, 4):
+        case = DeviceCase(cfg, W, ht, None, w, flags=flags)
+        try:
+            g = case.run(tok, 0.5)
+            assert (g.top1 < 0).all()
+            check_parity(o, g, tok, 0.5)
+        finally:
+            case.close()
 
 
 def test_smallest_window_and_batch_slicing_and_determinism():

@@ -55,8 +55,10 @@ typedef enum {
 enum {
     AJ_FLAG_FORCE_SIMT = 1u,  /* use the plain fp32-accumulate CUDA-core kernel for the projection */
     AJ_FLAG_TIME_KERNELS = 2u, /* record CUDA events around the projection kernel (see aj_last_gemm_ms) */
-    AJ_FLAG_ROW_TILES = 4u     /* tensor-core path with 128-row tiles of h on the UMMA M axis (the earlier
+    AJ_FLAG_ROW_TILES = 4u,    /* tensor-core path with 128-row tiles of h on the UMMA M axis (the earlier
                                   tiling, kept for comparison) instead of vocabulary-major tiles */
+    AJ_FLAG_ONE_SM = 8u        /* keep batches of more than 128 rows on the one-SM vocabulary-major kernel
+                                  instead of the two-SM (CTA pair) kernel; for comparison */
 };
 
 /*

@@ -36,6 +36,7 @@ struct aj_handle_s {
     unsigned flags = 0;
     int num_sms = 0;
     bool umma_ok = false;
+    bool pair_ok = false;  // the two-SM kernel can be launched on this device
     unsigned long long *keys = nullptr;
     bool keys_dirty = false;  // a cycle was started but its judge kernel was not enqueued
     int *status = nullptr;
@@ -103,6 +104,10 @@ const CUtensorMap *get_tmap(aj_handle h, const void *ptr, long long rows, int bo
 
 int choose_bn(int M) { return M <= 128 ? 128 : 256; }
 
+// Batches with more rows than this run on the two-SM kernel; smaller ones are bound by the W_lm
+// stream from HBM and keep the one-SM kernel, which has more loads in flight per SM.
+constexpr int PAIR_MIN_ROWS = 128;
+
 aj_status check_call(aj_handle h, const void *h_target, const void *h_draft, const void *W_lm, const int32_t *draft_tok,
                      const float *judge_w, int B, int K, int d, int V, const int32_t *accept_len,
                      const int32_t *next_tok) {
@@ -142,7 +147,7 @@ aj_status aj_create(aj_handle *out, int device, int max_B, int max_K, int d, int
     if (device < 0 || max_B < 1 || max_K < 1 || max_K > 1024 || d < 1 || d_draft < 0 || V < 1) return AJ_ERR_INVALID_ARG;
     if (dtype != AJ_BF16 && dtype != AJ_F32) return AJ_ERR_INVALID_ARG;
     if (layout != AJ_W_VD && layout != AJ_W_DV) return AJ_ERR_INVALID_ARG;
-    if (flags & ~(AJ_FLAG_FORCE_SIMT | AJ_FLAG_TIME_KERNELS | AJ_FLAG_ROW_TILES)) return AJ_ERR_INVALID_ARG;
+    if (flags & ~(AJ_FLAG_FORCE_SIMT | AJ_FLAG_TIME_KERNELS | AJ_FLAG_ROW_TILES | AJ_FLAG_ONE_SM)) return AJ_ERR_INVALID_ARG;
     if ((long long)max_B * (max_K + 1) > (1ll << 24)) return AJ_ERR_INVALID_ARG;
     if (dtype == AJ_BF16 && (d % 8 != 0 || d_draft % 8 != 0)) return AJ_ERR_UNSUPPORTED;
 
@@ -191,6 +196,8 @@ aj_status aj_create(aj_handle *out, int device, int max_B, int max_K, int d, int
              qres == cudaDriverEntryPointSuccess && fn != nullptr;
         h->encode = reinterpret_cast<EncodeTiledFn>(fn);
         if (ok) ok = umma_prepare() == cudaSuccess && umma_vm_prepare() == cudaSuccess;
+        if (ok) h->pair_ok = umma_pair_prepare(h->num_sms) == cudaSuccess && umma_pair_max_pairs() > 0;
+        if (!h->pair_ok) cudaGetLastError();  // no room for CTA pairs: the one-SM kernel serves every batch
     }
     if (!ok) {
         cudaGetLastError();
@@ -254,7 +261,21 @@ aj_status aj_verify(aj_handle h, const void *h_target, const void *h_draft, cons
     const int slot = (int)(h->n_timed % EVENT_RING);
     if (time_it && cudaEventRecord(h->ev0[slot], stream) != cudaSuccess) return AJ_ERR_CUDA;
     cudaError_t e;
-    if (h->umma_ok && !(h->flags & AJ_FLAG_ROW_TILES)) {
+    if (h->umma_ok && h->pair_ok && M > PAIR_MIN_ROWS && !(h->flags & (AJ_FLAG_ROW_TILES | AJ_FLAG_ONE_SM))) {
+        // tensor-bound regime: two-SM tiles of 256 vocabulary entries x up to 256 rows
+        UmmaPlan p;
+        p.bn = 256;
+        const CUtensorMap *tw = get_tmap(h, W_lm, V, 128);
+        const CUtensorMap *th = get_tmap(h, h_target, M, 128);
+        if (!th || !tw) return AJ_ERR_CUDA;
+        p.tmap_h = *th;
+        p.tmap_w = *tw;
+        const long long tiles = (long long)((M + 255) / 256) * ((V + 255) / 256);
+        const int pairs = umma_pair_max_pairs();
+        p.grid = 2 * (int)(tiles < pairs ? tiles : pairs);
+        e = launch_umma_pair(g, p, stream);
+        h->last_path = "umma_pair_256x256";
+    } else if (h->umma_ok && !(h->flags & AJ_FLAG_ROW_TILES)) {
         UmmaPlan p;
         p.bn = vm_choose_bn(M);
         const CUtensorMap *tw = get_tmap(h, W_lm, V, 128);

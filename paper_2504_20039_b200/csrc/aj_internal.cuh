@@ -74,6 +74,12 @@ cudaError_t umma_vm_prepare();
 cudaError_t launch_umma_vm(const GemmArgs &a, const UmmaPlan &p, cudaStream_t stream);
 const char *umma_vm_path_name(int bn);
 
+// tcgen05 projection + argmax on CTA pairs (cta_group::2): 256 vocabulary entries x up to 256 rows
+// per tile.  tmap_w and tmap_h both have 64 x 128 boxes; p.grid = 2 * number of pairs.
+cudaError_t umma_pair_prepare(int num_sms);
+int umma_pair_max_pairs();
+cudaError_t launch_umma_pair(const GemmArgs &a, const UmmaPlan &p, cudaStream_t stream);
+
 struct JudgeArgs {
     unsigned long long *keys;        // [B*(K+1)]; read, then cleared for the next cycle
     const void *h_target;            // [B, K+1, d]

@@ -143,3 +143,77 @@ __device__ inline void tmem_ld32(uint32_t taddr, float (&v)[32]) {
 }
 
 }  // namespace aj
+
+// ------------------------------------------------------------------ two-SM (CTA pair) forms
+//
+// A cluster of two CTAs on the two SMs of one pair shares one tcgen05.mma: the even CTA (the
+// leader) issues it, each CTA supplies half of both operands from its own shared memory and
+// receives its half of the accumulator rows in its own tensor memory.
+
+namespace aj {
+
+__device__ inline uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+
+// Address, in the cluster-wide shared window, of the location `local` (a shared::cta address) in
+// the shared memory of the CTA with rank `rank` in this cluster.
+__device__ inline uint32_t map_to_cta(uint32_t local, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local), "r"(rank));
+    return r;
+}
+
+// All threads of both CTAs: arrive (release) and wait (acquire) at the cluster's hardware barrier.
+__device__ inline void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+// Arrive on an mbarrier that may live in the other CTA (address from map_to_cta).
+__device__ inline void mbar_arrive_cluster(uint32_t cluster_bar) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
+}
+
+// 2-D tiled TMA load into THIS CTA's shared memory whose completion bytes are counted on an
+// mbarrier given by its cluster-wide address (the leader's barrier).  No multicast: every CTA
+// fetches its own half-tiles.
+__device__ inline void tma_load_2d_pair(uint32_t dst, const CUtensorMap *tmap, int c0, int c1, uint32_t cluster_bar,
+                                        unsigned long long policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%3, %4}], [%2], %5;"
+        ::"r"(dst), "l"(tmap), "r"(cluster_bar), "r"(c0), "r"(c1), "l"(policy)
+        : "memory");
+}
+
+__device__ inline void tmem_alloc_pair(uint32_t slot, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ inline void tmem_dealloc_pair(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+
+__device__ inline void umma_bf16_pair(uint32_t d_tmem, unsigned long long adesc, unsigned long long bdesc, uint32_t idesc,
+                                      uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+// When the MMAs issued so far have completed, arrive on the mbarrier at this shared-memory offset
+// in BOTH CTAs of the pair.
+__device__ inline void umma_commit_pair(uint32_t bar) {
+    const uint16_t mask = 3;
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"(mask)
+                 : "memory");
+}
+
+}  // namespace aj

@@ -1,0 +1,308 @@
+// Tensor-core projection + running argmax for sm_100a on CTA pairs (two SMs per tile), the
+// tensor-bound regime (more than 128 rows of hidden states):
+//
+//   logit[v, m] = sum_k W[v, k] * h[m, k]        bf16 x bf16 -> fp32 in tensor memory, never stored
+//   keys[m]     = max over v of pack(logit[v, m], v)
+//
+// A tile is 256 vocabulary entries (UMMA M = 256, 128 per SM = the 128 TMEM lanes of each SM) by
+// up to 256 rows of hidden states (UMMA N, any multiple of 16).  The two CTAs of a cluster sit on
+// one SM pair; the even CTA (the leader) issues tcgen05.mma.cta_group::2 for both.  Each CTA stages
+// its own 128 rows of W and HALF of the tile's rows of h, so a k-block costs 32 KB of L2 -> SM
+// traffic per SM where the one-SM kernel needs 48 KB for the same tensor work.  Nothing is
+// multicast: every CTA fetches its own half-tiles with ordinary tiled TMA loads, and the follower's
+// loads report their bytes to the leader's barrier.
+//
+// Roles in each CTA (192 threads):
+//   warp 0      TMA producer (one thread): waits for its own stage to be free, then loads
+//               W[v0 + 128*rank .. +128, kb] and h[n0 + (N/2)*rank .. , kb] with 128-byte swizzle;
+//   warp 1      allocates tensor memory (both CTAs); in the leader one thread issues the MMAs and
+//               commits stage-release and accumulator-ready barriers to both CTAs at once;
+//   warps 2..5  epilogue: thread = one TMEM lane = one vocabulary entry; per column (row of h) the
+//               warp maximum by redux.sync on the order-preserving image of the logit, the lowest
+//               lane attaining it by ballot; lane j keeps the running (max, argmax) of column j and
+//               merges it into the row's packed key with a 64-bit atomic max when the tile is done
+//               (skipped when the key in memory already beats it).
+// Two accumulator buffers of 256 columns: the epilogue of one tile runs under the MMAs of the next.
+// No split over k.  Every wait is bounded; a wait that runs out sets the status word, and both CTAs
+// still meet at the cluster barrier before tensor memory is freed.
+#include "aj_internal.cuh"
+#include "aj_ptx.cuh"
+
+namespace aj {
+
+namespace {
+
+constexpr int BV = 256;       // vocabulary entries per tile (128 per CTA)
+constexpr int BV_CTA = 128;
+constexpr int BN = 256;       // rows of h per tile (half of them staged by each CTA)
+constexpr int BK = 64;        // bf16 elements per k-block = 128 bytes = one swizzle span
+constexpr int UMMA_K = 16;
+constexpr int NUM_THREADS = 192;
+constexpr int A_BYTES = BV_CTA * BK * 2;        // 16 KB
+constexpr int B_BYTES = (BN / 2) * BK * 2;      // 16 KB
+constexpr int STAGE_BYTES = A_BYTES + B_BYTES;  // per CTA
+constexpr int STAGES = 6;
+constexpr int TMEM_COLS = 2 * BN;
+constexpr int NCH = BN / 32;
+constexpr int BAR_BYTES = 8 * (2 * STAGES + 4) + 16;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + BAR_BYTES + 1024;
+
+__device__ inline uint32_t ordered_image(float x) {
+    const uint32_t b = __float_as_uint(x + 0.0f);  // -0.0 + 0.0 = +0.0: the two zeros tie
+    return b ^ ((uint32_t)((int32_t)b >> 31) | 0x80000000u);
+}
+
+__device__ inline uint32_t warp_max(uint32_t x) {
+    uint32_t r;
+    asm volatile("redux.sync.max.u32 %0, %1, 0xffffffff;" : "=r"(r) : "r"(x));
+    return r;
+}
+
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_h,
+                 int M, int V, int d, int n_n, int n_v, int stream_w,
+                 unsigned long long *__restrict__ keys, int *__restrict__ status) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;  // the same offset in both CTAs: one descriptor serves both
+    uint8_t *smem = smem_raw + (base - raw);
+
+    const uint32_t bar_base = base + STAGES * STAGE_BYTES;
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };                      // used in the leader only
+    auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+    auto acc_full_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
+    auto acc_empty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };  // used in the leader only
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + STAGES * STAGE_BYTES + 8 * (2 * STAGES + 4));
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5;  // warp-uniform
+    const int lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();  // 0 = leader
+    const int pair = blockIdx.x >> 1;
+    const int num_pairs = gridDim.x >> 1;
+    const int num_kb = d / BK;
+    const int num_tiles = n_n * n_v;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; s++) {
+            mbar_init(full_bar(s), 1);   // the leader's producer; bytes arrive from both CTAs
+            mbar_init(empty_bar(s), 1);  // one commit from the leader's MMA thread
+        }
+        for (int a = 0; a < 2; a++) {
+            mbar_init(acc_full_bar(a), 1);
+            mbar_init(acc_empty_bar(a), 8);  // four epilogue warps in each of the two CTAs
+        }
+        *abort_flag = 0;
+        fence_barrier_init();
+    }
+    if (warp == 1) tmem_alloc_pair(smem_u32(const_cast<uint32_t *>(tmem_slot)), TMEM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();  // the peer's barriers exist before anything is sent to them
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    // Programmatic dependent launch: nothing the caller passed is read before this wait returns.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
+    auto give_up = [&]() {
+        *abort_flag = 1;
+        atomicCAS(status, DEV_OK, DEV_TIMEOUT);
+    };
+    auto tile_rows = [&](int n_tile) {  // UMMA N of this tile: valid rows rounded up to 16
+        const int rows_valid = min(BN, M - n_tile * BN);
+        return max(16, (rows_valid + 15) & ~15);
+    };
+
+    if (warp == 0) {
+        if (lane == 0) {
+            // ------------------------------------------------------------ TMA producer
+            const unsigned long long pol_h = policy_evict_last();
+            const unsigned long long pol_w = stream_w ? policy_evict_first() : policy_evict_normal();
+            int s = 0;
+            uint32_t ph = 0;
+            bool ok = true;
+            for (int t = pair; ok && t < num_tiles; t += num_pairs) {
+                const int n_tile = t % n_n, v_tile = t / n_n;
+                const int n_inst = tile_rows(n_tile);
+                const int w_row = v_tile * BV + (int)rank * BV_CTA;
+                const int h_row = n_tile * BN + (int)rank * (n_inst >> 1);
+                for (int kb = 0; kb < num_kb; kb++) {
+                    if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) {
+                        give_up();
+                        ok = false;
+                        break;
+                    }
+                    const uint32_t leader_full = map_to_cta(full_bar(s), 0);
+                    if (rank == 0) mbar_expect_tx(full_bar(s), 2 * STAGE_BYTES);
+                    const uint32_t a_dst = base + s * STAGE_BYTES;
+                    tma_load_2d_pair(a_dst, &tmap_w, kb * BK, w_row, leader_full, pol_w);
+                    tma_load_2d_pair(a_dst + A_BYTES, &tmap_h, kb * BK, h_row, leader_full, pol_h);
+                    if (++s == STAGES) {
+                        s = 0;
+                        ph ^= 1u;
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && rank == 0) {
+            // ------------------------------------------- MMA issuer (leader CTA only)
+            int s = 0;
+            uint32_t ph = 0;
+            bool ok = true;
+            int it = 0;
+            for (int t = pair; ok && t < num_tiles; t += num_pairs, ++it) {
+                const uint32_t idesc = instr_desc(BV, tile_rows(t % n_n));
+                const int ab = it & 1;
+                const uint32_t aph = (uint32_t)(it >> 1) & 1u;
+                if (!mbar_wait(acc_empty_bar(ab), aph ^ 1u, abort_flag)) {
+                    give_up();
+                    break;
+                }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(ab * BN);
+                for (int kb = 0; kb < num_kb; kb++) {
+                    if (!mbar_wait(full_bar(s), ph, abort_flag)) {
+                        give_up();
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint32_t a_addr = base + s * STAGE_BYTES;
+                    const unsigned long long adesc = smem_desc_sw128(a_addr);
+                    const unsigned long long bdesc = smem_desc_sw128(a_addr + A_BYTES);
+#pragma unroll
+                    for (int k = 0; k < BK / UMMA_K; k++)
+                        umma_bf16_pair(d_tmem, adesc + 2ull * k, bdesc + 2ull * k, idesc, (uint32_t)((kb | k) != 0));
+                    umma_commit_pair(empty_bar(s));  // frees the stage in both CTAs
+                    if (++s == STAGES) {
+                        s = 0;
+                        ph ^= 1u;
+                    }
+                }
+                if (ok) umma_commit_pair(acc_full_bar(ab));  // the accumulator halves in both CTAs are complete
+            }
+        }
+    } else {
+        // -------------------------------------------------------------------- epilogue
+        const int q = warp & 3;  // TMEM lane quadrant this warp may read
+        int it = 0;
+        for (int t = pair; t < num_tiles; t += num_pairs, ++it) {
+            const int n_tile = t % n_n, v_tile = t / n_n;
+            const int n_inst = tile_rows(n_tile);
+            const int ab = it & 1;
+            const uint32_t aph = (uint32_t)(it >> 1) & 1u;
+            // the whole warp takes one decision, so the aligned TMEM loads below stay converged
+            if (!__all_sync(0xffffffffu, mbar_wait(acc_full_bar(ab), aph, abort_flag))) {
+                give_up();
+                break;
+            }
+            tc_fence_after();
+            const int v_first = v_tile * BV + (int)rank * BV_CTA + q * 32;  // vocabulary entry of lane 0
+            const bool v_ok = v_first + lane < V;                            // entries past V hold zero-filled junk
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ab * BN);
+            uint32_t best_u[NCH];  // lane j, chunk c: maximum of column 32c + j over this warp's 32 entries
+            int best_i[NCH];
+#pragma unroll
+            for (int c = 0; c < NCH; c++) {
+                best_u[c] = 0u;
+                best_i[c] = 0;
+                if (c * 32 < n_inst) {  // warp-uniform
+                    float v[32];
+                    tmem_ld32(taddr + c * 32, v);
+#pragma unroll
+                    for (int j = 0; j < 32; j++) {
+                        const uint32_t u = v_ok ? ordered_image(v[j]) : 0u;
+                        const uint32_t m = warp_max(u);
+                        const uint32_t who = __ballot_sync(0xffffffffu, u == m);
+                        if (lane == j) {
+                            best_u[c] = m;
+                            best_i[c] = v_first + __ffs(who) - 1;  // the lowest entry that attains the maximum
+                        }
+                    }
+                }
+            }
+            // the accumulator buffer is drained: hand it back to the leader's MMA thread
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(acc_empty_bar(ab), 0));
+            // merge this tile's column maxima into the rows' keys
+#pragma unroll
+            for (int c = 0; c < NCH; c++) {
+                const int row = n_tile * BN + c * 32 + lane;
+                if (c * 32 < n_inst && row < M && best_u[c] != 0u) {
+                    const unsigned long long key = ((unsigned long long)best_u[c] << 32) | (uint32_t)(~(uint32_t)best_i[c]);
+                    if (key > *reinterpret_cast<volatile unsigned long long *>(&keys[row])) atomicMax(&keys[row], key);
+                }
+            }
+        }
+    }
+
+    __syncwarp();
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1 && *abort_flag) {
+        // copies or MMAs may still be in flight after an abort: give them time to land
+        const unsigned long long t0 = globaltimer_ns();
+        while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
+    }
+    cluster_sync_all();  // neither CTA leaves, or frees tensor memory, while the other may still signal it
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc_pair(tmem_base, TMEM_COLS);
+    }
+}
+
+int g_max_pairs = 0;
+
+}  // namespace
+
+cudaError_t umma_pair_prepare(int num_sms) {
+    cudaError_t e = cudaFuncSetAttribute(umma_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    // how many CTA pairs can be resident at once (pairs need both SMs of a pair free)
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)(num_sms & ~1));
+    cfg.blockDim = dim3(NUM_THREADS);
+    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    int clusters = 0;
+    e = cudaOccupancyMaxActiveClusters(&clusters, umma_pair_kernel, &cfg);
+    if (e != cudaSuccess) return e;
+    if (clusters < 1) return cudaErrorInvalidConfiguration;
+    g_max_pairs = clusters < num_sms / 2 ? clusters : num_sms / 2;
+    return cudaSuccess;
+}
+
+int umma_pair_max_pairs() { return g_max_pairs; }
+
+cudaError_t launch_umma_pair(const GemmArgs &a, const UmmaPlan &p, cudaStream_t stream) {
+    const int n_n = (a.M + BN - 1) / BN;
+    const int n_v = (a.V + BV - 1) / BV;
+    const int stream_w = (n_n == 1) ? 1 : 0;  // W is read by one pair only: do not keep it in L2
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)p.grid);  // 2 CTAs per pair
+    cfg.blockDim = dim3(NUM_THREADS);
+    cfg.dynamicSmemBytes = SMEM_BYTES;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = 2;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    return cudaLaunchKernelEx(&cfg, umma_pair_kernel, p.tmap_w, p.tmap_h, a.M, a.V, a.d, n_n, n_v, stream_w, a.keys,
+                              a.status);
+}
+
+}  // namespace aj

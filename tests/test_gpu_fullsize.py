@@ -80,17 +80,17 @@ def test_c2_8b_batch1_every_row():
 
 
 def test_c3_8b_batched_sampled_sequences():
-    reps = _run_workload(gen.C3, (gen.C3.tau,), 8, "umma_vm_128x256")
+    reps = _run_workload(gen.C3, (gen.C3.tau,), 8, "umma_pair_256x256")
     assert reps[0].seqs >= 8 and reps[0].seqs_exempt <= reps[0].seqs // 2
 
 
 def test_c5_sweep_points_on_the_8b_shape():
     # smallest, the HBM/tensor crossover, and the largest point of the sweep
-    for B, K, path in [(1, 8, "umma_vm_128x32"), (8, 32, "umma_vm_128x256"), (256, 8, "umma_vm_128x256"), (256, 64, "umma_vm_128x256")]:
+    for B, K, path in [(1, 8, "umma_vm_128x32"), (8, 32, "umma_pair_256x256"), (256, 8, "umma_pair_256x256"), (256, 64, "umma_pair_256x256")]:
         reps = _run_workload(gen.sweep_config(B, K), (0.5,), 3, path)
         assert reps[0].seqs >= min(B, 3)
 
 
 def test_c4_70b_sampled_sequences_tau_sweep():
-    reps = _run_workload(gen.C4, gen.C4_TAUS, 4, "umma_vm_128x256")
+    reps = _run_workload(gen.C4, gen.C4_TAUS, 4, "umma_pair_256x256")
     assert len(reps) == 9 and all(r.seqs >= 4 for r in reps)

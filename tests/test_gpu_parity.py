@@ -92,11 +92,13 @@ SHAPES = [
     ("many_vocab_tiles", 3, 7, 128, 64, 70001),   # more vocabulary tiles than SMs, odd tail
     ("v_below_one_tile", 2, 3, 64, 64, 100),
     ("window_above_64", 2, 100, 64, 0, 700),      # K > 64: several ballots; target-only features
+    ("pair_ragged_rows", 9, 63, 320, 64, 3000),   # M = 576 = 2*256 + 64: a 64-row tail tile on the two-SM kernel; V = 11*256 + 184
+    ("pair_odd_tail", 3, 86, 192, 0, 1111),       # M = 261 = 256 + 5: a 16-row tail tile, 3 k-blocks
 ]
 
 
 @pytest.mark.parametrize("shape", SHAPES, ids=[s[0] for s in SHAPES])
-@pytest.mark.parametrize("flags", [0, 4, 1], ids=["umma_vm", "umma_rows", "simt"])
+@pytest.mark.parametrize("flags", [0, 8, 4, 1], ids=["umma_default", "umma_one_sm", "umma_rows", "simt"])
 def test_cut_down_shapes_bf16(shape, flags):
     name, B, K, d, dd, V = shape
     cfg = gen.Config(name, B=B, K=K, d=d, d_draft=dd, V=V, sigma_W=0.2, sigma_w=0.05, match_lo=0.5, match_hi=0.95, seed=3)
@@ -132,7 +134,7 @@ def test_ties_zeros_and_out_of_range_draft_tokens():
     tok = gen.plant_draft_tokens(cfg, y)
     tok[0, 1] = -5          # ids outside the vocabulary are data: they simply never match
     tok[1, 2] = cfg.V + 9
-    for flags in (0, 4, 1):
+    for flags in (0, 8, 4, 1):
         case = DeviceCase(cfg, W, ht, hd, w, flags=flags)
         try:
             o = orc.verify(ht, hd, W, tok, w, 0.0, 0.5, cfg.dtype)
@@ -156,6 +158,41 @@ def test_ties_zeros_and_out_of_range_draft_tokens():
             case.close()
 
 
+def test_two_sm_kernel_ties_within_and_across_the_pair():
+    # More than 128 rows selects the two-SM kernel.  The winner of every row is duplicated 37 entries
+    # later (same warp or the next one) and 128 entries later (the other SM of the pair, or the next
+    # tile): the lowest index must win whichever SM, warp or tile sees the copy first.
+    orc = _oracle()
+    cfg = gen.Config("pair_ties", B=3, K=50, d=128, d_draft=64, V=900, sigma_w=0.05, seed=12)
+    W, ht, hd, w = _host_case(cfg)
+    W = W.copy()
+    y0 = _oracle_y(cfg, W, ht)
+    for v in np.unique(y0):
+        for off in (37, 128):
+            if v + off < cfg.V:
+                W[v + off] = W[v]
+    y = _oracle_y(cfg, W, ht)
+    tok = gen.plant_draft_tokens(cfg, y)
+    o = orc.verify(ht, hd, W, tok, w, 0.0, 0.5, cfg.dtype)
+    assert (o.gap == 0).sum() >= cfg.M // 2  # most rows really are tied
+    for flags in (0, 8):
+        case = DeviceCase(cfg, W, ht, hd, w, flags=flags)
+        try:
+            g = case.run(tok, 0.5)
+            assert g.path == ("umma_pair_256x256" if flags == 0 else "umma_vm_128x256")
+            np.testing.assert_array_equal(g.target_tok, o.target_tok)
+            np.testing.assert_array_equal(g.accept_len, o.accept_len)
+            np.testing.assert_array_equal(g.next_tok, o.next_tok)
+        finally:
+            case.close()
+    case = DeviceCase(cfg, np.zeros_like(W), ht, hd, w)
+    try:
+        g = case.run(np.zeros((cfg.B, cfg.K), np.int32), 0.5)
+        assert (g.target_tok == 0).all() and (g.accept_len == cfg.K).all() and (g.top1 == 0).all()
+    finally:
+        case.close()
+
+
 def test_all_negative_logits_are_not_beaten_by_the_zero_filled_tail():
     # V = 300 leaves 212 zero-filled columns in the last 256-wide (or 128-wide) tile; make every
     # real logit negative so that an unmasked tail (logit 0) would win.
@@ -167,7 +204,7 @@ def test_all_negative_logits_are_not_beaten_by_the_zero_filled_tail():
     y = _oracle_y(cfg, W, ht)
     tok = gen.plant_draft_tokens(cfg, y)
     o = orc.verify(ht, None, W, tok, w, 0.0, 0.5, cfg.dtype)
-    for flags in (0, 4):
+    for flags in (0, 8, 4):  # M = 153: two-SM kernel, one-SM kernel, row tiles
         case = DeviceCase(cfg, W, ht, None, w, flags=flags)
         try:
             g = case.run(tok, 0.5)

@@ -105,7 +105,7 @@ class ClockSampler:
 class GpuWorkload:
     """One workload resident on the device: rotating copies of W_lm, inputs, outputs, handles."""
 
-    def __init__(self, cfg: gen.Config, device: int, w_copies: int, W_host=None):
+    def __init__(self, cfg: gen.Config, device: int, w_copies: int, W_host=None, flags: int = 0):
         import torch
 
         import paper_2504_20039_b200 as aj
@@ -125,8 +125,8 @@ class GpuWorkload:
         self.acc = torch.empty(cfg.B, **i32)
         self.nxt = torch.empty(cfg.B, **i32)
         self.tt = torch.empty((cfg.B, cfg.K + 1), **i32)
-        self.handle = aj.Handle(device, cfg.B, cfg.K, cfg.d, cfg.d_draft, cfg.V, aj.AJ_BF16, aj.AJ_W_VD, 0)
-        self.handle_t = aj.Handle(device, cfg.B, cfg.K, cfg.d, cfg.d_draft, cfg.V, aj.AJ_BF16, aj.AJ_W_VD, aj.AJ_FLAG_TIME_KERNELS)
+        self.handle = aj.Handle(device, cfg.B, cfg.K, cfg.d, cfg.d_draft, cfg.V, aj.AJ_BF16, aj.AJ_W_VD, flags)
+        self.handle_t = aj.Handle(device, cfg.B, cfg.K, cfg.d, cfg.d_draft, cfg.V, aj.AJ_BF16, aj.AJ_W_VD, flags | aj.AJ_FLAG_TIME_KERNELS)
         # draft tokens planted against the device's own greedy tokens (a benchmark input, never an oracle input)
         self.tok = torch.from_numpy(gen.random_draft_tokens(cfg)).to(dev)
         self.step(self.handle, 0)
@@ -185,6 +185,36 @@ class GpuWorkload:
         self.handle_t.destroy()
 
 
+# DRAM traffic per launch of the projection kernel (dram__bytes_read.sum + dram__bytes_write.sum of one
+# ncu capture; summaries under profiles/).  A figure is reported only while the kernel's sources still
+# hash to what was captured.
+CSRC = os.path.join(ROOT, "paper_2504_20039_b200", "csrc")
+NCU_TRAFFIC = {
+    # (workload, kernel configuration): (bytes per launch, kernel source files, sha1 of those files)
+}
+
+
+def _sources_sha(files):
+    import hashlib
+
+    h = hashlib.sha1()
+    for f in files:
+        with open(os.path.join(CSRC, f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:12]
+
+
+def traffic_of(cfg: gen.Config, path: str):
+    ent = NCU_TRAFFIC.get((cfg.name, path))
+    if not ent:
+        return None
+    byts, files, sha = ent
+    try:
+        return byts if _sources_sha(files) == sha else None
+    except OSError:
+        return None
+
+
 def roofline_of(cfg: gen.Config, gemm_ms: float, pk):
     """Roofline of the projection kernel: W streamed once from HBM vs 2*M*d*V flops on the tensor pipe."""
     flops = 2.0 * cfg.M * cfg.d * cfg.V
@@ -202,8 +232,8 @@ def roofline_of(cfg: gen.Config, gemm_ms: float, pk):
             "kernel_ms": gemm_ms, "algorithmic_flops": flops}
 
 
-def bench_one(cfg, device, steps, warmup, barrier, reduce_max, pk, w_copies, W_host=None, with_e2e=True):
-    wl = GpuWorkload(cfg, device, w_copies, W_host)
+def bench_one(cfg, device, steps, warmup, barrier, reduce_max, pk, w_copies, W_host=None, with_e2e=True, flags=0):
+    wl = GpuWorkload(cfg, device, w_copies, W_host, flags)
     try:
         wl.run(wl.handle, warmup)
         with ClockSampler(device) as cs:
@@ -219,7 +249,8 @@ def bench_one(cfg, device, steps, warmup, barrier, reduce_max, pk, w_copies, W_h
         assert wl.handle.last_status() == wl.aj.AJ_OK and wl.handle_t.last_status() == wl.aj.AJ_OK
         res = {
             "ms_per_step": ms / steps, "clocks": clocks, "path": wl.handle.last_gemm_path(),
-            "roofline": roofline_of(cfg, gemm_mean, pk), "gemm_ms_min": gemm_min, "gemm_launches_timed": n,
+            "roofline": dict(roofline_of(cfg, gemm_mean, pk), traffic=traffic_of(cfg, wl.handle.last_gemm_path())),
+            "gemm_ms_min": gemm_min, "gemm_launches_timed": n,
             "launches_per_step": wl.handle.last_launch_count(),
             "mean_accept_len": float(wl.acc.float().mean().item()),
         }
@@ -232,22 +263,27 @@ def bench_one(cfg, device, steps, warmup, barrier, reduce_max, pk, w_copies, W_h
         wl.close()
 
 
-def cpu_baseline(cfg: gen.Config, W_host=None):
-    """The CPU oracle, as it stands, on a bounded sample of the workload (whole sequences)."""
+def cpu_baseline(cfg: gen.Config, W_host=None, budget_s: float = 12.0):
+    """The CPU oracle, as it stands, on a bounded sample of the workload: whole sequences (K+1 rows
+    against the full vocabulary), one per pass, cycling through the batch until about `budget_s`
+    seconds of CPU work have been timed (at least one pass)."""
     from oracle import aj_oracle as orc
 
-    n_seq = 1  # one whole sequence: (K+1) rows against the full vocabulary
-    sub = gen.scaled(cfg, B=n_seq)
+    sub = gen.scaled(cfg, B=1)
     W = gen.make_W(cfg) if W_host is None else W_host
     ht, hd = gen.make_hidden(cfg)
-    ht, hd = ht[:n_seq], hd[:n_seq]
     w = gen.make_judge(cfg)
     tok = gen.random_draft_tokens(sub)
-    t0 = time.perf_counter()
-    r = orc.verify(ht, hd, W, tok, w, cfg.judge_b, cfg.tau, cfg.dtype)
-    dt = time.perf_counter() - t0
-    return {"value": n_seq * cfg.K / dt, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle",
-            "sample": f"{n_seq} of {cfg.B} sequences ({cfg.K + 1} rows x V={cfg.V}, d={cfg.d}), {dt:.2f} s, fp64 loops"}, r
+    passes, dt, r = 0, 0.0, None
+    while passes == 0 or dt < budget_s:
+        b = passes % cfg.B
+        t0 = time.perf_counter()
+        r = orc.verify(ht[b : b + 1], None if hd is None else hd[b : b + 1], W, tok, w, cfg.judge_b, cfg.tau, cfg.dtype)
+        dt += time.perf_counter() - t0
+        passes += 1
+    return {"value": passes * cfg.K / dt, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle",
+            "sample": f"{passes} passes of one whole sequence each ({cfg.K + 1} rows x V={cfg.V}, d={cfg.d}; batch of {cfg.B}), "
+                      f"{dt:.1f} s of fp64 loops"}, r
 
 
 def reference_arm(args):
@@ -262,10 +298,10 @@ def reference_arm(args):
     warmup = args.warmup if args.warmup is not None else 1
     W = gen.make_W(cfg)
     for _ in range(warmup):
-        cpu_baseline(cfg, W)
+        cpu_baseline(cfg, W, budget_s=0.0)
     t0 = time.perf_counter()
     for _ in range(steps):
-        base, _ = cpu_baseline(cfg, W)
+        base, _ = cpu_baseline(cfg, W, budget_s=0.0)  # one pass = one whole sequence per step
     dt = (time.perf_counter() - t0) / steps
     value = cfg.K / dt  # one sequence per step
     line = {
@@ -290,6 +326,7 @@ def main():
     ap.add_argument("--no-extra", action="store_true", help="skip the batched configurations reported under 'extra'")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer (end-to-end) measurement; for profiler captures")
+    ap.add_argument("--flags", type=int, default=0, help="extra aj_create flags (kernel selection switches, for comparisons)")
     ap.add_argument("--w-copies", type=int, default=None, help="copies of W_lm to rotate over (default 3, or 2 for the 70B shape)")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -326,7 +363,7 @@ def main():
     copies = args.w_copies or (3 if head.d * head.V * 2 < 1.5e9 else 2)
 
     W_host = gen.make_W(head)
-    r = bench_one(head, local, steps, warmup, barrier, reduce_max, pk, copies, W_host, with_e2e=not args.no_e2e)
+    r = bench_one(head, local, steps, warmup, barrier, reduce_max, pk, copies, W_host, with_e2e=not args.no_e2e, flags=args.flags)
     positions = head.B * head.K * world
     line = {
         "metric": METRIC, "value": positions / (r["ms_per_step"] * 1e-3), "unit": UNIT, "n_gpus": world, "steps": steps,
@@ -355,7 +392,7 @@ def main():
         for cfg in todo:
             same_W = cfg.d == head.d and cfg.V == head.V
             n = max(20, int(0.4 / max(2.0 * cfg.M * cfg.d * cfg.V / 1.2e15, 1.7e-4)))
-            rr = bench_one(cfg, local, n, 5, barrier, reduce_max, pk, 2 if not same_W else copies, W_host if same_W else None, with_e2e=False)
+            rr = bench_one(cfg, local, n, 5, barrier, reduce_max, pk, 2 if not same_W else copies, W_host if same_W else None, with_e2e=False, flags=args.flags)
             extra.append({"workload": cfg.name, "B": cfg.B, "K": cfg.K, "d": cfg.d, "V": cfg.V, "steps": n,
                           "ms_per_step": rr["ms_per_step"], "value": cfg.B * cfg.K * world / (rr["ms_per_step"] * 1e-3), "unit": UNIT,
                           "gemm_path": rr["path"], "roofline": rr["roofline"], "clocks": rr["clocks"]})

@@ -65,7 +65,7 @@ enum {
  * Create a handle for fixed model dimensions on CUDA device `device`.
  *   max_B, max_K  largest batch and window a later call may use (1 <= K <= 1024)
  *   d, d_draft, V target hidden width, draft hidden width (0 = the judge sees target features
- *                 only, the paper's vLLM variant, Appendix D), vocabulary size
+ *                 only, as in the paper's appendix "vLLM Inference Implementation Details"), vocabulary size
  *   dtype, layout storage of the hidden states and of W_lm
  * The handle owns a small device workspace: 8 bytes per row (max_B*(max_K+1)) for the per-row
  * packed (max, argmax) keys, a status word, and staging buffers for aj_verify_host.  This is the
@@ -138,6 +138,18 @@ aj_status aj_gemm_ms_stats(aj_handle h, float *mean_ms, float *min_ms, int *coun
 /* Number of kernels of this library that the most recent aj_verify / aj_verify_host call launched
  * (the projection kernel and the judge kernel; the memset that clears the keys is not counted). */
 int aj_last_launch_count(aj_handle h);
+
+/*
+ * How the two-SM projection kernel cuts a batch of M = B*(K+1) rows against a vocabulary of V entries
+ * (host arithmetic only, no device needed; for tests and diagnostics).  out receives
+ *   [0] blocks of 256 vocabulary entries        [1] row tiles (each at most 256 rows)
+ *   [2],[3] row tile i holds out[2] + (i < out[3]) units of 16 rows
+ *   [4] rows of h_target each SM of a pair stages per 64-column block
+ *   [5] groups the row tiles are walked in (each group against the whole vocabulary, so that a
+ *       group's rows of h_target stay in L2)    [6],[7] group g holds out[6] + (g < out[7]) row tiles
+ * Errors: AJ_ERR_INVALID_ARG.
+ */
+aj_status aj_pair_schedule(int M, int d, int V, int32_t out[8]);
 
 /* Name of the projection kernel configuration the most recent call used, e.g. "umma_128x256". */
 const char *aj_last_gemm_path(aj_handle h);

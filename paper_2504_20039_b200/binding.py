@@ -19,7 +19,7 @@ AJ_FLAG_FORCE_SIMT, AJ_FLAG_TIME_KERNELS, AJ_FLAG_ROW_TILES, AJ_FLAG_ONE_SM = 1,
 
 EXPORTS = (
     "aj_create", "aj_verify", "aj_verify_host", "aj_last_status", "aj_last_gemm_ms", "aj_gemm_ms_stats", "aj_last_launch_count",
-    "aj_last_gemm_path", "aj_destroy", "aj_status_string", "aj_version", "aj_verify_static",
+    "aj_last_gemm_path", "aj_pair_schedule", "aj_destroy", "aj_status_string", "aj_version", "aj_verify_static",
 )
 
 _lib = None
@@ -64,6 +64,8 @@ def lib() -> ctypes.CDLL:
         L.aj_status_string.restype = ctypes.c_char_p
         L.aj_verify_static.argtypes = [vp, vp, vp, vp, vp, cf, cf, ci, ci, ci, ci, ci, ci, ci, vp, vp, vp, vp, vp, vp, vp]
         L.aj_verify_static.restype = ci
+        L.aj_pair_schedule.argtypes = [ci, ci, ci, ctypes.POINTER(ctypes.c_int32)]
+        L.aj_pair_schedule.restype = ci
         L.aj_version.argtypes = []
         L.aj_version.restype = ctypes.c_char_p
         _lib = L
@@ -90,6 +92,16 @@ def _ptr(t):
 
 
 AJ_STATIC_MAX_ROWS = 32768
+
+
+def pair_schedule(M: int, d: int, V: int) -> dict:
+    """aj_pair_schedule: how the two-SM kernel tiles M rows against V vocabulary entries (host arithmetic)."""
+    out = (ctypes.c_int32 * 8)()
+    st = lib().aj_pair_schedule(M, d, V, out)
+    if st != AJ_OK:
+        raise AjError(st, "aj_pair_schedule")
+    keys = ("n_v", "n_n", "u_base", "u_rem", "box_rows", "n_groups", "g_base", "g_rem")
+    return dict(zip(keys, (int(x) for x in out)))
 
 
 def verify_static(h_target, h_draft, W_lm, draft_tok, judge_w, judge_b: float, tau: float, B: int, K: int, d: int,

@@ -265,12 +265,13 @@ aj_status aj_verify(aj_handle h, const void *h_target, const void *h_draft, cons
         // tensor-bound regime: two-SM tiles of 256 vocabulary entries x up to 256 rows
         UmmaPlan p;
         p.bn = 256;
+        const PairSched sc = pair_schedule(M, V, d);
         const CUtensorMap *tw = get_tmap(h, W_lm, V, 128);
-        const CUtensorMap *th = get_tmap(h, h_target, M, 128);
+        const CUtensorMap *th = get_tmap(h, h_target, M, sc.box_rows);
         if (!th || !tw) return AJ_ERR_CUDA;
         p.tmap_h = *th;
         p.tmap_w = *tw;
-        const long long tiles = (long long)((M + 255) / 256) * ((V + 255) / 256);
+        const long long tiles = (long long)sc.n_n * sc.n_v;
         const int pairs = umma_pair_max_pairs();
         p.grid = 2 * (int)(tiles < pairs ? tiles : pairs);
         e = launch_umma_pair(g, p, stream);
@@ -408,6 +409,20 @@ aj_status aj_gemm_ms_stats(aj_handle h, float *mean_ms, float *min_ms, int *coun
 }
 
 int aj_last_launch_count(aj_handle h) { return h ? h->last_launches : 0; }
+
+aj_status aj_pair_schedule(int M, int d, int V, int32_t out[8]) {
+    if (!out || M < 1 || d < 1 || V < 1) return AJ_ERR_INVALID_ARG;
+    const PairSched sc = pair_schedule(M, V, d);
+    out[0] = sc.n_v;
+    out[1] = sc.n_n;
+    out[2] = sc.u_base;
+    out[3] = sc.u_rem;
+    out[4] = sc.box_rows;
+    out[5] = sc.n_groups;
+    out[6] = sc.g_base;
+    out[7] = sc.g_rem;
+    return AJ_OK;
+}
 
 const char *aj_last_gemm_path(aj_handle h) { return h ? h->last_path : "none"; }
 

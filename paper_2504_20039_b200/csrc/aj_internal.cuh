@@ -75,7 +75,17 @@ cudaError_t launch_umma_vm(const GemmArgs &a, const UmmaPlan &p, cudaStream_t st
 const char *umma_vm_path_name(int bn);
 
 // tcgen05 projection + argmax on CTA pairs (cta_group::2): 256 vocabulary entries x up to 256 rows
-// per tile.  tmap_w and tmap_h both have 64 x 128 boxes; p.grid = 2 * number of pairs.
+// per tile.  tmap_w has a 64 x 128 box, tmap_h a 64 x pair_schedule().box_rows box; p.grid = 2 *
+// number of pairs.
+struct PairSched {
+    int n_v;               // blocks of 256 vocabulary entries
+    int n_n;               // row tiles
+    int u_base, u_rem;     // row tile i holds u_base + (i < u_rem) units of 16 rows
+    int box_rows;          // rows of h each CTA of a pair stages per k-block
+    int n_groups;          // row tiles are walked in groups ...
+    int g_base, g_rem;     // ... group g holds g_base + (g < g_rem) row tiles
+};
+PairSched pair_schedule(int M, int V, int d);
 cudaError_t umma_pair_prepare(int num_sms);
 int umma_pair_max_pairs();
 cudaError_t launch_umma_pair(const GemmArgs &a, const UmmaPlan &p, cudaStream_t stream);

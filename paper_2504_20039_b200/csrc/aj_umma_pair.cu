@@ -5,12 +5,17 @@
 //   keys[m]     = max over v of pack(logit[v, m], v)
 //
 // A tile is 256 vocabulary entries (UMMA M = 256, 128 per SM = the 128 TMEM lanes of each SM) by
-// up to 256 rows of hidden states (UMMA N, any multiple of 16).  The two CTAs of a cluster sit on
-// one SM pair; the even CTA (the leader) issues tcgen05.mma.cta_group::2 for both.  Each CTA stages
-// its own 128 rows of W and HALF of the tile's rows of h, so a k-block costs 32 KB of L2 -> SM
-// traffic per SM where the one-SM kernel needs 48 KB for the same tensor work.  Nothing is
-// multicast: every CTA fetches its own half-tiles with ordinary tiled TMA loads, and the follower's
-// loads report their bytes to the leader's barrier.
+// up to 256 rows of hidden states (UMMA N, any multiple of 16).  The rows are cut into the fewest
+// tiles of at most 256 rows and spread over them evenly in units of 16 rows (2112 rows = 6 tiles of
+// 240 + 3 of 224), so no tensor work is spent on padding and all tiles take nearly the same time,
+// which keeps the pairs that share a block of W in step and that block in L2.  When h_target
+// outgrows L2 the row tiles are walked in groups, each group against the whole vocabulary.
+//
+// The two CTAs of a cluster sit on one SM pair; the even CTA (the leader) issues
+// tcgen05.mma.cta_group::2 for both.  Each CTA stages its own 128 rows of W and HALF of the tile's
+// rows of h, so a k-block costs at most 32 KB of L2 -> SM traffic per SM where the one-SM kernel
+// needs 48 KB for the same tensor work.  Nothing is multicast: every CTA fetches its own half-tiles
+// with ordinary tiled TMA loads, and the follower's loads report their bytes to the leader's barrier.
 //
 // Roles in each CTA (192 threads):
 //   warp 0      TMA producer (one thread): waits for its own stage to be free, then loads
@@ -58,9 +63,38 @@ __device__ inline uint32_t warp_max(uint32_t x) {
     return r;
 }
 
+struct Tile {
+    int v_tile;  // block of 256 vocabulary entries
+    int row0;    // first row of h
+    int n_inst;  // rows in the tile = UMMA N, a multiple of 16
+};
+
+// Tile t of the schedule.  Row tiles come in groups; a group is walked against every vocabulary
+// block (row tile fastest) before the next group starts.  Consecutive tiles, which run on
+// neighbouring pairs at the same time, share a block of W.  Which row tile of the group a pair gets
+// rotates with the vocabulary block, so that pairs whose number is a multiple of the group size
+// apart do not always get the larger (or the smaller) row tiles and drift away from the pairs they
+// share W with.
+__device__ inline Tile decode_tile(const PairSched &sc, int t) {
+    int g = 0, start = 0, sz = sc.g_base + (0 < sc.g_rem ? 1 : 0);
+    while (g + 1 < sc.n_groups && t >= start + sz * sc.n_v) {
+        start += sz * sc.n_v;
+        ++g;
+        sz = sc.g_base + (g < sc.g_rem ? 1 : 0);
+    }
+    const int first = g * sc.g_base + min(g, sc.g_rem);
+    const int local = t - start;
+    Tile r;
+    r.v_tile = local / sz;
+    const int n_tile = first + (local % sz + r.v_tile) % sz;
+    r.row0 = 16 * (n_tile * sc.u_base + min(n_tile, sc.u_rem));
+    r.n_inst = 16 * (sc.u_base + (n_tile < sc.u_rem ? 1 : 0));
+    return r;
+}
+
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_h,
-                 int M, int V, int d, int n_n, int n_v, int stream_w,
+                 int M, int V, int d, PairSched sc, int stream_w,
                  unsigned long long *__restrict__ keys, int *__restrict__ status) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -81,7 +115,8 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
     const int pair = blockIdx.x >> 1;
     const int num_pairs = gridDim.x >> 1;
     const int num_kb = d / BK;
-    const int num_tiles = n_n * n_v;
+    const int num_tiles = sc.n_n * sc.n_v;
+    const uint32_t stage_tx = 2u * (uint32_t)(A_BYTES + sc.box_rows * BK * 2);  // bytes both CTAs load per stage
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; s++) {
@@ -109,10 +144,6 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
         *abort_flag = 1;
         atomicCAS(status, DEV_OK, DEV_TIMEOUT);
     };
-    auto tile_rows = [&](int n_tile) {  // UMMA N of this tile: valid rows rounded up to 16
-        const int rows_valid = min(BN, M - n_tile * BN);
-        return max(16, (rows_valid + 15) & ~15);
-    };
 
     if (warp == 0) {
         if (lane == 0) {
@@ -123,10 +154,9 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
             uint32_t ph = 0;
             bool ok = true;
             for (int t = pair; ok && t < num_tiles; t += num_pairs) {
-                const int n_tile = t % n_n, v_tile = t / n_n;
-                const int n_inst = tile_rows(n_tile);
-                const int w_row = v_tile * BV + (int)rank * BV_CTA;
-                const int h_row = n_tile * BN + (int)rank * (n_inst >> 1);
+                const Tile tl = decode_tile(sc, t);
+                const int w_row = tl.v_tile * BV + (int)rank * BV_CTA;
+                const int h_row = tl.row0 + (int)rank * (tl.n_inst >> 1);
                 for (int kb = 0; kb < num_kb; kb++) {
                     if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) {
                         give_up();
@@ -134,7 +164,7 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
                         break;
                     }
                     const uint32_t leader_full = map_to_cta(full_bar(s), 0);
-                    if (rank == 0) mbar_expect_tx(full_bar(s), 2 * STAGE_BYTES);
+                    if (rank == 0) mbar_expect_tx(full_bar(s), stage_tx);
                     const uint32_t a_dst = base + s * STAGE_BYTES;
                     tma_load_2d_pair(a_dst, &tmap_w, kb * BK, w_row, leader_full, pol_w);
                     tma_load_2d_pair(a_dst + A_BYTES, &tmap_h, kb * BK, h_row, leader_full, pol_h);
@@ -153,7 +183,7 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
             bool ok = true;
             int it = 0;
             for (int t = pair; ok && t < num_tiles; t += num_pairs, ++it) {
-                const uint32_t idesc = instr_desc(BV, tile_rows(t % n_n));
+                const uint32_t idesc = instr_desc(BV, decode_tile(sc, t).n_inst);
                 const int ab = it & 1;
                 const uint32_t aph = (uint32_t)(it >> 1) & 1u;
                 if (!mbar_wait(acc_empty_bar(ab), aph ^ 1u, abort_flag)) {
@@ -189,8 +219,8 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
         const int q = warp & 3;  // TMEM lane quadrant this warp may read
         int it = 0;
         for (int t = pair; t < num_tiles; t += num_pairs, ++it) {
-            const int n_tile = t % n_n, v_tile = t / n_n;
-            const int n_inst = tile_rows(n_tile);
+            const Tile tl = decode_tile(sc, t);
+            const int n_inst = tl.n_inst;
             const int ab = it & 1;
             const uint32_t aph = (uint32_t)(it >> 1) & 1u;
             // the whole warp takes one decision, so the aligned TMEM loads below stay converged
@@ -199,7 +229,7 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
                 break;
             }
             tc_fence_after();
-            const int v_first = v_tile * BV + (int)rank * BV_CTA + q * 32;  // vocabulary entry of lane 0
+            const int v_first = tl.v_tile * BV + (int)rank * BV_CTA + q * 32;  // vocabulary entry of lane 0
             const bool v_ok = v_first + lane < V;                            // entries past V hold zero-filled junk
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ab * BN);
             uint32_t best_u[NCH];  // lane j, chunk c: maximum of column 32c + j over this warp's 32 entries
@@ -230,8 +260,8 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
             // merge this tile's column maxima into the rows' keys
 #pragma unroll
             for (int c = 0; c < NCH; c++) {
-                const int row = n_tile * BN + c * 32 + lane;
-                if (c * 32 < n_inst && row < M && best_u[c] != 0u) {
+                const int row = tl.row0 + c * 32 + lane;
+                if (c * 32 + lane < n_inst && row < M && best_u[c] != 0u) {
                     const unsigned long long key = ((unsigned long long)best_u[c] << 32) | (uint32_t)(~(uint32_t)best_i[c]);
                     if (key > *reinterpret_cast<volatile unsigned long long *>(&keys[row])) atomicMax(&keys[row], key);
                 }
@@ -283,10 +313,27 @@ cudaError_t umma_pair_prepare(int num_sms) {
 
 int umma_pair_max_pairs() { return g_max_pairs; }
 
+PairSched pair_schedule(int M, int V, int d) {
+    PairSched sc;
+    const int units = (M + 15) / 16;  // rows in units of 16 (the UMMA N granule)
+    sc.n_n = (units + 15) / 16;       // fewest tiles of at most 256 rows
+    sc.u_base = units / sc.n_n;
+    sc.u_rem = units % sc.n_n;
+    sc.n_v = (V + BV - 1) / BV;
+    sc.box_rows = 8 * (sc.u_base + (sc.u_rem ? 1 : 0));  // rows of h each CTA stages: half of the largest tile
+    // row tiles per group: keep a group's rows of h (tile rows x d x 2 bytes) within about 40 MB of L2
+    const long long tile_bytes = 256ll * d * 2;
+    int g_max = (int)((40ll << 20) / tile_bytes);
+    if (g_max < 1) g_max = 1;
+    sc.n_groups = (sc.n_n + g_max - 1) / g_max;
+    sc.g_base = sc.n_n / sc.n_groups;
+    sc.g_rem = sc.n_n % sc.n_groups;
+    return sc;
+}
+
 cudaError_t launch_umma_pair(const GemmArgs &a, const UmmaPlan &p, cudaStream_t stream) {
-    const int n_n = (a.M + BN - 1) / BN;
-    const int n_v = (a.V + BV - 1) / BV;
-    const int stream_w = (n_n == 1) ? 1 : 0;  // W is read by one pair only: do not keep it in L2
+    const PairSched sc = pair_schedule(a.M, a.V, a.d);
+    const int stream_w = (sc.n_n == 1) ? 1 : 0;  // W is read by one pair only: do not keep it in L2
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)p.grid);  // 2 CTAs per pair
     cfg.blockDim = dim3(NUM_THREADS);
@@ -301,8 +348,7 @@ cudaError_t launch_umma_pair(const GemmArgs &a, const UmmaPlan &p, cudaStream_t 
     attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, umma_pair_kernel, p.tmap_w, p.tmap_h, a.M, a.V, a.d, n_n, n_v, stream_w, a.keys,
-                              a.status);
+    return cudaLaunchKernelEx(&cfg, umma_pair_kernel, p.tmap_w, p.tmap_h, a.M, a.V, a.d, sc, stream_w, a.keys, a.status);
 }
 
 }  // namespace aj

@@ -68,3 +68,26 @@ def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "nope.so"))
     with pytest.raises(ImportError):
         binding.lib()
+
+
+def test_two_sm_schedule_covers_every_row_once(built):
+    """Host arithmetic of the two-SM kernel's tiling: tiles of at most 256 rows in units of 16 that
+    cover the batch exactly once with no padded tile, and groups that cover every tile once."""
+    import paper_2504_20039_b200 as aj
+
+    for M, d in [(129, 4096), (136, 4096), (256, 4096), (257, 4096), (264, 4096), (520, 4096), (2112, 4096),
+                 (2080, 8192), (8448, 4096), (16640, 4096), (16640, 8192), (4097, 64)]:
+        s = aj.pair_schedule(M, d, 128256)
+        assert s["n_v"] == 501
+        units = (M + 15) // 16
+        sizes = [s["u_base"] + (i < s["u_rem"]) for i in range(s["n_n"])]
+        assert sum(sizes) == units and max(sizes) <= 16 and min(sizes) >= 1
+        assert s["n_n"] == -(-units // 16)                    # the fewest tiles of at most 256 rows
+        assert max(sizes) - min(sizes) <= 1                   # spread evenly
+        assert s["box_rows"] == 8 * max(sizes) <= 128
+        groups = [s["g_base"] + (g < s["g_rem"]) for g in range(s["n_groups"])]
+        assert sum(groups) == s["n_n"] and min(groups) >= 1 and max(groups) - min(groups) <= 1
+        assert max(groups) * 256 * d * 2 <= 40 << 20 or max(groups) == 1
+    assert aj.pair_schedule(2112, 4096, 128256)["n_groups"] == 1
+    assert aj.pair_schedule(2080, 8192, 128256)["n_groups"] == 1
+    assert aj.pair_schedule(16640, 4096, 128256)["n_groups"] == 4

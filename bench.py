@@ -337,26 +337,13 @@ def main():
 
     import torch
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_2504_20039_b200 import dist as ajd
+
+    info = ajd.rank_info()
+    rank, world, local = info.rank, info.world, info.local_rank
     torch.cuda.set_device(local)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-
-        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
-
-    def barrier():
-        if dist is not None:
-            dist.barrier()
-
-    def reduce_max(x):
-        if dist is None:
-            return float(x)
-        t = torch.tensor([float(x)], device=f"cuda:{local}", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+    group = ajd.Group(info, backend="nccl", device=torch.device(f"cuda:{local}"))
+    barrier, reduce_max = group.barrier, group.max_over_ranks
 
     pk = peaks()
     head = workload("c2" if args.workload == "sweep" else args.workload)
@@ -365,9 +352,10 @@ def main():
     warmup = max(3, args.warmup if args.warmup is not None else 10)
     copies = args.w_copies or (3 if head.d * head.V * 2 < 1.5e9 else 2)
 
+    head = ajd.rank_config(head, rank)  # every rank verifies its own sequences
     W_host = gen.make_W(head)
     r = bench_one(head, local, steps, warmup, barrier, reduce_max, pk, copies, W_host, with_e2e=not args.no_e2e, flags=args.flags)
-    positions = head.B * head.K * world
+    positions = ajd.job_positions(head, world)
     line = {
         "metric": METRIC, "value": positions / (r["ms_per_step"] * 1e-3), "unit": UNIT, "n_gpus": world, "steps": steps,
         "warmup": warmup, "ms_per_step": r["ms_per_step"], "us_per_cycle": r["ms_per_step"] * 1e3, "higher_is_better": True,
@@ -393,6 +381,7 @@ def main():
         elif args.workload == "c2":
             todo = [gen.C3, gen.C4]
         for cfg in todo:
+            cfg = ajd.rank_config(cfg, rank)
             same_W = cfg.d == head.d and cfg.V == head.V
             n = max(20, int(0.4 / max(2.0 * cfg.M * cfg.d * cfg.V / 1.2e15, 1.7e-4)))
             rr = bench_one(cfg, local, n, 5, barrier, reduce_max, pk, 2 if not same_W else copies, W_host if same_W else None, with_e2e=False, flags=args.flags)
@@ -406,8 +395,7 @@ def main():
         line["cpu_baseline"] = base
     if rank == 0:
         print(json.dumps(line))
-    if dist is not None:
-        dist.destroy_process_group()
+    group.close()
 
 
 if __name__ == "__main__":

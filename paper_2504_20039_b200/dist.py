@@ -1,0 +1,105 @@
+"""Process-group plumbing for running the verify-and-judge step on several GPUs of one node.
+
+One process per GPU.  Sequences are independent (each is verified against the whole LM head), so the
+batch-parallel form needs no data-path collective: every rank verifies its own batch against its own
+copy of W_lm, and the process group only serves the barrier and the max-over-ranks of the timings.
+torch.distributed is used for exactly that; on a machine without GPUs the same code runs over gloo.
+"""
+from __future__ import annotations
+
+import os
+from dataclasses import dataclass, replace
+
+
+@dataclass(frozen=True)
+class RankInfo:
+    rank: int
+    world: int
+    local_rank: int
+
+
+def rank_info() -> RankInfo:
+    """Rank layout from the launcher's environment (torchrun / torch.distributed.run)."""
+    return RankInfo(int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1")),
+                    int(os.environ.get("LOCAL_RANK", "0")))
+
+
+def rank_config(cfg, rank: int):
+    """The batch rank `rank` verifies: the same shape as cfg, its own seeded sequences.
+
+    Rank 0 keeps cfg's seed, so a one-rank job is exactly the single-GPU workload."""
+    return cfg if rank == 0 else replace(cfg, seed=cfg.seed + 7919 * rank)
+
+
+def job_positions(cfg, world: int) -> int:
+    """Draft positions the whole job verifies per step: every rank's B*K."""
+    return cfg.B * cfg.K * world
+
+
+def split_sequences(total: int, world: int):
+    """Contiguous, near-equal shares of `total` sequences: [(start, count)] per rank; every sequence
+    lands on exactly one rank.  Used when a fixed global batch is divided over the ranks."""
+    base, rem = divmod(total, world)
+    out, start = [], 0
+    for r in range(world):
+        n = base + (1 if r < rem else 0)
+        out.append((start, n))
+        start += n
+    return out
+
+
+class Group:
+    """A thin wrapper over torch.distributed that degrades to a no-op for a single process."""
+
+    def __init__(self, info: RankInfo | None = None, backend: str | None = None, device=None):
+        self.info = info or rank_info()
+        self.device = device
+        self.dist = None
+        self.backend = backend
+        if self.info.world > 1:
+            import torch
+            import torch.distributed as dist
+
+            if backend is None:
+                backend = "nccl" if torch.cuda.is_available() else "gloo"
+            kw = {}
+            if backend == "nccl" and device is not None:
+                kw["device_id"] = device
+            if not dist.is_initialized():
+                dist.init_process_group(backend, rank=self.info.rank, world_size=self.info.world, **kw)
+            self.dist = dist
+            self.backend = backend
+
+    def _reduce(self, x: float, op_name: str) -> float:
+        if self.dist is None:
+            return float(x)
+        import torch
+
+        dev = self.device if (self.backend == "nccl" and self.device is not None) else "cpu"
+        t = torch.tensor([float(x)], dtype=torch.float64, device=dev)
+        self.dist.all_reduce(t, op=getattr(self.dist.ReduceOp, op_name))
+        return float(t.item())
+
+    def barrier(self) -> None:
+        if self.dist is not None:
+            self.dist.barrier()
+
+    def max_over_ranks(self, x: float) -> float:
+        """The slowest rank's value: multi-GPU timings are reported as the max over ranks."""
+        return self._reduce(x, "MAX")
+
+    def sum_over_ranks(self, x: float) -> float:
+        return self._reduce(x, "SUM")
+
+    def all_gather_bytes(self, payload: bytes):
+        """Every rank's `payload`, in rank order (used to exchange IPC handles of exchange buffers)."""
+        if self.dist is None:
+            return [bytes(payload)]
+        out = [None] * self.info.world
+        self.dist.all_gather_object(out, bytes(payload))
+        return out
+
+    def close(self) -> None:
+        if self.dist is not None and self.dist.is_initialized():
+            self.dist.destroy_process_group()
+            self.dist = None

@@ -1,0 +1,69 @@
+"""The multi-process plumbing (one process per GPU) over gloo on CPU, world size 2: rank layout,
+per-rank batches, max-over-ranks timing, whole-job throughput arithmetic, handle exchange."""
+import os
+import socket
+
+import pytest
+
+import aj_inputs as gen
+from paper_2504_20039_b200 import dist as ajd
+
+
+def _free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def _worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world), LOCAL_RANK=str(rank))
+    g = ajd.Group(backend="gloo")
+    try:
+        assert g.info == ajd.RankInfo(rank, world, rank)
+        cfg = ajd.rank_config(gen.scaled(gen.C1, B=3), rank)
+        ht, _ = gen.make_hidden(cfg)
+        g.barrier()
+        slowest = g.max_over_ranks(10.0 + rank)          # rank r "took" 10 + r ms
+        total = g.sum_over_ranks(float(cfg.B * cfg.K))    # positions verified by the whole job
+        handles = g.all_gather_bytes(bytes([rank]) * 64)  # stand-ins for 64-byte IPC handles
+        out.put((rank, cfg.seed, float(ht.astype("float64").sum()), slowest, total, [h[0] for h in handles], len(handles[0])))
+    finally:
+        g.close()
+
+
+def test_two_ranks_over_gloo():
+    import torch.multiprocessing as mp
+
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_worker, args=(r, 2, port, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    res = sorted(out.get(timeout=120) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    (r0, seed0, sum0, slow0, tot0, hs0, n0), (r1, seed1, sum1, slow1, tot1, hs1, n1) = res
+    assert (r0, r1) == (0, 1)
+    assert seed0 == gen.C1.seed and seed1 != seed0 and sum0 != sum1      # each rank verifies its own sequences
+    assert slow0 == slow1 == 11.0                                          # every rank reports the slowest rank's time
+    assert tot0 == tot1 == ajd.job_positions(gen.scaled(gen.C1, B=3), 2)   # value = all ranks' positions / that time
+    assert hs0 == hs1 == [0, 1] and n0 == n1 == 64                         # handles arrive in rank order on every rank
+
+
+def test_single_process_group_is_a_no_op():
+    g = ajd.Group(ajd.RankInfo(0, 1, 0))
+    g.barrier()
+    assert g.max_over_ranks(3.5) == 3.5 and g.sum_over_ranks(2.0) == 2.0
+    assert g.all_gather_bytes(b"ab") == [b"ab"]
+    g.close()
+
+
+@pytest.mark.parametrize("total,world", [(64, 8), (7, 2), (3, 4), (256, 3)])
+def test_split_sequences_covers_every_sequence_once(total, world):
+    parts = ajd.split_sequences(total, world)
+    assert len(parts) == world and parts[0][0] == 0
+    assert sum(n for _, n in parts) == total
+    assert all(parts[i][0] + parts[i][1] == parts[i + 1][0] for i in range(world - 1))
+    assert max(n for _, n in parts) - min(n for _, n in parts) <= 1

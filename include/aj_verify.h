@@ -27,6 +27,7 @@
 #ifndef AJ_VERIFY_H
 #define AJ_VERIFY_H
 
+#include <stddef.h>
 #include <stdint.h>
 
 #ifdef __cplusplus
@@ -182,6 +183,65 @@ aj_status aj_verify_static(const void *h_target, const void *h_draft, const void
                            int B, int K, int d, int d_draft, int V, aj_dtype dtype, aj_w_layout layout,
                            int32_t *accept_len, int32_t *next_tok, int32_t *target_tok,
                            float *top1_val, float *judge_p, int32_t *dev_status, void *cuda_stream);
+
+/*
+ * ---------------------------------------------------------------------------------------------
+ * Vocabulary-parallel form: the LM head split by vocabulary entries over up to 8 GPUs of one node,
+ * the layout of the paper's tensor-parallel deployments (Section 4.3: the 70B target on 4 GPUs, the
+ * 405B target on 8).  GPU r holds rows [v_begin, v_begin + v_count) of W_lm, projects the same
+ * h_target against them, and the per-row (max, argmax) keys of all GPUs are merged by one 64-bit
+ * max.  The projection kernel performs the exchange itself: its last CTA stores this GPU's keys into
+ * a slot of EVERY GPU's exchange buffer (peer stores over NVLink) and then the cycle number into a
+ * flag there; each GPU's judge kernel waits (at most 2 s, then AJ_ERR_TIMEOUT in aj_last_status)
+ * for all flags of its own buffer and reduces the slots.  Every GPU computes the same accept_len and
+ * next_tok.  One process per GPU; all ranks make the same sequence of calls with the same B and K.
+ *
+ * Exchange buffers are caller-owned device memory of aj_shard_exchange_bytes() bytes, 256-byte
+ * aligned, one per GPU, each mapped into every process (aj_ipc_export / aj_ipc_import, or any other
+ * peer mapping).  exchange[g] is rank g's buffer as addressable from THIS device; exchange[rank] is
+ * this GPU's own.  aj_create_sharded zeroes the own buffer: put a barrier over all ranks between
+ * creating the handles and the first cycle, and between the last cycle and freeing the buffers.
+ */
+
+/* Bytes of one GPU's exchange buffer; 0 if an argument is out of range (world in 1..8). */
+size_t aj_shard_exchange_bytes(int max_B, int max_K, int world);
+
+/* The contiguous vocabulary range of rank `rank` among `world` GPUs: whole blocks of 256 entries,
+ * spread evenly.  Errors: AJ_ERR_INVALID_ARG (also when V has fewer than `world` blocks). */
+aj_status aj_shard_range(int V, int world, int rank, int *v_begin, int *v_count);
+
+/*
+ * aj_create for one GPU of a vocabulary-parallel group.  V is the WHOLE vocabulary (token ids in
+ * the outputs are global); this GPU's W_lm argument in later calls is its shard, v_count rows
+ * (layout AJ_W_VD: [v_count, d]; AJ_W_DV: [d, v_count]).  AJ_FLAG_ROW_TILES is not available here.
+ * Errors: as aj_create, and AJ_ERR_INVALID_ARG for a bad rank, range or buffer.
+ */
+aj_status aj_create_sharded(aj_handle *out, int device, int max_B, int max_K, int d, int d_draft, int V,
+                            aj_dtype dtype, aj_w_layout layout, unsigned flags,
+                            int rank, int world, int v_begin, int v_count, void *const *exchange);
+
+/*
+ * On a sharded handle aj_verify and aj_verify_host run a whole cycle (W_lm = this GPU's shard).
+ * The two halves can also be enqueued separately: aj_shard_project enqueues the projection of the
+ * shard and the exchange; aj_shard_finish enqueues the wait for all GPUs' keys, the judge and the
+ * prefix scan.  Arguments as in aj_verify.  Every aj_shard_project must be followed by its
+ * aj_shard_finish before the next cycle.  Errors: as aj_verify.
+ */
+aj_status aj_shard_project(aj_handle h, const void *h_target, const void *W_shard, int B, int K, void *cuda_stream);
+aj_status aj_shard_finish(aj_handle h, const void *h_target, const void *h_draft, const int32_t *draft_tok,
+                          const float *judge_w, float judge_b, float tau, int B, int K,
+                          int32_t *accept_len, int32_t *next_tok, int32_t *target_tok,
+                          float *top1_val, float *judge_p, void *cuda_stream);
+
+/*
+ * Sharing an exchange buffer between the processes of one node (thin wrappers over CUDA IPC, so that
+ * a caller needs no CUDA binding of its own): export gives 64 opaque bytes for a cudaMalloc'ed
+ * device pointer; import, in another process with its own device current, maps that memory and
+ * enables peer access; close unmaps it.  Errors: AJ_ERR_INVALID_ARG, AJ_ERR_CUDA.
+ */
+aj_status aj_ipc_export(const void *device_ptr, unsigned char handle_out[64]);
+aj_status aj_ipc_import(const unsigned char handle_in[64], void **device_ptr_out);
+aj_status aj_ipc_close(void *device_ptr);
 
 /* Free the handle and its workspace.  The caller must have synchronised all work using it. */
 aj_status aj_destroy(aj_handle h);

@@ -19,7 +19,8 @@ AJ_FLAG_FORCE_SIMT, AJ_FLAG_TIME_KERNELS, AJ_FLAG_ROW_TILES, AJ_FLAG_ONE_SM = 1,
 
 EXPORTS = (
     "aj_create", "aj_verify", "aj_verify_host", "aj_last_status", "aj_last_gemm_ms", "aj_gemm_ms_stats", "aj_last_launch_count",
-    "aj_last_gemm_path", "aj_pair_schedule", "aj_destroy", "aj_status_string", "aj_version", "aj_verify_static",
+    "aj_last_gemm_path", "aj_pair_schedule", "aj_destroy", "aj_shard_exchange_bytes", "aj_shard_range", "aj_create_sharded",
+    "aj_shard_project", "aj_shard_finish", "aj_ipc_export", "aj_ipc_import", "aj_ipc_close", "aj_status_string", "aj_version", "aj_verify_static",
 )
 
 _lib = None
@@ -66,6 +67,22 @@ def lib() -> ctypes.CDLL:
         L.aj_verify_static.restype = ci
         L.aj_pair_schedule.argtypes = [ci, ci, ci, ctypes.POINTER(ctypes.c_int32)]
         L.aj_pair_schedule.restype = ci
+        L.aj_shard_exchange_bytes.argtypes = [ci, ci, ci]
+        L.aj_shard_exchange_bytes.restype = ctypes.c_size_t
+        L.aj_shard_range.argtypes = [ci, ci, ci, ctypes.POINTER(ci), ctypes.POINTER(ci)]
+        L.aj_shard_range.restype = ci
+        L.aj_create_sharded.argtypes = [ctypes.POINTER(vp), ci, ci, ci, ci, ci, ci, ci, ci, cu, ci, ci, ci, ci, ctypes.POINTER(vp)]
+        L.aj_create_sharded.restype = ci
+        L.aj_shard_project.argtypes = [vp, vp, vp, ci, ci, vp]
+        L.aj_shard_project.restype = ci
+        L.aj_shard_finish.argtypes = [vp, vp, vp, vp, vp, cf, cf, ci, ci, vp, vp, vp, vp, vp, vp]
+        L.aj_shard_finish.restype = ci
+        L.aj_ipc_export.argtypes = [vp, ctypes.c_char_p]
+        L.aj_ipc_export.restype = ci
+        L.aj_ipc_import.argtypes = [ctypes.c_char_p, ctypes.POINTER(vp)]
+        L.aj_ipc_import.restype = ci
+        L.aj_ipc_close.argtypes = [vp]
+        L.aj_ipc_close.restype = ci
         L.aj_version.argtypes = []
         L.aj_version.restype = ctypes.c_char_p
         _lib = L
@@ -121,17 +138,82 @@ def verify_static(h_target, h_draft, W_lm, draft_tok, judge_w, judge_b: float, t
     return st
 
 
+def shard_exchange_bytes(max_B: int, max_K: int, world: int) -> int:
+    """aj_shard_exchange_bytes: size of one GPU's exchange buffer for a vocabulary-parallel group."""
+    return int(lib().aj_shard_exchange_bytes(max_B, max_K, world))
+
+
+def shard_range(V: int, world: int, rank: int):
+    """aj_shard_range: (v_begin, v_count) of rank `rank` among `world` GPUs."""
+    b, n = ctypes.c_int(), ctypes.c_int()
+    st = lib().aj_shard_range(V, world, rank, ctypes.byref(b), ctypes.byref(n))
+    if st != AJ_OK:
+        raise AjError(st, "aj_shard_range")
+    return int(b.value), int(n.value)
+
+
+def ipc_export(device_ptr) -> bytes:
+    """aj_ipc_export: 64 opaque bytes another process of this node can import."""
+    buf = ctypes.create_string_buffer(64)
+    st = lib().aj_ipc_export(_ptr(device_ptr), buf)
+    if st != AJ_OK:
+        raise AjError(st, "aj_ipc_export")
+    return buf.raw
+
+
+def ipc_import(handle: bytes) -> int:
+    """aj_ipc_import: the device address at which this process sees the exported memory."""
+    out = ctypes.c_void_p()
+    st = lib().aj_ipc_import(ctypes.create_string_buffer(bytes(handle), 64), ctypes.byref(out))
+    if st != AJ_OK:
+        raise AjError(st, "aj_ipc_import")
+    return int(out.value)
+
+
+def ipc_close(device_ptr: int) -> None:
+    st = lib().aj_ipc_close(device_ptr)
+    if st != AJ_OK:
+        raise AjError(st, "aj_ipc_close")
+
+
 class Handle:
-    """aj_create / aj_destroy as an object; methods mirror the C entry points."""
+    """aj_create / aj_destroy as an object; methods mirror the C entry points.
+
+    With `shard=(rank, world, v_begin, v_count, exchange)` the handle is one GPU of a vocabulary-parallel
+    group (aj_create_sharded); `exchange` lists every rank's exchange buffer (tensors or addresses)."""
 
     def __init__(self, device: int, max_B: int, max_K: int, d: int, d_draft: int, V: int,
-                 dtype: int = AJ_BF16, layout: int = AJ_W_VD, flags: int = 0):
+                 dtype: int = AJ_BF16, layout: int = AJ_W_VD, flags: int = 0, shard=None):
         self._h = ctypes.c_void_p()
-        st = lib().aj_create(ctypes.byref(self._h), device, max_B, max_K, d, d_draft, V, dtype, layout, flags)
+        if shard is None:
+            st = lib().aj_create(ctypes.byref(self._h), device, max_B, max_K, d, d_draft, V, dtype, layout, flags)
+        else:
+            rank, world, v_begin, v_count, exchange = shard
+            ptrs = (ctypes.c_void_p * len(exchange))(*[_ptr(e) for e in exchange])
+            st = lib().aj_create_sharded(ctypes.byref(self._h), device, max_B, max_K, d, d_draft, V, dtype, layout, flags,
+                                         rank, world, v_begin, v_count, ptrs)
         if st != AJ_OK:
             self._h = ctypes.c_void_p()
-            raise AjError(st, "aj_create")
+            raise AjError(st, "aj_create" if shard is None else "aj_create_sharded")
         self.d, self.V, self.d_draft = d, V, d_draft
+
+    def shard_project(self, h_target, W_shard, B: int, K: int, stream: int = 0, check: bool = True) -> int:
+        """aj_shard_project: this GPU's projection + exchange of one cycle."""
+        st = lib().aj_shard_project(self._h, _ptr(h_target), _ptr(W_shard), B, K, stream or None)
+        if check and st != AJ_OK:
+            raise AjError(st, "aj_shard_project")
+        return st
+
+    def shard_finish(self, h_target, h_draft, draft_tok, judge_w, judge_b: float, tau: float, B: int, K: int,
+                     accept_len, next_tok, target_tok=None, top1_val=None, judge_p=None, stream: int = 0,
+                     check: bool = True) -> int:
+        """aj_shard_finish: wait for every GPU's keys, then judge + prefix scan."""
+        st = lib().aj_shard_finish(self._h, _ptr(h_target), _ptr(h_draft), _ptr(draft_tok), _ptr(judge_w), float(judge_b),
+                                   float(tau), B, K, _ptr(accept_len), _ptr(next_tok), _ptr(target_tok), _ptr(top1_val),
+                                   _ptr(judge_p), stream or None)
+        if check and st != AJ_OK:
+            raise AjError(st, "aj_shard_finish")
+        return st
 
     def verify(self, h_target, h_draft, W_lm, draft_tok, judge_w, judge_b: float, tau: float, B: int, K: int,
                accept_len, next_tok, target_tok=None, top1_val=None, judge_p=None, stream: int = 0, check: bool = True) -> int:

@@ -50,7 +50,17 @@ struct aj_handle_s {
     long long n_timed = 0;                                   // calls recorded since the last read-out
     int last_launches = 0;
     const char *last_path = "none";
+    // vocabulary-parallel handles (aj_create_sharded)
+    int world = 0, rank = 0;         // world == 0: the handle holds the whole LM head
+    int v_begin = 0, v_count = 0;    // this GPU's vocabulary entries
+    unsigned long long *exchange[MAX_SHARD_WORLD] = {};  // every GPU's exchange buffer, as mapped on this device
+    unsigned long long epoch = 0;    // cycles started; the same on every rank, which call in step
+    bool projected = false;          // aj_shard_project was enqueued and its aj_shard_finish is still due
 };
+
+// Exchange buffer of one GPU: 256 bytes of flags (one 8-byte epoch per source GPU), then two slot
+// arrays (one per epoch parity) of world x max_M keys.
+constexpr size_t EXCHANGE_FLAG_BYTES = 256;
 
 namespace {
 
@@ -227,17 +237,11 @@ aj_status aj_destroy(aj_handle h) {
     return AJ_OK;
 }
 
-aj_status aj_verify(aj_handle h, const void *h_target, const void *h_draft, const void *W_lm, const int32_t *draft_tok,
-                    const float *judge_w, float judge_b, float tau, int B, int K, int d, int V, int32_t *accept_len,
-                    int32_t *next_tok, int32_t *target_tok, float *top1_val, float *judge_p, void *cuda_stream) {
-    aj_status st = check_call(h, h_target, h_draft, W_lm, draft_tok, judge_w, B, K, d, V, accept_len, next_tok);
-    if (st != AJ_OK) return st;
-    if (h->dtype == AJ_BF16 && (!aligned16(h_target) || !aligned16(W_lm) || (h_draft && !aligned16(h_draft))))
-        return AJ_ERR_UNSUPPORTED;
-    DeviceGuard guard(h->device);
-    if (!guard.ok()) return AJ_ERR_CUDA;
-    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+// Enqueue the projection + argmax kernel of one cycle (and, on a sharded handle, its exchange).
+static aj_status enqueue_project(aj_handle h, const void *h_target, const void *W_lm, int B, int K, cudaStream_t stream) {
     const int M = B * (K + 1);
+    const int d = h->d;
+    const int V = h->world ? h->v_count : h->V;  // vocabulary entries this GPU projects
     h->last_launches = 0;
 
     if (h->keys_dirty) {
@@ -252,10 +256,24 @@ aj_status aj_verify(aj_handle h, const void *h_target, const void *h_draft, cons
     g.M = M;
     g.d = d;
     g.V = V;
+    g.v_offset = h->world ? h->v_begin : 0;
     g.dtype = h->dtype;
     g.w_layout = h->layout;
     g.keys = h->keys;
     g.status = h->status;
+    if (h->world) {
+        ++h->epoch;
+        const size_t max_M = (size_t)h->max_B * (h->max_K + 1);
+        g.pub.world = h->world;
+        g.pub.M = M;
+        g.pub.epoch = h->epoch;
+        g.pub.done = reinterpret_cast<unsigned *>(h->status) + 16;
+        for (int r = 0; r < h->world; r++) {
+            unsigned long long *buf = h->exchange[r];
+            g.pub.flag[r] = buf + h->rank;
+            g.pub.slot[r] = buf + EXCHANGE_FLAG_BYTES / 8 + ((h->epoch & 1) * h->world + h->rank) * max_M;
+        }
+    }
 
     const bool time_it = (h->flags & AJ_FLAG_TIME_KERNELS) != 0;
     const int slot = (int)(h->n_timed % EVENT_RING);
@@ -312,8 +330,26 @@ aj_status aj_verify(aj_handle h, const void *h_target, const void *h_draft, cons
         h->n_timed++;
     }
 
+    return AJ_OK;
+}
+
+// Enqueue the judge + prefix-scan kernel of the cycle whose projection was enqueued last.
+static aj_status enqueue_finish(aj_handle h, const void *h_target, const void *h_draft, const int32_t *draft_tok,
+                                const float *judge_w, float judge_b, float tau, int B, int K, int32_t *accept_len,
+                                int32_t *next_tok, int32_t *target_tok, float *top1_val, float *judge_p,
+                                cudaStream_t stream) {
     JudgeArgs j;
     j.keys = h->keys;
+    j.status = h->status;
+    if (h->world) {
+        const size_t max_M = (size_t)h->max_B * (h->max_K + 1);
+        const unsigned long long *own = h->exchange[h->rank];
+        j.gather.world = h->world;
+        j.gather.stride = (int)max_M;
+        j.gather.epoch = h->epoch;
+        j.gather.flags = own;
+        j.gather.slots = own + EXCHANGE_FLAG_BYTES / 8 + (h->epoch & 1) * h->world * max_M;
+    }
     j.h_target = h_target;
     j.h_draft = h_draft;
     j.draft_tok = draft_tok;
@@ -322,7 +358,7 @@ aj_status aj_verify(aj_handle h, const void *h_target, const void *h_draft, cons
     j.tau = tau;
     j.B = B;
     j.K = K;
-    j.d = d;
+    j.d = h->d;
     j.d_draft = h->d_draft;
     j.dtype = h->dtype;
     j.accept_len = accept_len;
@@ -334,6 +370,23 @@ aj_status aj_verify(aj_handle h, const void *h_target, const void *h_draft, cons
     h->keys_dirty = false;
     h->last_launches++;
     return AJ_OK;
+}
+
+aj_status aj_verify(aj_handle h, const void *h_target, const void *h_draft, const void *W_lm, const int32_t *draft_tok,
+                    const float *judge_w, float judge_b, float tau, int B, int K, int d, int V, int32_t *accept_len,
+                    int32_t *next_tok, int32_t *target_tok, float *top1_val, float *judge_p, void *cuda_stream) {
+    aj_status st = check_call(h, h_target, h_draft, W_lm, draft_tok, judge_w, B, K, d, V, accept_len, next_tok);
+    if (st != AJ_OK) return st;
+    if (h->dtype == AJ_BF16 && (!aligned16(h_target) || !aligned16(W_lm) || (h_draft && !aligned16(h_draft))))
+        return AJ_ERR_UNSUPPORTED;
+    if (h->projected) return AJ_ERR_INVALID_ARG;  // an aj_shard_project is waiting for its aj_shard_finish
+    DeviceGuard guard(h->device);
+    if (!guard.ok()) return AJ_ERR_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    st = enqueue_project(h, h_target, W_lm, B, K, stream);
+    if (st != AJ_OK) return st;
+    return enqueue_finish(h, h_target, h_draft, draft_tok, judge_w, judge_b, tau, B, K, accept_len, next_tok, target_tok,
+                          top1_val, judge_p, stream);
 }
 
 aj_status aj_verify_host(aj_handle h, const void *h_target_host, const void *h_draft_host, const void *W_lm,
@@ -405,6 +458,117 @@ aj_status aj_gemm_ms_stats(aj_handle h, float *mean_ms, float *min_ms, int *coun
     if (min_ms) *min_ms = lo;
     *count = (int)n;
     h->n_timed = 0;
+    return AJ_OK;
+}
+
+size_t aj_shard_exchange_bytes(int max_B, int max_K, int world) {
+    if (max_B < 1 || max_K < 1 || world < 1 || world > MAX_SHARD_WORLD) return 0;
+    return EXCHANGE_FLAG_BYTES + 2 * (size_t)world * ((size_t)max_B * (max_K + 1)) * sizeof(unsigned long long);
+}
+
+aj_status aj_shard_range(int V, int world, int rank, int *v_begin, int *v_count) {
+    if (!v_begin || !v_count || V < 1 || world < 1 || world > MAX_SHARD_WORLD || rank < 0 || rank >= world)
+        return AJ_ERR_INVALID_ARG;
+    const int blocks = (V + 255) / 256;  // whole blocks of 256 entries, so that shards start on a tile boundary
+    if (blocks < world) return AJ_ERR_INVALID_ARG;  // some GPU would get nothing
+    const int base = blocks / world, rem = blocks % world;
+    const long long b0 = (long long)rank * base + (rank < rem ? rank : rem);
+    const long long b1 = b0 + base + (rank < rem ? 1 : 0);
+    const long long lo = b0 * 256 < V ? b0 * 256 : V, hi = b1 * 256 < V ? b1 * 256 : V;
+    *v_begin = (int)lo;
+    *v_count = (int)(hi - lo);
+    return AJ_OK;
+}
+
+aj_status aj_create_sharded(aj_handle *out, int device, int max_B, int max_K, int d, int d_draft, int V, aj_dtype dtype,
+                            aj_w_layout layout, unsigned flags, int rank, int world, int v_begin, int v_count,
+                            void *const *exchange) {
+    if (!out) return AJ_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!exchange || world < 1 || world > MAX_SHARD_WORLD || rank < 0 || rank >= world) return AJ_ERR_INVALID_ARG;
+    if (v_begin < 0 || v_count < 1 || (long long)v_begin + v_count > V) return AJ_ERR_INVALID_ARG;
+    for (int r = 0; r < world; r++)
+        if (!exchange[r] || (reinterpret_cast<uintptr_t>(exchange[r]) & 255)) return AJ_ERR_INVALID_ARG;
+    if (flags & AJ_FLAG_ROW_TILES) return AJ_ERR_UNSUPPORTED;
+    aj_handle h = nullptr;
+    aj_status st = aj_create(&h, device, max_B, max_K, d, d_draft, V, dtype, layout, flags);
+    if (st != AJ_OK) return st;
+    h->world = world;
+    h->rank = rank;
+    h->v_begin = v_begin;
+    h->v_count = v_count;
+    for (int r = 0; r < world; r++) h->exchange[r] = static_cast<unsigned long long *>(exchange[r]);
+    // this GPU's own buffer starts from zero flags; peers must not publish before every rank has
+    // created its handle (the caller puts a barrier between creation and the first cycle)
+    DeviceGuard guard(device);
+    if (!guard.ok() || cudaMemset(exchange[rank], 0, aj_shard_exchange_bytes(max_B, max_K, world)) != cudaSuccess ||
+        cudaDeviceSynchronize() != cudaSuccess) {
+        cudaGetLastError();
+        aj_destroy(h);
+        return AJ_ERR_CUDA;
+    }
+    *out = h;
+    return AJ_OK;
+}
+
+aj_status aj_shard_project(aj_handle h, const void *h_target, const void *W_shard, int B, int K, void *cuda_stream) {
+    if (!h || !h->world || !h_target || !W_shard || B < 1 || K < 1) return AJ_ERR_INVALID_ARG;
+    if (B > h->max_B || K > h->max_K) return AJ_ERR_WORKSPACE;
+    if (h->projected) return AJ_ERR_INVALID_ARG;
+    if (h->dtype == AJ_BF16 && (!aligned16(h_target) || !aligned16(W_shard))) return AJ_ERR_UNSUPPORTED;
+    DeviceGuard guard(h->device);
+    if (!guard.ok()) return AJ_ERR_CUDA;
+    aj_status st = enqueue_project(h, h_target, W_shard, B, K, static_cast<cudaStream_t>(cuda_stream));
+    if (st == AJ_OK) h->projected = true;
+    return st;
+}
+
+aj_status aj_shard_finish(aj_handle h, const void *h_target, const void *h_draft, const int32_t *draft_tok,
+                          const float *judge_w, float judge_b, float tau, int B, int K, int32_t *accept_len,
+                          int32_t *next_tok, int32_t *target_tok, float *top1_val, float *judge_p, void *cuda_stream) {
+    if (!h || !h->world || !h->projected) return AJ_ERR_INVALID_ARG;
+    if (!h_target || !draft_tok || !judge_w || !accept_len || !next_tok) return AJ_ERR_INVALID_ARG;
+    if ((h->d_draft > 0) != (h_draft != nullptr) || B < 1 || K < 1) return AJ_ERR_INVALID_ARG;
+    if (B > h->max_B || K > h->max_K) return AJ_ERR_WORKSPACE;
+    if (h->dtype == AJ_BF16 && (!aligned16(h_target) || (h_draft && !aligned16(h_draft)))) return AJ_ERR_UNSUPPORTED;
+    DeviceGuard guard(h->device);
+    if (!guard.ok()) return AJ_ERR_CUDA;
+    aj_status st = enqueue_finish(h, h_target, h_draft, draft_tok, judge_w, judge_b, tau, B, K, accept_len, next_tok,
+                                  target_tok, top1_val, judge_p, static_cast<cudaStream_t>(cuda_stream));
+    if (st == AJ_OK) h->projected = false;
+    return st;
+}
+
+aj_status aj_ipc_export(const void *device_ptr, unsigned char handle_out[64]) {
+    if (!device_ptr || !handle_out) return AJ_ERR_INVALID_ARG;
+    static_assert(sizeof(cudaIpcMemHandle_t) == 64, "IPC handle size");
+    cudaIpcMemHandle_t hd;
+    if (cudaIpcGetMemHandle(&hd, const_cast<void *>(device_ptr)) != cudaSuccess) {
+        cudaGetLastError();
+        return AJ_ERR_CUDA;
+    }
+    memcpy(handle_out, &hd, 64);
+    return AJ_OK;
+}
+
+aj_status aj_ipc_import(const unsigned char handle_in[64], void **device_ptr_out) {
+    if (!handle_in || !device_ptr_out) return AJ_ERR_INVALID_ARG;
+    cudaIpcMemHandle_t hd;
+    memcpy(&hd, handle_in, 64);
+    if (cudaIpcOpenMemHandle(device_ptr_out, hd, cudaIpcMemLazyEnablePeerAccess) != cudaSuccess) {
+        cudaGetLastError();
+        *device_ptr_out = nullptr;
+        return AJ_ERR_CUDA;
+    }
+    return AJ_OK;
+}
+
+aj_status aj_ipc_close(void *device_ptr) {
+    if (!device_ptr) return AJ_ERR_INVALID_ARG;
+    if (cudaIpcCloseMemHandle(device_ptr) != cudaSuccess) {
+        cudaGetLastError();
+        return AJ_ERR_CUDA;
+    }
     return AJ_OK;
 }
 

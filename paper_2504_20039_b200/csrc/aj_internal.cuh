@@ -41,16 +41,73 @@ __device__ inline int key_index(unsigned long long key) { return (int)(~(uint32_
 // Device status word values (mirrors aj_status where they overlap).
 enum : int { DEV_OK = 0, DEV_TIMEOUT = 5 };
 
+// ------------------------------------------------------- vocabulary-parallel exchange of keys
+//
+// When the LM head is split by vocabulary over several GPUs, each GPU projects its own entries
+// and the per-row keys of all GPUs are merged by the same 64-bit max.  The projection kernel does
+// the exchange itself: the CTA that finishes last copies this GPU's keys into a slot of every
+// GPU's exchange buffer (plain stores, over NVLink for the peers) and then stores the cycle's
+// epoch into a flag in each of those buffers with release semantics.  The judge kernel of every
+// GPU waits (bounded) until all flags of its own buffer show the epoch and takes the max over
+// the slots.  Nothing is multicast and no kernel reads a peer's memory.
+constexpr int MAX_SHARD_WORLD = 8;
+
+struct Publish {
+    int world = 0;                 // 0: the handle is not sharded, nothing is published
+    int M = 0;
+    unsigned long long epoch = 0;  // the value stored into the flags
+    unsigned *done = nullptr;      // CTAs of this launch that have finished (wraps to zero by itself)
+    unsigned long long *slot[MAX_SHARD_WORLD] = {};  // [M] in GPU g's buffer: where it wants this GPU's keys
+    unsigned long long *flag[MAX_SHARD_WORLD] = {};  // in GPU g's buffer: where it wants this GPU's epoch
+};
+
+struct Gather {
+    int world = 0;                              // 0: read and clear the handle's own keys
+    int stride = 0;                             // rows per slot
+    unsigned long long epoch = 0;
+    const unsigned long long *slots = nullptr;  // [world][stride], in this GPU's buffer
+    const unsigned long long *flags = nullptr;  // [world], in this GPU's buffer
+};
+
+#ifdef __CUDACC__
+// Called by every thread of every CTA of a projection kernel once the CTA's own key updates have
+// been issued.  The last CTA to arrive publishes the keys and clears them for the next cycle.
+__device__ inline void publish_keys(const Publish &p, unsigned long long *keys) {
+    if (p.world == 0) return;  // the same for the whole grid
+    __shared__ int is_last;
+    __threadfence();  // this thread's key updates are performed before its CTA is counted
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const unsigned total = gridDim.x * gridDim.y * gridDim.z;
+        is_last = atomicInc(p.done, total - 1) == total - 1;
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    for (int j = threadIdx.x; j < p.M; j += blockDim.x) {
+        const unsigned long long k = __ldcg(keys + j);
+        keys[j] = 0ull;  // every CTA is done with them: leave the workspace clean
+        for (int g = 0; g < p.world; g++) p.slot[g][j] = k;
+    }
+    __threadfence_system();
+    __syncthreads();
+    if ((int)threadIdx.x < p.world)
+        asm volatile("st.release.sys.global.u64 [%0], %1;" ::"l"(p.flag[threadIdx.x]), "l"(p.epoch) : "memory");
+}
+#endif
+
 // ------------------------------------------------------------------------------ launchers
 
 struct GemmArgs {
     const void *h;       // [M, d]
-    const void *W;       // [V, d] or [d, V]
+    const void *W;       // [V, d] or [d, V]; V entries starting at vocabulary index v_offset
     int M, d, V;
+    int v_offset = 0;    // added to every index stored in a key (vocabulary-parallel shards)
     int dtype;           // 0 bf16, 1 f32
     int w_layout;        // 0 [V,d], 1 [d,V]
     unsigned long long *keys;  // [M], must be zero on entry (the judge kernel clears what it reads)
     int *status;
+    Publish pub;
 };
 
 // CUDA-core projection + argmax (any dtype / layout).
@@ -91,7 +148,9 @@ int umma_pair_max_pairs();
 cudaError_t launch_umma_pair(const GemmArgs &a, const UmmaPlan &p, cudaStream_t stream);
 
 struct JudgeArgs {
-    unsigned long long *keys;        // [B*(K+1)]; read, then cleared for the next cycle
+    unsigned long long *keys;        // [B*(K+1)]; read, then cleared for the next cycle (unless gathered)
+    Gather gather;                   // vocabulary-parallel: where the merged keys come from
+    int *status = nullptr;           // device status word (set when a bounded wait runs out)
     const void *h_target;            // [B, K+1, d]
     const void *h_draft;             // [B, K+1, d_draft] or nullptr
     const int32_t *draft_tok;        // [B, K]

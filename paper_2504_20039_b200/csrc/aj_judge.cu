@@ -136,10 +136,43 @@ __global__ void __maxnreg__(96) judge_scan_kernel(JudgeArgs a) {
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
     // ---- the projection kernel has finished and its keys are visible
+    if (a.gather.world > 0) {
+        // Vocabulary-parallel: every GPU's projection kernel stores its keys into a slot of this
+        // GPU's exchange buffer and then the cycle's epoch into a flag.  Wait for all flags.
+        if ((int)threadIdx.x < a.gather.world) {
+            const unsigned long long *f = a.gather.flags + threadIdx.x;
+            unsigned long long seen, t0 = 0;
+            for (unsigned spin = 0;; ++spin) {
+                asm volatile("ld.acquire.sys.global.u64 %0, [%1];" : "=l"(seen) : "l"(f) : "memory");
+                if (seen >= a.gather.epoch) break;
+                if ((spin & 0x3F) == 0x3F) {
+                    unsigned long long now;
+                    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+                    if (t0 == 0) {
+                        t0 = now;
+                    } else if (now - t0 > 2000000000ull) {  // 2 s: a peer never published
+                        atomicCAS(a.status, DEV_OK, DEV_TIMEOUT);
+                        break;
+                    }
+                    __nanosleep(200);
+                }
+            }
+        }
+        __syncthreads();
+    }
     for (int j = threadIdx.x; j < R; j += blockDim.x) {
-        unsigned long long *kp = a.keys + (size_t)b * R + j;
-        const unsigned long long key = *kp;
-        *kp = 0ull;  // leave the workspace clean for the next cycle
+        unsigned long long key;
+        if (a.gather.world > 0) {
+            key = 0ull;
+            for (int g = 0; g < a.gather.world; g++) {
+                const unsigned long long k = __ldcg(a.gather.slots + (size_t)g * a.gather.stride + (size_t)b * R + j);
+                key = k > key ? k : key;  // the same merge the projection kernel's atomic max performs
+            }
+        } else {
+            unsigned long long *kp = a.keys + (size_t)b * R + j;
+            key = *kp;
+            *kp = 0ull;  // leave the workspace clean for the next cycle
+        }
         const int y = key_index(key);
         y_s[j] = y;
         if (a.target_tok) a.target_tok[(size_t)b * R + j] = y;

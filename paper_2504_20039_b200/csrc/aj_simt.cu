@@ -18,19 +18,18 @@ __device__ inline float load_as_float(const __nv_bfloat16 *p, size_t i) { return
 
 template <typename T>
 __global__ void __launch_bounds__(256) simt_gemm_argmax_kernel(const T *__restrict__ h, const T *__restrict__ W,
-                                                               int M, int d, int V, int w_layout,
-                                                               unsigned long long *__restrict__ keys) {
+                                                               int M, int d, int V, int w_layout, int v_offset,
+                                                               unsigned long long *__restrict__ keys, const Publish pub) {
     const int lane = threadIdx.x & 31;
     const int warps_per_block = blockDim.x >> 5;
     const long long warp = (long long)blockIdx.x * warps_per_block + (threadIdx.x >> 5);
     const long long warps_total = (long long)gridDim.x * warps_per_block;
     const int per = (int)((V + warps_total - 1) / warps_total);
     const long long v0l = warp * per;
-    if (v0l >= V) return;
-    const int v0 = (int)v0l;
+    const int v0 = (int)(v0l < V ? v0l : V);  // a warp past the end has an empty slice
     const int v1 = min(V, v0 + per);
 
-    for (int m0 = 0; m0 < M; m0 += ROWS) {
+    for (int m0 = 0; m0 < M && v0 < v1; m0 += ROWS) {
         float best[ROWS];
         int bidx[ROWS];
 #pragma unroll
@@ -65,9 +64,10 @@ __global__ void __launch_bounds__(256) simt_gemm_argmax_kernel(const T *__restri
         if (lane == 0) {
 #pragma unroll
             for (int r = 0; r < ROWS; r++)
-                if (m0 + r < M) atomicMax(&keys[m0 + r], pack_key(best[r], bidx[r]));
+                if (m0 + r < M) atomicMax(&keys[m0 + r], pack_key(best[r], bidx[r] + v_offset));
         }
     }
+    publish_keys(pub, keys);
 }
 
 }  // namespace
@@ -82,10 +82,10 @@ cudaError_t launch_simt_gemm_argmax(const GemmArgs &a, int num_sms, cudaStream_t
     if (blocks < 1) blocks = 1;
     if (a.dtype == 0)
         simt_gemm_argmax_kernel<__nv_bfloat16><<<(unsigned)blocks, threads, 0, stream>>>(
-            (const __nv_bfloat16 *)a.h, (const __nv_bfloat16 *)a.W, a.M, a.d, a.V, a.w_layout, a.keys);
+            (const __nv_bfloat16 *)a.h, (const __nv_bfloat16 *)a.W, a.M, a.d, a.V, a.w_layout, a.v_offset, a.keys, a.pub);
     else
         simt_gemm_argmax_kernel<float><<<(unsigned)blocks, threads, 0, stream>>>(
-            (const float *)a.h, (const float *)a.W, a.M, a.d, a.V, a.w_layout, a.keys);
+            (const float *)a.h, (const float *)a.W, a.M, a.d, a.V, a.w_layout, a.v_offset, a.keys, a.pub);
     return cudaGetLastError();
 }
 

@@ -152,6 +152,7 @@ extern "C" aj_status aj_verify_static(const void *h_target, const void *h_draft,
 
     JudgeArgs j;
     j.keys = keys;
+    j.status = status;
     j.h_target = h_target;
     j.h_draft = h_draft;
     j.draft_tok = draft_tok;

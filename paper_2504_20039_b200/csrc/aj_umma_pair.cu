@@ -94,8 +94,8 @@ __device__ inline Tile decode_tile(const PairSched &sc, int t) {
 
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_h,
-                 int M, int V, int d, PairSched sc, int stream_w,
-                 unsigned long long *__restrict__ keys, int *__restrict__ status) {
+                 int M, int V, int d, PairSched sc, int stream_w, int v_offset,
+                 unsigned long long *__restrict__ keys, int *__restrict__ status, const Publish pub) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;  // the same offset in both CTAs: one descriptor serves both
@@ -262,7 +262,8 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
             for (int c = 0; c < NCH; c++) {
                 const int row = tl.row0 + c * 32 + lane;
                 if (c * 32 + lane < n_inst && row < M && best_u[c] != 0u) {
-                    const unsigned long long key = ((unsigned long long)best_u[c] << 32) | (uint32_t)(~(uint32_t)best_i[c]);
+                    const unsigned long long key =
+                        ((unsigned long long)best_u[c] << 32) | (uint32_t)(~(uint32_t)(best_i[c] + v_offset));
                     if (key > *reinterpret_cast<volatile unsigned long long *>(&keys[row])) atomicMax(&keys[row], key);
                 }
             }
@@ -272,6 +273,7 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
     __syncwarp();
     tc_fence_before();
     __syncthreads();
+    publish_keys(pub, keys);
     if (warp == 1 && *abort_flag) {
         // copies or MMAs may still be in flight after an abort: give them time to land
         const unsigned long long t0 = globaltimer_ns();
@@ -348,7 +350,8 @@ cudaError_t launch_umma_pair(const GemmArgs &a, const UmmaPlan &p, cudaStream_t 
     attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, umma_pair_kernel, p.tmap_w, p.tmap_h, a.M, a.V, a.d, sc, stream_w, a.keys, a.status);
+    return cudaLaunchKernelEx(&cfg, umma_pair_kernel, p.tmap_w, p.tmap_h, a.M, a.V, a.d, sc, stream_w, a.v_offset, a.keys,
+                              a.status, a.pub);
 }
 
 }  // namespace aj

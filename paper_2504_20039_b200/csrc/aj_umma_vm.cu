@@ -61,8 +61,8 @@ __device__ inline uint32_t warp_max_u32(uint32_t x) {
 template <int BN>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 umma_vm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_h,
-               int M, int V, int d, int n_n, int n_v, int stream_w,
-               unsigned long long *__restrict__ keys, int *__restrict__ status) {
+               int M, int V, int d, int n_n, int n_v, int stream_w, int v_offset,
+               unsigned long long *__restrict__ keys, int *__restrict__ status, const Publish pub) {
     using C = VCfg<BN>;
     constexpr int STAGES = C::STAGES;
     extern __shared__ uint8_t smem_raw[];
@@ -195,7 +195,7 @@ umma_vm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
             for (int c = 0; c < C::NCH; c++) {
                 const int row = n_tile * BN + c * 32 + lane;
                 if (row < M && rb_u[c] != 0u)
-                    atomicMax(&keys[row], ((unsigned long long)rb_u[c] << 32) | (uint32_t)(~(uint32_t)rb_i[c]));
+                    atomicMax(&keys[row], ((unsigned long long)rb_u[c] << 32) | (uint32_t)(~(uint32_t)(rb_i[c] + v_offset)));
                 rb_u[c] = 0u;
             }
         };
@@ -242,6 +242,7 @@ umma_vm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
     __syncwarp();
     tc_fence_before();
     __syncthreads();
+    publish_keys(pub, keys);
     if (warp == 1) {
         if (*abort_flag) {
             // copies or MMAs may still be in flight after an abort: give them time to land
@@ -268,8 +269,8 @@ cudaError_t launch_vm(const GemmArgs &a, const UmmaPlan &p, cudaStream_t stream)
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, umma_vm_kernel<BN>, p.tmap_w, p.tmap_h, a.M, a.V, a.d, n_n, n_v, stream_w, a.keys,
-                              a.status);
+    return cudaLaunchKernelEx(&cfg, umma_vm_kernel<BN>, p.tmap_w, p.tmap_h, a.M, a.V, a.d, n_n, n_v, stream_w, a.v_offset,
+                              a.keys, a.status, a.pub);
 }
 
 }  // namespace

@@ -91,3 +91,28 @@ def test_two_sm_schedule_covers_every_row_once(built):
     assert aj.pair_schedule(2112, 4096, 128256)["n_groups"] == 1
     assert aj.pair_schedule(2080, 8192, 128256)["n_groups"] == 1
     assert aj.pair_schedule(16640, 4096, 128256)["n_groups"] == 4
+
+
+def test_shard_ranges_are_whole_blocks_that_cover_the_vocabulary(built):
+    import paper_2504_20039_b200 as aj
+
+    for V in (128256, 1000, 256, 255, 70001):
+        for world in range(1, 9):
+            if -(-V // 256) < world:  # fewer blocks than GPUs: refused, no GPU gets an empty shard
+                with pytest.raises(aj.AjError):
+                    aj.shard_range(V, world, 0)
+                continue
+            parts = [aj.shard_range(V, world, r) for r in range(world)]
+            assert min(n for _, n in parts) >= 1
+            assert parts[0][0] == 0 and sum(n for _, n in parts) == V
+            for (b0, n0), (b1, _) in zip(parts, parts[1:]):
+                assert b0 + n0 == b1
+            assert all(b % 256 == 0 for b, _ in parts)
+            blocks = [-(-n // 256) for _, n in parts]
+            assert max(blocks) - min(blocks) <= 1
+    assert aj.shard_range(128256, 8, 0) == (0, 63 * 256) and aj.shard_range(128256, 8, 7) == (128256 - 62 * 256, 62 * 256)
+    assert aj.shard_exchange_bytes(4, 8, 9) == 0 and aj.shard_exchange_bytes(4, 8, 2) == 256 + 2 * 2 * 36 * 8
+    with pytest.raises(aj.AjError):
+        aj.shard_range(1000, 9, 0)
+    with pytest.raises(aj.AjError):
+        aj.shard_range(1000, 2, 2)

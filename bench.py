@@ -10,6 +10,8 @@ measurements use (batch size 1); the batched 8B- and 70B-shaped configurations a
 
 Rank layout for N > 1: one process per GPU, every rank verifies its own batch against its own copy
 of W_lm (sequences are independent, there is no data-path collective): weak scaling.
+With --sharding vocab the LM head is instead split by vocabulary over the ranks, all ranks verify the
+SAME batch and exchange their per-row keys inside the kernels (peer stores over NVLink): strong scaling.
 """
 from __future__ import annotations
 
@@ -105,7 +107,7 @@ class ClockSampler:
 class GpuWorkload:
     """One workload resident on the device: rotating copies of W_lm, inputs, outputs, handles."""
 
-    def __init__(self, cfg: gen.Config, device: int, w_copies: int, W_host=None, flags: int = 0):
+    def __init__(self, cfg: gen.Config, device: int, w_copies: int, W_host=None, flags: int = 0, group=None):
         import torch
 
         import paper_2504_20039_b200 as aj
@@ -114,6 +116,19 @@ class GpuWorkload:
         dev = f"cuda:{device}"
         bf = lambda a: torch.from_numpy(a.view(np.int16)).to(dev).view(torch.bfloat16)
         W_host = gen.make_W(cfg) if W_host is None else W_host
+        self.exchanges = []
+        self.v_count = cfg.V
+        shard = [None, None]
+        if group is not None:  # vocabulary-parallel: this rank keeps only its rows of W_lm
+            from paper_2504_20039_b200 import dist as ajd
+
+            v0, vn = aj.shard_range(cfg.V, group.info.world, group.info.rank)
+            W_host = W_host[v0 : v0 + vn]
+            self.v_count = vn
+            for i in range(2):  # one set of exchange buffers per handle: each handle counts its own cycles
+                ex = ajd.Exchange(group, cfg.B, cfg.K)
+                self.exchanges.append(ex)
+                shard[i] = (group.info.rank, group.info.world, v0, vn, ex.buffers)
         self.W = [bf(W_host)]
         for _ in range(w_copies - 1):
             self.W.append(self.W[0].clone())
@@ -125,8 +140,11 @@ class GpuWorkload:
         self.acc = torch.empty(cfg.B, **i32)
         self.nxt = torch.empty(cfg.B, **i32)
         self.tt = torch.empty((cfg.B, cfg.K + 1), **i32)
-        self.handle = aj.Handle(device, cfg.B, cfg.K, cfg.d, cfg.d_draft, cfg.V, aj.AJ_BF16, aj.AJ_W_VD, flags)
-        self.handle_t = aj.Handle(device, cfg.B, cfg.K, cfg.d, cfg.d_draft, cfg.V, aj.AJ_BF16, aj.AJ_W_VD, flags | aj.AJ_FLAG_TIME_KERNELS)
+        self.handle = aj.Handle(device, cfg.B, cfg.K, cfg.d, cfg.d_draft, cfg.V, aj.AJ_BF16, aj.AJ_W_VD, flags, shard=shard[0])
+        self.handle_t = aj.Handle(device, cfg.B, cfg.K, cfg.d, cfg.d_draft, cfg.V, aj.AJ_BF16, aj.AJ_W_VD,
+                                  flags | aj.AJ_FLAG_TIME_KERNELS, shard=shard[1])
+        for ex in self.exchanges:
+            ex.ready()
         # draft tokens planted against the device's own greedy tokens (a benchmark input, never an oracle input)
         self.tok = torch.from_numpy(gen.random_draft_tokens(cfg)).to(dev)
         self.step(self.handle, 0)
@@ -181,6 +199,9 @@ class GpuWorkload:
         return dt / steps, h2d, d2h
 
     def close(self):
+        self.torch.cuda.synchronize()
+        for ex in self.exchanges:
+            ex.close()
         self.handle.destroy()
         self.handle_t.destroy()
 
@@ -218,10 +239,12 @@ def traffic_of(cfg: gen.Config, path: str):
         return None
 
 
-def roofline_of(cfg: gen.Config, gemm_ms: float, pk):
-    """Roofline of the projection kernel: W streamed once from HBM vs 2*M*d*V flops on the tensor pipe."""
-    flops = 2.0 * cfg.M * cfg.d * cfg.V
-    byts = 2.0 * cfg.d * cfg.V + 2.0 * cfg.M * cfg.d + 8.0 * cfg.M
+def roofline_of(cfg: gen.Config, gemm_ms: float, pk, v_count=None):
+    """Roofline of the projection kernel: W streamed once from HBM vs 2*M*d*V flops on the tensor pipe
+    (V = the vocabulary entries this GPU projects)."""
+    V = cfg.V if v_count is None else v_count
+    flops = 2.0 * cfg.M * cfg.d * V
+    byts = 2.0 * cfg.d * V + 2.0 * cfg.M * cfg.d + 8.0 * cfg.M
     t_hbm = byts / (pk["hbm_gbs"] * 1e9)
     t_tc = flops / (pk["bf16_tflops"] * 1e12)
     s = gemm_ms * 1e-3
@@ -235,8 +258,8 @@ def roofline_of(cfg: gen.Config, gemm_ms: float, pk):
             "kernel_ms": gemm_ms, "algorithmic_flops": flops}
 
 
-def bench_one(cfg, device, steps, warmup, barrier, reduce_max, pk, w_copies, W_host=None, with_e2e=True, flags=0):
-    wl = GpuWorkload(cfg, device, w_copies, W_host, flags)
+def bench_one(cfg, device, steps, warmup, barrier, reduce_max, pk, w_copies, W_host=None, with_e2e=True, flags=0, group=None):
+    wl = GpuWorkload(cfg, device, w_copies, W_host, flags, group)
     try:
         wl.run(wl.handle, warmup)
         with ClockSampler(device) as cs:
@@ -252,7 +275,7 @@ def bench_one(cfg, device, steps, warmup, barrier, reduce_max, pk, w_copies, W_h
         assert wl.handle.last_status() == wl.aj.AJ_OK and wl.handle_t.last_status() == wl.aj.AJ_OK
         res = {
             "ms_per_step": ms / steps, "clocks": clocks, "path": wl.handle.last_gemm_path(),
-            "roofline": dict(roofline_of(cfg, gemm_mean, pk), traffic=traffic_of(cfg, wl.handle.last_gemm_path())),
+            "roofline": dict(roofline_of(cfg, gemm_mean, pk, wl.v_count), traffic=None if group is not None else traffic_of(cfg, wl.handle.last_gemm_path())),
             "gemm_ms_min": gemm_min, "gemm_launches_timed": n,
             "launches_per_step": wl.handle.last_launch_count(),
             "mean_accept_len": float(wl.acc.float().mean().item()),
@@ -329,6 +352,8 @@ def main():
     ap.add_argument("--no-extra", action="store_true", help="skip the batched configurations reported under 'extra'")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer (end-to-end) measurement; for profiler captures")
+    ap.add_argument("--sharding", default="batch", choices=["batch", "vocab"],
+                    help="batch: every rank its own batch and its own W_lm (default); vocab: W_lm split by vocabulary over the ranks")
     ap.add_argument("--flags", type=int, default=0, help="extra aj_create flags (kernel selection switches, for comparisons)")
     ap.add_argument("--w-copies", type=int, default=None, help="copies of W_lm to rotate over (default 3, or 2 for the 70B shape)")
     args = ap.parse_args()
@@ -352,16 +377,20 @@ def main():
     warmup = max(3, args.warmup if args.warmup is not None else 10)
     copies = args.w_copies or (3 if head.d * head.V * 2 < 1.5e9 else 2)
 
-    head = ajd.rank_config(head, rank)  # every rank verifies its own sequences
+    vocab = args.sharding == "vocab"
+    if not vocab:
+        head = ajd.rank_config(head, rank)  # every rank verifies its own sequences
     W_host = gen.make_W(head)
-    r = bench_one(head, local, steps, warmup, barrier, reduce_max, pk, copies, W_host, with_e2e=not args.no_e2e, flags=args.flags)
-    positions = ajd.job_positions(head, world)
+    r = bench_one(head, local, steps, warmup, barrier, reduce_max, pk, copies, W_host, with_e2e=not args.no_e2e, flags=args.flags,
+                  group=group if vocab else None)
+    positions = head.B * head.K if vocab else ajd.job_positions(head, world)
     line = {
         "metric": METRIC, "value": positions / (r["ms_per_step"] * 1e-3), "unit": UNIT, "n_gpus": world, "steps": steps,
         "warmup": warmup, "ms_per_step": r["ms_per_step"], "us_per_cycle": r["ms_per_step"] * 1e3, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "scaling": "strong" if vocab else "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": head.name, "B": head.B, "K": head.K, "d": head.d, "d_draft": head.d_draft, "V": head.V,
-                   "tau": head.tau, "match_rate": [head.match_lo, head.match_hi], "parallelism": f"replicated W, batch per rank x{world}",
+                   "tau": head.tau, "match_rate": [head.match_lo, head.match_hi], "parallelism": (f"W_lm split by vocabulary over {world} GPU(s), one batch, keys exchanged by peer stores inside the kernels"
+                                   if vocab else f"replicated W, batch per rank x{world}"),
                    "l2": f"W_lm rotates over {copies} copies of {head.d * head.V * 2 / 1e9:.2f} GB each (inputs larger than the 126 MB L2)",
                    "gemm_path": r["path"], "mean_accept_len": r["mean_accept_len"]},
         "clocks": r["clocks"], "roofline": r["roofline"],
@@ -378,7 +407,7 @@ def main():
         todo = []
         if args.workload == "sweep":
             todo = [gen.sweep_config(B, K) for B in gen.SWEEP_B for K in gen.SWEEP_K]
-        elif args.workload == "c2":
+        elif args.workload == "c2" and not vocab:
             todo = [gen.C3, gen.C4]
         for cfg in todo:
             cfg = ajd.rank_config(cfg, rank)

@@ -206,6 +206,15 @@ aj_status aj_verify_static(const void *h_target, const void *h_draft, const void
 /* Bytes of one GPU's exchange buffer; 0 if an argument is out of range (world in 1..8). */
 size_t aj_shard_exchange_bytes(int max_B, int max_K, int world);
 
+/*
+ * An exchange buffer on the CURRENT device, as its own cudaMalloc allocation (so that aj_ipc_export
+ * describes exactly this buffer), zero-filled; and its release.  A caller may instead pass any
+ * 256-byte aligned device memory of aj_shard_exchange_bytes() bytes that its peers can address.
+ * Errors: AJ_ERR_INVALID_ARG, AJ_ERR_CUDA.
+ */
+aj_status aj_shard_exchange_alloc(int max_B, int max_K, int world, void **device_ptr_out);
+aj_status aj_shard_exchange_free(void *device_ptr);
+
 /* The contiguous vocabulary range of rank `rank` among `world` GPUs: whole blocks of 256 entries,
  * spread evenly.  Errors: AJ_ERR_INVALID_ARG (also when V has fewer than `world` blocks). */
 aj_status aj_shard_range(int V, int world, int rank, int *v_begin, int *v_count);

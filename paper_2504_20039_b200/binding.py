@@ -19,7 +19,7 @@ AJ_FLAG_FORCE_SIMT, AJ_FLAG_TIME_KERNELS, AJ_FLAG_ROW_TILES, AJ_FLAG_ONE_SM = 1,
 
 EXPORTS = (
     "aj_create", "aj_verify", "aj_verify_host", "aj_last_status", "aj_last_gemm_ms", "aj_gemm_ms_stats", "aj_last_launch_count",
-    "aj_last_gemm_path", "aj_pair_schedule", "aj_destroy", "aj_shard_exchange_bytes", "aj_shard_range", "aj_create_sharded",
+    "aj_last_gemm_path", "aj_pair_schedule", "aj_destroy", "aj_shard_exchange_bytes", "aj_shard_exchange_alloc", "aj_shard_exchange_free", "aj_shard_range", "aj_create_sharded",
     "aj_shard_project", "aj_shard_finish", "aj_ipc_export", "aj_ipc_import", "aj_ipc_close", "aj_status_string", "aj_version", "aj_verify_static",
 )
 
@@ -69,6 +69,10 @@ def lib() -> ctypes.CDLL:
         L.aj_pair_schedule.restype = ci
         L.aj_shard_exchange_bytes.argtypes = [ci, ci, ci]
         L.aj_shard_exchange_bytes.restype = ctypes.c_size_t
+        L.aj_shard_exchange_alloc.argtypes = [ci, ci, ci, ctypes.POINTER(vp)]
+        L.aj_shard_exchange_alloc.restype = ci
+        L.aj_shard_exchange_free.argtypes = [vp]
+        L.aj_shard_exchange_free.restype = ci
         L.aj_shard_range.argtypes = [ci, ci, ci, ctypes.POINTER(ci), ctypes.POINTER(ci)]
         L.aj_shard_range.restype = ci
         L.aj_create_sharded.argtypes = [ctypes.POINTER(vp), ci, ci, ci, ci, ci, ci, ci, ci, cu, ci, ci, ci, ci, ctypes.POINTER(vp)]
@@ -141,6 +145,21 @@ def verify_static(h_target, h_draft, W_lm, draft_tok, judge_w, judge_b: float, t
 def shard_exchange_bytes(max_B: int, max_K: int, world: int) -> int:
     """aj_shard_exchange_bytes: size of one GPU's exchange buffer for a vocabulary-parallel group."""
     return int(lib().aj_shard_exchange_bytes(max_B, max_K, world))
+
+
+def shard_exchange_alloc(max_B: int, max_K: int, world: int) -> int:
+    """aj_shard_exchange_alloc: a zero-filled exchange buffer on the current device (its device address)."""
+    out = ctypes.c_void_p()
+    st = lib().aj_shard_exchange_alloc(max_B, max_K, world, ctypes.byref(out))
+    if st != AJ_OK:
+        raise AjError(st, "aj_shard_exchange_alloc")
+    return int(out.value)
+
+
+def shard_exchange_free(device_ptr: int) -> None:
+    st = lib().aj_shard_exchange_free(device_ptr)
+    if st != AJ_OK:
+        raise AjError(st, "aj_shard_exchange_free")
 
 
 def shard_range(V: int, world: int, rank: int):

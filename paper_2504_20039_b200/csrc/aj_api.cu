@@ -539,6 +539,30 @@ aj_status aj_shard_finish(aj_handle h, const void *h_target, const void *h_draft
     return st;
 }
 
+aj_status aj_shard_exchange_alloc(int max_B, int max_K, int world, void **device_ptr_out) {
+    if (!device_ptr_out) return AJ_ERR_INVALID_ARG;
+    *device_ptr_out = nullptr;
+    const size_t n = aj_shard_exchange_bytes(max_B, max_K, world);
+    if (n == 0) return AJ_ERR_INVALID_ARG;
+    void *p = nullptr;
+    if (cudaMalloc(&p, n) != cudaSuccess || cudaMemset(p, 0, n) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) {
+        cudaGetLastError();
+        if (p) cudaFree(p);
+        return AJ_ERR_CUDA;
+    }
+    *device_ptr_out = p;
+    return AJ_OK;
+}
+
+aj_status aj_shard_exchange_free(void *device_ptr) {
+    if (!device_ptr) return AJ_ERR_INVALID_ARG;
+    if (cudaFree(device_ptr) != cudaSuccess) {
+        cudaGetLastError();
+        return AJ_ERR_CUDA;
+    }
+    return AJ_OK;
+}
+
 aj_status aj_ipc_export(const void *device_ptr, unsigned char handle_out[64]) {
     if (!device_ptr || !handle_out) return AJ_ERR_INVALID_ARG;
     static_assert(sizeof(cudaIpcMemHandle_t) == 64, "IPC handle size");

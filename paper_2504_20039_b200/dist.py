@@ -48,6 +48,36 @@ def split_sequences(total: int, world: int):
     return out
 
 
+class Exchange:
+    """The exchange buffers of a vocabulary-parallel group, one per rank, as addressable from this
+    process: the own buffer is allocated here, the peers' are mapped through CUDA IPC handles that the
+    ranks swap over the process group.  `buffers[r]` is rank r's; pass the list to Handle(shard=...)."""
+
+    def __init__(self, group: "Group", max_B: int, max_K: int):
+        from . import binding as aj
+
+        self._aj, self.group = aj, group
+        rank, world = group.info.rank, group.info.world
+        self.own = aj.shard_exchange_alloc(max_B, max_K, world)
+        handles = group.all_gather_bytes(aj.ipc_export(self.own))
+        self.buffers = [self.own if r == rank else aj.ipc_import(handles[r]) for r in range(world)]
+        group.barrier()  # every rank has mapped every buffer
+
+    def ready(self) -> None:
+        """Call after every rank has created its handle (which clears its own buffer) and before the first cycle."""
+        self.group.barrier()
+
+    def close(self) -> None:
+        """Call after the last cycle has finished on this rank's stream."""
+        self.group.barrier()  # no rank is still publishing into a buffer about to go away
+        for r, p in enumerate(self.buffers):
+            if r != self.group.info.rank:
+                self._aj.ipc_close(p)
+        self.group.barrier()
+        self._aj.shard_exchange_free(self.own)
+        self.buffers = []
+
+
 class Group:
     """A thin wrapper over torch.distributed that degrades to a no-op for a single process."""
 

@@ -143,14 +143,17 @@ int aj_last_launch_count(aj_handle h);
 /*
  * How the two-SM projection kernel cuts a batch of M = B*(K+1) rows against a vocabulary of V entries
  * (host arithmetic only, no device needed; for tests and diagnostics).  out receives
- *   [0] blocks of 256 vocabulary entries        [1] row tiles (each at most 256 rows)
+ *   [0] blocks of 256 vocabulary entries        [1] row tiles
  *   [2],[3] row tile i holds out[2] + (i < out[3]) units of 16 rows
- *   [4] rows of h_target each SM of a pair stages per 64-column block
+ *   [4] rows of h_target each SM of a pair stages per 64-column block and accumulator
  *   [5] groups the row tiles are walked in (each group against the whole vocabulary, so that a
  *       group's rows of h_target stay in L2)    [6],[7] group g holds out[6] + (g < out[7]) row tiles
+ *   [8] 1 if each tile uses two accumulators that share the staged block of W_lm (257..512 rows: one
+ *       pass over W_lm for all rows, a tile then holds up to 512 rows), else 0 (tiles of at most 256
+ *       rows on one accumulator, double-buffered)      [9] depth of the shared-memory ring
  * Errors: AJ_ERR_INVALID_ARG.
  */
-aj_status aj_pair_schedule(int M, int d, int V, int32_t out[8]);
+aj_status aj_pair_schedule(int M, int d, int V, int32_t out[10]);
 
 /* Name of the projection kernel configuration the most recent call used, e.g. "umma_128x256". */
 const char *aj_last_gemm_path(aj_handle h);

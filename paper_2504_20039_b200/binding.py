@@ -117,11 +117,11 @@ AJ_STATIC_MAX_ROWS = 32768
 
 def pair_schedule(M: int, d: int, V: int) -> dict:
     """aj_pair_schedule: how the two-SM kernel tiles M rows against V vocabulary entries (host arithmetic)."""
-    out = (ctypes.c_int32 * 8)()
+    out = (ctypes.c_int32 * 10)()
     st = lib().aj_pair_schedule(M, d, V, out)
     if st != AJ_OK:
         raise AjError(st, "aj_pair_schedule")
-    keys = ("n_v", "n_n", "u_base", "u_rem", "box_rows", "n_groups", "g_base", "g_rem")
+    keys = ("n_v", "n_n", "u_base", "u_rem", "box_rows", "n_groups", "g_base", "g_rem", "dual", "stages")
     return dict(zip(keys, (int(x) for x in out)))
 
 

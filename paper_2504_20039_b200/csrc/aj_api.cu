@@ -598,7 +598,7 @@ aj_status aj_ipc_close(void *device_ptr) {
 
 int aj_last_launch_count(aj_handle h) { return h ? h->last_launches : 0; }
 
-aj_status aj_pair_schedule(int M, int d, int V, int32_t out[8]) {
+aj_status aj_pair_schedule(int M, int d, int V, int32_t out[10]) {
     if (!out || M < 1 || d < 1 || V < 1) return AJ_ERR_INVALID_ARG;
     const PairSched sc = pair_schedule(M, V, d);
     out[0] = sc.n_v;
@@ -609,6 +609,8 @@ aj_status aj_pair_schedule(int M, int d, int V, int32_t out[8]) {
     out[5] = sc.n_groups;
     out[6] = sc.g_base;
     out[7] = sc.g_rem;
+    out[8] = sc.dual;
+    out[9] = sc.stages;
     return AJ_OK;
 }
 

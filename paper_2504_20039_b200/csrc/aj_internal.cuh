@@ -138,7 +138,9 @@ struct PairSched {
     int n_v;               // blocks of 256 vocabulary entries
     int n_n;               // row tiles
     int u_base, u_rem;     // row tile i holds u_base + (i < u_rem) units of 16 rows
-    int box_rows;          // rows of h each CTA of a pair stages per k-block
+    int box_rows;          // rows of h each CTA of a pair stages per k-block and accumulator
+    int dual;              // 1: every tile uses two accumulators that share the staged block of W
+    int stages;            // depth of the shared-memory ring
     int n_groups;          // row tiles are walked in groups ...
     int g_base, g_rem;     // ... group g holds g_base + (g < g_rem) row tiles
 };

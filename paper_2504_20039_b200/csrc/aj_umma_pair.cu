@@ -39,18 +39,17 @@ namespace {
 
 constexpr int BV = 256;       // vocabulary entries per tile (128 per CTA)
 constexpr int BV_CTA = 128;
-constexpr int BN = 256;       // rows of h per tile (half of them staged by each CTA)
+constexpr int BN = 256;       // rows of h per accumulator (half of them staged by each CTA)
 constexpr int BK = 64;        // bf16 elements per k-block = 128 bytes = one swizzle span
 constexpr int UMMA_K = 16;
 constexpr int NUM_THREADS = 192;
-constexpr int A_BYTES = BV_CTA * BK * 2;        // 16 KB
-constexpr int B_BYTES = (BN / 2) * BK * 2;      // 16 KB
-constexpr int STAGE_BYTES = A_BYTES + B_BYTES;  // per CTA
-constexpr int STAGES = 6;
+constexpr int A_BYTES = BV_CTA * BK * 2;   // 16 KB: this CTA's 128 rows of W, one k-block
+constexpr int RING_BYTES = 192 * 1024;     // shared memory given to the stage ring
+constexpr int MAX_STAGES = 8;
 constexpr int TMEM_COLS = 2 * BN;
 constexpr int NCH = BN / 32;
-constexpr int BAR_BYTES = 8 * (2 * STAGES + 4) + 16;
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + BAR_BYTES + 1024;
+constexpr int BAR_BYTES = 8 * (2 * MAX_STAGES + 4) + 16;
+constexpr int SMEM_BYTES = RING_BYTES + BAR_BYTES + 1024;
 
 __device__ inline uint32_t ordered_image(float x) {
     const uint32_t b = __float_as_uint(x + 0.0f);  // -0.0 + 0.0 = +0.0: the two zeros tie
@@ -64,9 +63,9 @@ __device__ inline uint32_t warp_max(uint32_t x) {
 }
 
 struct Tile {
-    int v_tile;  // block of 256 vocabulary entries
-    int row0;    // first row of h
-    int n_inst;  // rows in the tile = UMMA N, a multiple of 16
+    int v_tile;     // block of 256 vocabulary entries
+    int row0[2];    // first row of h of each accumulator
+    int n_inst[2];  // rows of each accumulator = UMMA N, a multiple of 16 (the second is 0 in single mode)
 };
 
 // Tile t of the schedule.  Row tiles come in groups; a group is walked against every vocabulary
@@ -74,7 +73,7 @@ struct Tile {
 // neighbouring pairs at the same time, share a block of W.  Which row tile of the group a pair gets
 // rotates with the vocabulary block, so that pairs whose number is a multiple of the group size
 // apart do not always get the larger (or the smaller) row tiles and drift away from the pairs they
-// share W with.
+// share W with.  In dual mode a row tile is split over the two accumulators.
 __device__ inline Tile decode_tile(const PairSched &sc, int t) {
     int g = 0, start = 0, sz = sc.g_base + (0 < sc.g_rem ? 1 : 0);
     while (g + 1 < sc.n_groups && t >= start + sz * sc.n_v) {
@@ -87,8 +86,13 @@ __device__ inline Tile decode_tile(const PairSched &sc, int t) {
     Tile r;
     r.v_tile = local / sz;
     const int n_tile = first + (local % sz + r.v_tile) % sz;
-    r.row0 = 16 * (n_tile * sc.u_base + min(n_tile, sc.u_rem));
-    r.n_inst = 16 * (sc.u_base + (n_tile < sc.u_rem ? 1 : 0));
+    const int u0 = n_tile * sc.u_base + min(n_tile, sc.u_rem);
+    const int nu = sc.u_base + (n_tile < sc.u_rem ? 1 : 0);
+    const int nu0 = sc.dual ? (nu + 1) >> 1 : nu;
+    r.row0[0] = 16 * u0;
+    r.n_inst[0] = 16 * nu0;
+    r.row0[1] = 16 * (u0 + nu0);
+    r.n_inst[1] = 16 * (nu - nu0);
     return r;
 }
 
@@ -101,12 +105,12 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
     const uint32_t base = (raw + 1023u) & ~1023u;  // the same offset in both CTAs: one descriptor serves both
     uint8_t *smem = smem_raw + (base - raw);
 
-    const uint32_t bar_base = base + STAGES * STAGE_BYTES;
-    auto full_bar = [&](int s) { return bar_base + 8u * s; };                      // used in the leader only
-    auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
-    auto acc_full_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
-    auto acc_empty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };  // used in the leader only
-    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + STAGES * STAGE_BYTES + 8 * (2 * STAGES + 4));
+    const uint32_t bar_base = base + RING_BYTES;
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };                                  // used in the leader only
+    auto empty_bar = [&](int s) { return bar_base + 8u * (MAX_STAGES + s); };
+    auto acc_full_bar = [&](int a) { return bar_base + 8u * (2 * MAX_STAGES + a); };
+    auto acc_empty_bar = [&](int a) { return bar_base + 8u * (2 * MAX_STAGES + 2 + a); };      // used in the leader only
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + RING_BYTES + 8 * (2 * MAX_STAGES + 4));
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5;  // warp-uniform
@@ -116,10 +120,14 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
     const int num_pairs = gridDim.x >> 1;
     const int num_kb = d / BK;
     const int num_tiles = sc.n_n * sc.n_v;
-    const uint32_t stage_tx = 2u * (uint32_t)(A_BYTES + sc.box_rows * BK * 2);  // bytes both CTAs load per stage
+    const int n_acc = sc.dual ? 2 : 1;
+    const int stages = sc.stages;
+    const uint32_t b_bytes = (uint32_t)sc.box_rows * BK * 2;       // one accumulator's rows of h staged by this CTA
+    const uint32_t stage_bytes = A_BYTES + n_acc * b_bytes;         // a multiple of 1024
+    const uint32_t stage_tx = 2u * stage_bytes;                     // bytes both CTAs load per stage
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; s++) {
+        for (int s = 0; s < MAX_STAGES; s++) {
             mbar_init(full_bar(s), 1);   // the leader's producer; bytes arrive from both CTAs
             mbar_init(empty_bar(s), 1);  // one commit from the leader's MMA thread
         }
@@ -144,6 +152,11 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
         *abort_flag = 1;
         atomicCAS(status, DEV_OK, DEV_TIMEOUT);
     };
+    // Accumulator hand-over.  Single mode: the two 256-column buffers alternate from tile to tile
+    // (buffer it & 1, each with its own pair of barriers).  Dual mode: every tile uses both buffers
+    // as two accumulators that share the staged block of W, and one pair of barriers.
+    auto acc_slot = [&](int it) { return sc.dual ? 0 : (it & 1); };
+    auto acc_phase = [&](int it) { return (uint32_t)(sc.dual ? it : (it >> 1)) & 1u; };
 
     if (warp == 0) {
         if (lane == 0) {
@@ -156,7 +169,8 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
             for (int t = pair; ok && t < num_tiles; t += num_pairs) {
                 const Tile tl = decode_tile(sc, t);
                 const int w_row = tl.v_tile * BV + (int)rank * BV_CTA;
-                const int h_row = tl.row0 + (int)rank * (tl.n_inst >> 1);
+                const int h_row0 = tl.row0[0] + (int)rank * (tl.n_inst[0] >> 1);
+                const int h_row1 = tl.row0[1] + (int)rank * (tl.n_inst[1] >> 1);
                 for (int kb = 0; kb < num_kb; kb++) {
                     if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) {
                         give_up();
@@ -165,10 +179,11 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
                     }
                     const uint32_t leader_full = map_to_cta(full_bar(s), 0);
                     if (rank == 0) mbar_expect_tx(full_bar(s), stage_tx);
-                    const uint32_t a_dst = base + s * STAGE_BYTES;
+                    const uint32_t a_dst = base + s * stage_bytes;
                     tma_load_2d_pair(a_dst, &tmap_w, kb * BK, w_row, leader_full, pol_w);
-                    tma_load_2d_pair(a_dst + A_BYTES, &tmap_h, kb * BK, h_row, leader_full, pol_h);
-                    if (++s == STAGES) {
+                    tma_load_2d_pair(a_dst + A_BYTES, &tmap_h, kb * BK, h_row0, leader_full, pol_h);
+                    if (n_acc == 2) tma_load_2d_pair(a_dst + A_BYTES + b_bytes, &tmap_h, kb * BK, h_row1, leader_full, pol_h);
+                    if (++s == stages) {
                         s = 0;
                         ph ^= 1u;
                     }
@@ -183,15 +198,17 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
             bool ok = true;
             int it = 0;
             for (int t = pair; ok && t < num_tiles; t += num_pairs, ++it) {
-                const uint32_t idesc = instr_desc(BV, decode_tile(sc, t).n_inst);
-                const int ab = it & 1;
-                const uint32_t aph = (uint32_t)(it >> 1) & 1u;
-                if (!mbar_wait(acc_empty_bar(ab), aph ^ 1u, abort_flag)) {
+                const Tile tl = decode_tile(sc, t);
+                const uint32_t idesc0 = instr_desc(BV, tl.n_inst[0]);
+                const uint32_t idesc1 = instr_desc(BV, tl.n_inst[1]);
+                const int slot = acc_slot(it);
+                if (!mbar_wait(acc_empty_bar(slot), acc_phase(it) ^ 1u, abort_flag)) {
                     give_up();
                     break;
                 }
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(ab * BN);
+                const uint32_t d_tmem0 = tmem_base + (uint32_t)(slot * BN);
+                const uint32_t d_tmem1 = tmem_base + (uint32_t)BN;  // dual mode only
                 for (int kb = 0; kb < num_kb; kb++) {
                     if (!mbar_wait(full_bar(s), ph, abort_flag)) {
                         give_up();
@@ -199,19 +216,25 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
                         break;
                     }
                     tc_fence_after();
-                    const uint32_t a_addr = base + s * STAGE_BYTES;
+                    const uint32_t a_addr = base + s * stage_bytes;
                     const unsigned long long adesc = smem_desc_sw128(a_addr);
-                    const unsigned long long bdesc = smem_desc_sw128(a_addr + A_BYTES);
+                    const unsigned long long bdesc0 = smem_desc_sw128(a_addr + A_BYTES);
 #pragma unroll
                     for (int k = 0; k < BK / UMMA_K; k++)
-                        umma_bf16_pair(d_tmem, adesc + 2ull * k, bdesc + 2ull * k, idesc, (uint32_t)((kb | k) != 0));
+                        umma_bf16_pair(d_tmem0, adesc + 2ull * k, bdesc0 + 2ull * k, idesc0, (uint32_t)((kb | k) != 0));
+                    if (n_acc == 2) {
+                        const unsigned long long bdesc1 = smem_desc_sw128(a_addr + A_BYTES + b_bytes);
+#pragma unroll
+                        for (int k = 0; k < BK / UMMA_K; k++)
+                            umma_bf16_pair(d_tmem1, adesc + 2ull * k, bdesc1 + 2ull * k, idesc1, (uint32_t)((kb | k) != 0));
+                    }
                     umma_commit_pair(empty_bar(s));  // frees the stage in both CTAs
-                    if (++s == STAGES) {
+                    if (++s == stages) {
                         s = 0;
                         ph ^= 1u;
                     }
                 }
-                if (ok) umma_commit_pair(acc_full_bar(ab));  // the accumulator halves in both CTAs are complete
+                if (ok) umma_commit_pair(acc_full_bar(slot));  // the accumulators in both CTAs are complete
             }
         }
     } else {
@@ -220,51 +243,55 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
         int it = 0;
         for (int t = pair; t < num_tiles; t += num_pairs, ++it) {
             const Tile tl = decode_tile(sc, t);
-            const int n_inst = tl.n_inst;
-            const int ab = it & 1;
-            const uint32_t aph = (uint32_t)(it >> 1) & 1u;
+            const int slot = acc_slot(it);
             // the whole warp takes one decision, so the aligned TMEM loads below stay converged
-            if (!__all_sync(0xffffffffu, mbar_wait(acc_full_bar(ab), aph, abort_flag))) {
+            if (!__all_sync(0xffffffffu, mbar_wait(acc_full_bar(slot), acc_phase(it), abort_flag))) {
                 give_up();
                 break;
             }
             tc_fence_after();
             const int v_first = tl.v_tile * BV + (int)rank * BV_CTA + q * 32;  // vocabulary entry of lane 0
             const bool v_ok = v_first + lane < V;                            // entries past V hold zero-filled junk
-            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ab * BN);
-            uint32_t best_u[NCH];  // lane j, chunk c: maximum of column 32c + j over this warp's 32 entries
-            int best_i[NCH];
+#pragma unroll 1
+            for (int a = 0; a < n_acc; a++) {
+                const int n_inst = tl.n_inst[a];
+                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)((sc.dual ? a : slot) * BN);
+                uint32_t best_u[NCH];  // lane j, chunk c: maximum of column 32c + j over this warp's 32 entries
+                int best_i[NCH];
 #pragma unroll
-            for (int c = 0; c < NCH; c++) {
-                best_u[c] = 0u;
-                best_i[c] = 0;
-                if (c * 32 < n_inst) {  // warp-uniform
-                    float v[32];
-                    tmem_ld32(taddr + c * 32, v);
+                for (int c = 0; c < NCH; c++) {
+                    best_u[c] = 0u;
+                    best_i[c] = 0;
+                    if (c * 32 < n_inst) {  // warp-uniform
+                        float v[32];
+                        tmem_ld32(taddr + c * 32, v);
 #pragma unroll
-                    for (int j = 0; j < 32; j++) {
-                        const uint32_t u = v_ok ? ordered_image(v[j]) : 0u;
-                        const uint32_t m = warp_max(u);
-                        const uint32_t who = __ballot_sync(0xffffffffu, u == m);
-                        if (lane == j) {
-                            best_u[c] = m;
-                            best_i[c] = v_first + __ffs(who) - 1;  // the lowest entry that attains the maximum
+                        for (int j = 0; j < 32; j++) {
+                            const uint32_t u = v_ok ? ordered_image(v[j]) : 0u;
+                            const uint32_t m = warp_max(u);
+                            const uint32_t who = __ballot_sync(0xffffffffu, u == m);
+                            if (lane == j) {
+                                best_u[c] = m;
+                                best_i[c] = v_first + __ffs(who) - 1;  // the lowest entry that attains the maximum
+                            }
                         }
                     }
                 }
-            }
-            // the accumulator buffer is drained: hand it back to the leader's MMA thread
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(map_to_cta(acc_empty_bar(ab), 0));
-            // merge this tile's column maxima into the rows' keys
+                if (a == n_acc - 1) {
+                    // the accumulators are drained: hand them back to the leader's MMA thread
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_cluster(map_to_cta(acc_empty_bar(slot), 0));
+                }
+                // merge this accumulator's column maxima into the rows' keys
 #pragma unroll
-            for (int c = 0; c < NCH; c++) {
-                const int row = tl.row0 + c * 32 + lane;
-                if (c * 32 + lane < n_inst && row < M && best_u[c] != 0u) {
-                    const unsigned long long key =
-                        ((unsigned long long)best_u[c] << 32) | (uint32_t)(~(uint32_t)(best_i[c] + v_offset));
-                    if (key > *reinterpret_cast<volatile unsigned long long *>(&keys[row])) atomicMax(&keys[row], key);
+                for (int c = 0; c < NCH; c++) {
+                    const int row = tl.row0[a] + c * 32 + lane;
+                    if (c * 32 + lane < n_inst && row < M && best_u[c] != 0u) {
+                        const unsigned long long key =
+                            ((unsigned long long)best_u[c] << 32) | (uint32_t)(~(uint32_t)(best_i[c] + v_offset));
+                        if (key > *reinterpret_cast<volatile unsigned long long *>(&keys[row])) atomicMax(&keys[row], key);
+                    }
                 }
             }
         }
@@ -318,11 +345,20 @@ int umma_pair_max_pairs() { return g_max_pairs; }
 PairSched pair_schedule(int M, int V, int d) {
     PairSched sc;
     const int units = (M + 15) / 16;  // rows in units of 16 (the UMMA N granule)
-    sc.n_n = (units + 15) / 16;       // fewest tiles of at most 256 rows
+    // Between 257 and 512 rows one tile takes all rows on two accumulators that share each staged
+    // block of W (no second pass over W, no accumulator double-buffering); otherwise the fewest
+    // tiles of at most 256 rows, one accumulator each, double-buffered.
+    sc.dual = (units > 16 && units <= 32) ? 1 : 0;
+    const int cap = sc.dual ? 32 : 16;
+    sc.n_n = (units + cap - 1) / cap;
     sc.u_base = units / sc.n_n;
     sc.u_rem = units % sc.n_n;
     sc.n_v = (V + BV - 1) / BV;
-    sc.box_rows = 8 * (sc.u_base + (sc.u_rem ? 1 : 0));  // rows of h each CTA stages: half of the largest tile
+    const int u_max = sc.u_base + (sc.u_rem ? 1 : 0);
+    // rows of h each CTA stages per accumulator: half of the largest accumulator
+    sc.box_rows = 8 * (sc.dual ? (u_max + 1) / 2 : u_max);
+    const int stage_bytes = A_BYTES + (sc.dual ? 2 : 1) * sc.box_rows * BK * 2;
+    sc.stages = RING_BYTES / stage_bytes < MAX_STAGES ? RING_BYTES / stage_bytes : MAX_STAGES;
     // row tiles per group: keep a group's rows of h (tile rows x d x 2 bytes) within about 40 MB of L2
     const long long tile_bytes = 256ll * d * 2;
     int g_max = (int)((40ll << 20) / tile_bytes);

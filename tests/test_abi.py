@@ -75,16 +75,21 @@ def test_two_sm_schedule_covers_every_row_once(built):
     cover the batch exactly once with no padded tile, and groups that cover every tile once."""
     import paper_2504_20039_b200 as aj
 
-    for M, d in [(129, 4096), (136, 4096), (256, 4096), (257, 4096), (264, 4096), (520, 4096), (2112, 4096),
-                 (2080, 8192), (8448, 4096), (16640, 4096), (16640, 8192), (4097, 64)]:
+    for M, d in [(129, 4096), (136, 4096), (256, 4096), (257, 4096), (264, 4096), (500, 4096), (512, 4096), (513, 4096),
+                 (520, 4096), (2112, 4096), (2080, 8192), (8448, 4096), (16640, 4096), (16640, 8192), (4097, 64)]:
         s = aj.pair_schedule(M, d, 128256)
         assert s["n_v"] == 501
         units = (M + 15) // 16
+        assert s["dual"] == (1 if 256 < M <= 512 else 0)
+        cap = 32 if s["dual"] else 16                         # units per tile: two accumulators or one
         sizes = [s["u_base"] + (i < s["u_rem"]) for i in range(s["n_n"])]
-        assert sum(sizes) == units and max(sizes) <= 16 and min(sizes) >= 1
-        assert s["n_n"] == -(-units // 16)                    # the fewest tiles of at most 256 rows
+        assert sum(sizes) == units and max(sizes) <= cap and min(sizes) >= (2 if s["dual"] else 1)
+        assert s["n_n"] == -(-units // cap)                   # the fewest tiles
         assert max(sizes) - min(sizes) <= 1                   # spread evenly
-        assert s["box_rows"] == 8 * max(sizes) <= 128
+        per_acc = -(-max(sizes) // 2) if s["dual"] else max(sizes)
+        assert s["box_rows"] == 8 * per_acc <= 128
+        stage = 16384 + (2 if s["dual"] else 1) * s["box_rows"] * 128
+        assert 4 <= s["stages"] == min(8, (192 * 1024) // stage) and s["stages"] * stage <= 192 * 1024
         groups = [s["g_base"] + (g < s["g_rem"]) for g in range(s["n_groups"])]
         assert sum(groups) == s["n_n"] and min(groups) >= 1 and max(groups) - min(groups) <= 1
         assert max(groups) * 256 * d * 2 <= 40 << 20 or max(groups) == 1

@@ -44,7 +44,7 @@ constexpr int BK = 64;        // bf16 elements per k-block = 128 bytes = one swi
 constexpr int UMMA_K = 16;
 constexpr int NUM_THREADS = 192;
 constexpr int A_BYTES = BV_CTA * BK * 2;   // 16 KB: this CTA's 128 rows of W, one k-block
-constexpr int RING_BYTES = 192 * 1024;     // shared memory given to the stage ring
+constexpr int RING_BYTES = 224 * 1024;     // shared memory given to the stage ring (the SM has 227 KB per CTA)
 constexpr int MAX_STAGES = 8;
 constexpr int TMEM_COLS = 2 * BN;
 constexpr int NCH = BN / 32;

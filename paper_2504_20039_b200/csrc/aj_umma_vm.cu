@@ -39,7 +39,7 @@ constexpr int A_BYTES = BV * BK * 2;
 template <int BN> struct VCfg {
     static constexpr int B_BYTES = BN * BK * 2;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int STAGES = (192 * 1024) / STAGE_BYTES;
+    static constexpr int STAGES = (224 * 1024) / STAGE_BYTES;  // the SM has 227 KB per CTA
     static constexpr int TMEM_COLS = 2 * BN < 32 ? 32 : 2 * BN;
     static constexpr int NCH = (BN + 31) / 32;  // 32-column chunks per accumulator
     static constexpr int BAR_BYTES = 8 * (2 * STAGES + 4) + 16;

@@ -22,11 +22,11 @@
 //               W[v0 + 128*rank .. +128, kb] and h[n0 + (N/2)*rank .. , kb] with 128-byte swizzle;
 //   warp 1      allocates tensor memory (both CTAs); in the leader one thread issues the MMAs and
 //               commits stage-release and accumulator-ready barriers to both CTAs at once;
-//   warps 2..5  epilogue: thread = one TMEM lane = one vocabulary entry; per column (row of h) the
-//               warp maximum by redux.sync on the order-preserving image of the logit, the lowest
-//               lane attaining it by ballot; lane j keeps the running (max, argmax) of column j and
-//               merges it into the row's packed key with a 64-bit atomic max when the tile is done
-//               (skipped when the key in memory already beats it).
+//   warps 2..5  epilogue: thread = one TMEM lane = one vocabulary entry.  32 columns (rows of h) at a
+//               time are compared with the best value each row has so far (read from its key); only
+//               a chunk in which some logit reaches that value is reduced (per column the warp
+//               maximum by redux.sync on the order-preserving image of the logit, the lowest lane
+//               attaining it by ballot) and merged into the row's packed key by a 64-bit atomic max.
 // Two accumulator buffers of 256 columns: the epilogue of one tile runs under the MMAs of the next.
 // No split over k.  Every wait is bounded; a wait that runs out sets the status word, and both CTAs
 // still meet at the cluster barrier before tensor memory is freed.
@@ -47,7 +47,6 @@ constexpr int A_BYTES = BV_CTA * BK * 2;   // 16 KB: this CTA's 128 rows of W, o
 constexpr int RING_BYTES = 224 * 1024;     // shared memory given to the stage ring (the SM has 227 KB per CTA)
 constexpr int MAX_STAGES = 8;
 constexpr int TMEM_COLS = 2 * BN;
-constexpr int NCH = BN / 32;
 constexpr int BAR_BYTES = 8 * (2 * MAX_STAGES + 4) + 16;
 constexpr int SMEM_BYTES = RING_BYTES + BAR_BYTES + 1024;
 
@@ -239,11 +238,32 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
         }
     } else {
         // -------------------------------------------------------------------- epilogue
+        // A logit can only matter if it reaches the best value its row has so far.  Lane j reads
+        // that value for column 32c + j from the row's key before the tile's accumulators are
+        // ready (a stale value is only lower, never wrong).  A chunk of 32 columns is then checked
+        // with one comparison per element against the shuffled-in thresholds and one vote; only
+        // if some element qualifies does the chunk take the reduction path (warp maximum per
+        // column by redux.sync, lowest lane by ballot, 64-bit atomic max into the key).  After the
+        // first few vocabulary blocks nearly every chunk is skipped.
         const int q = warp & 3;  // TMEM lane quadrant this warp may read
+        const float never = __int_as_float(0x7fc00000);  // NaN: no comparison with it is ever true
+        // Chunk g of a tile is columns 32 (g & 7) .. + 32 of accumulator g >> 3.  Its threshold for
+        // lane j is the best value the row of column 32 (g & 7) + j has so far, read from the key.
+        auto load_thr = [&](const Tile &tl, int g) {
+            const int a = g >> 3, col = (g & 7) * 32 + lane;
+            const int row = (a ? tl.row0[1] : tl.row0[0]) + col;
+            if (a >= n_acc || col >= (a ? tl.n_inst[1] : tl.n_inst[0]) || row >= M) return never;
+            const unsigned long long k = __ldcg(keys + row);
+            return k == 0ull ? -INFINITY : key_value(k);
+        };
+        constexpr int GRP = 4;  // thresholds are fetched four chunks ahead of their use: an L2 round trip
         int it = 0;
         for (int t = pair; t < num_tiles; t += num_pairs, ++it) {
             const Tile tl = decode_tile(sc, t);
             const int slot = acc_slot(it);
+            float cur[GRP], nxt[GRP];
+#pragma unroll
+            for (int u = 0; u < GRP; u++) cur[u] = load_thr(tl, u);  // in flight while the accumulators are being computed
             // the whole warp takes one decision, so the aligned TMEM loads below stay converged
             if (!__all_sync(0xffffffffu, mbar_wait(acc_full_bar(slot), acc_phase(it), abort_flag))) {
                 give_up();
@@ -252,48 +272,52 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
             tc_fence_after();
             const int v_first = tl.v_tile * BV + (int)rank * BV_CTA + q * 32;  // vocabulary entry of lane 0
             const bool v_ok = v_first + lane < V;                            // entries past V hold zero-filled junk
+            const uint32_t tbase = tmem_base + ((uint32_t)(q * 32) << 16);
+            // the group loop is kept rolled: one copy of the code stays in the instruction cache
 #pragma unroll 1
-            for (int a = 0; a < n_acc; a++) {
-                const int n_inst = tl.n_inst[a];
-                const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)((sc.dual ? a : slot) * BN);
-                uint32_t best_u[NCH];  // lane j, chunk c: maximum of column 32c + j over this warp's 32 entries
-                int best_i[NCH];
+            for (int g0 = 0; g0 < 8 * n_acc; g0 += GRP) {
 #pragma unroll
-                for (int c = 0; c < NCH; c++) {
-                    best_u[c] = 0u;
-                    best_i[c] = 0;
+                for (int u = 0; u < GRP; u++) nxt[u] = (g0 + GRP < 8 * n_acc) ? load_thr(tl, g0 + GRP + u) : never;
+#pragma unroll
+                for (int u = 0; u < GRP; u++) {
+                    const int g = g0 + u, a = g >> 3, c = g & 7;
+                    const int n_inst = a ? tl.n_inst[1] : tl.n_inst[0];
                     if (c * 32 < n_inst) {  // warp-uniform
+                        const float thr = cur[u];
                         float v[32];
-                        tmem_ld32(taddr + c * 32, v);
+                        tmem_ld32(tbase + (uint32_t)((sc.dual ? a : slot) * BN + c * 32), v);
+                        bool hit = false;
 #pragma unroll
-                        for (int j = 0; j < 32; j++) {
-                            const uint32_t u = v_ok ? ordered_image(v[j]) : 0u;
-                            const uint32_t m = warp_max(u);
-                            const uint32_t who = __ballot_sync(0xffffffffu, u == m);
-                            if (lane == j) {
-                                best_u[c] = m;
-                                best_i[c] = v_first + __ffs(who) - 1;  // the lowest entry that attains the maximum
+                        for (int j = 0; j < 32; j++) hit |= v[j] >= __shfl_sync(0xffffffffu, thr, j);
+                        if (__any_sync(0xffffffffu, hit && v_ok)) {
+                            uint32_t best_u = 0u;  // lane j: maximum of column 32c + j over this warp's 32 entries
+                            int best_i = 0;
+#pragma unroll
+                            for (int j = 0; j < 32; j++) {
+                                const uint32_t x = v_ok ? ordered_image(v[j]) : 0u;
+                                const uint32_t m = warp_max(x);
+                                const uint32_t who = __ballot_sync(0xffffffffu, x == m);
+                                if (lane == j) {
+                                    best_u = m;
+                                    best_i = v_first + __ffs(who) - 1;  // the lowest entry that attains the maximum
+                                }
+                            }
+                            const int row = (a ? tl.row0[1] : tl.row0[0]) + c * 32 + lane;
+                            if (c * 32 + lane < n_inst && row < M && best_u != 0u) {
+                                const unsigned long long key =
+                                    ((unsigned long long)best_u << 32) | (uint32_t)(~(uint32_t)(best_i + v_offset));
+                                if (key > *reinterpret_cast<volatile unsigned long long *>(&keys[row])) atomicMax(&keys[row], key);
                             }
                         }
                     }
                 }
-                if (a == n_acc - 1) {
-                    // the accumulators are drained: hand them back to the leader's MMA thread
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive_cluster(map_to_cta(acc_empty_bar(slot), 0));
-                }
-                // merge this accumulator's column maxima into the rows' keys
 #pragma unroll
-                for (int c = 0; c < NCH; c++) {
-                    const int row = tl.row0[a] + c * 32 + lane;
-                    if (c * 32 + lane < n_inst && row < M && best_u[c] != 0u) {
-                        const unsigned long long key =
-                            ((unsigned long long)best_u[c] << 32) | (uint32_t)(~(uint32_t)(best_i[c] + v_offset));
-                        if (key > *reinterpret_cast<volatile unsigned long long *>(&keys[row])) atomicMax(&keys[row], key);
-                    }
-                }
+                for (int u = 0; u < GRP; u++) cur[u] = nxt[u];
             }
+            // the accumulators are drained: hand them back to the leader's MMA thread
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(acc_empty_bar(slot), 0));
         }
     }
 

@@ -220,13 +220,18 @@ umma_vm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                 if (c * 32 < n_inst) {  // warp-uniform
                     float v[32];
                     tmem_ld32(taddr + c * 32, v);
+                    // all 32 reductions are issued before any result is used, so that their
+                    // latencies overlap instead of adding up
+                    uint32_t u[32], m[32];
+#pragma unroll
+                    for (int j = 0; j < 32; j++) u[j] = v_ok ? ordered_u32(v[j]) : 0u;
+#pragma unroll
+                    for (int j = 0; j < 32; j++) m[j] = warp_max_u32(u[j]);
 #pragma unroll
                     for (int j = 0; j < 32; j++) {
-                        const uint32_t u = v_ok ? ordered_u32(v[j]) : 0u;
-                        const uint32_t m = warp_max_u32(u);
-                        const uint32_t who = __ballot_sync(0xffffffffu, u == m);
-                        if (lane == j && m > rb_u[c]) {  // strict: an earlier (lower) entry keeps a tie
-                            rb_u[c] = m;
+                        const uint32_t who = __ballot_sync(0xffffffffu, u[j] == m[j]);
+                        if (lane == j && m[j] > rb_u[c]) {  // strict: an earlier (lower) entry keeps a tie
+                            rb_u[c] = m[j];
                             rb_i[c] = v_first + __ffs(who) - 1;
                         }
                     }

@@ -58,8 +58,13 @@ enum {
     AJ_FLAG_TIME_KERNELS = 2u, /* record CUDA events around the projection kernel (see aj_last_gemm_ms) */
     AJ_FLAG_ROW_TILES = 4u,    /* tensor-core path with 128-row tiles of h on the UMMA M axis (the earlier
                                   tiling, kept for comparison) instead of vocabulary-major tiles */
-    AJ_FLAG_ONE_SM = 8u        /* keep batches of more than 128 rows on the one-SM vocabulary-major kernel
+    AJ_FLAG_ONE_SM = 8u,       /* keep batches of more than 128 rows on the one-SM vocabulary-major kernel
                                   instead of the two-SM (CTA pair) kernel; for comparison */
+    AJ_FLAG_NO_EXTRA_ROW = 16u /* the caller does not encode the last draft token (Section 3.2, design choice 1,
+                                  second way): h_target and h_draft are [B, K, ...], target_tok and top1_val are
+                                  [B, K]; a mismatch at the last position is rejected without the classifier
+                                  (judge_p there is NaN); when all K tokens pass, next_tok is -1 (there is no
+                                  row to predict a further token from) */
 };
 
 /*

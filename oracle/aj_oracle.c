@@ -27,6 +27,12 @@
  * tau <= 0 never forgives and tau >= 1 always forgives; feature order is [draft ; target];
  * the comparison p < tau is taken on p rounded to fp32 (the precision the kernel decides in).
  *
+ * Variant without the extra row (Section 3.2, design choice 1, the second way to handle the
+ * last window token): only K rows of hidden states are given, so the states that encode the last
+ * draft token do not exist; a mismatch at the last position is then rejected without consulting
+ * the classifier, and when all K positions pass there is no row to predict a further token from
+ * (next_tok = -1).
+ *
  * All inputs are converted exactly to double; every sum is accumulated in double.
  *
  * parity pins: see tests/test_oracle_pins.py (library matmul special case, one-hot
@@ -152,16 +158,16 @@ static int forgiven(double p, float tau)
 }
 
 /*
- * The whole step for B sequences.
- *   h_target [B][K+1][d], h_draft [B][K+1][d_draft] (NULL iff d_draft == 0), W per w_layout,
+ * The whole step for B sequences.  R = K + 1 rows per sequence, or R = K when extra_row == 0.
+ *   h_target [B][R][d], h_draft [B][R][d_draft] (NULL iff d_draft == 0), W per w_layout,
  *   draft_tok [B][K], judge_w [d_draft + d].
  * Outputs (all caller-allocated, all required):
- *   accept_len [B], next_tok [B], target_tok [B][K+1], top1 [B][K+1], gap [B][K+1],
- *   judge_p [B][K]  (p at every mismatching position, NaN where the draft token matched).
+ *   accept_len [B], next_tok [B], target_tok [B][R], top1 [B][R], gap [B][R],
+ *   judge_p [B][K]  (p at every mismatching position whose features exist, NaN elsewhere).
  */
 int ajo_verify(const void *h_target, const void *h_draft, const void *W,
                const int32_t *draft_tok, const float *judge_w, float judge_b, float tau,
-               int dtype, int w_layout, int B, int K, int d, int d_draft, int V,
+               int dtype, int w_layout, int B, int K, int d, int d_draft, int V, int extra_row,
                int32_t *accept_len, int32_t *next_tok, int32_t *target_tok,
                double *top1, double *gap, double *judge_p)
 {
@@ -169,7 +175,7 @@ int ajo_verify(const void *h_target, const void *h_draft, const void *W,
         d_draft < 0 || (d_draft > 0 && !h_draft))
         return 1;
     size_t esz = (dtype == AJO_BF16) ? 2 : 4;
-    int R = K + 1;
+    int R = extra_row ? K + 1 : K;
     double *logits = (double *)malloc((size_t)R * V * sizeof(double));
     if (!logits) return 2;
 
@@ -186,7 +192,7 @@ int ajo_verify(const void *h_target, const void *h_draft, const void *W,
         /* p at every mismatch (the device evaluates all mismatches, so all are comparable) */
         for (int i = 0; i < K; i++) {
             double p = NAN;
-            if (draft_tok[(size_t)b * K + i] != y[i])
+            if (draft_tok[(size_t)b * K + i] != y[i] && i + 1 < R) /* row i+1 encodes draft token i */
                 p = ajo_judge_p(hdr ? hdr + (size_t)(i + 1) * d_draft * esz : NULL,
                                 ht + (size_t)(i + 1) * d * esz, dtype, judge_w, judge_b, d_draft, d);
             judge_p[(size_t)b * K + i] = p;
@@ -195,11 +201,14 @@ int ajo_verify(const void *h_target, const void *h_draft, const void *W,
         /* walk the window in order; stop at the first mismatch the judge does not forgive */
         int n = 0;
         while (n < K) {
-            if (draft_tok[(size_t)b * K + n] != y[n] && !forgiven(judge_p[(size_t)b * K + n], tau)) break;
+            if (draft_tok[(size_t)b * K + n] != y[n]) {
+                if (n + 1 >= R) break; /* no features for the last token: rejected without the classifier */
+                if (!forgiven(judge_p[(size_t)b * K + n], tau)) break;
+            }
             n++;
         }
         accept_len[b] = n;
-        next_tok[b] = y[n];
+        next_tok[b] = n < R ? y[n] : -1;
     }
     free(logits);
     return 0;

@@ -64,7 +64,7 @@ def _lib():
         L.ajo_argmax.restype = None
         L.ajo_judge_p.argtypes = [vp, vp, ci, fp, cf, ci, ci]
         L.ajo_judge_p.restype = ctypes.c_double
-        L.ajo_verify.argtypes = [vp, vp, vp, ip, fp, cf, cf, ci, ci, ci, ci, ci, ci, ci, ip, ip, ip, dp, dp, dp]
+        L.ajo_verify.argtypes = [vp, vp, vp, ip, fp, cf, cf, ci, ci, ci, ci, ci, ci, ci, ci, ip, ip, ip, dp, dp, dp]
         L.ajo_verify.restype = ci
         _LIB = L
     return _LIB
@@ -130,15 +130,18 @@ class OracleResult:
     judge_p: np.ndarray  # [B, K] float64, NaN where the draft token matched
 
 
-def verify(h_target, h_draft, W, draft_tok, judge_w, judge_b, tau, dtype: int, w_layout: int = 0) -> OracleResult:
-    """The whole verify-and-judge step for B sequences (see aj_oracle.c for the definition)."""
+def verify(h_target, h_draft, W, draft_tok, judge_w, judge_b, tau, dtype: int, w_layout: int = 0,
+           extra_row: bool = True) -> OracleResult:
+    """The whole verify-and-judge step for B sequences (see aj_oracle.c for the definition).
+
+    extra_row=False: the hidden states have K rows, not K + 1 (the last draft token is not encoded)."""
     ht = _check_storage(h_target, dtype, "h_target")
     hd = None if h_draft is None else _check_storage(h_draft, dtype, "h_draft")
     W = _check_storage(W, dtype, "W")
     tok = np.ascontiguousarray(draft_tok, dtype=np.int32)
     w = np.ascontiguousarray(judge_w, dtype=np.float32)
     B, R, d = ht.shape
-    K = R - 1
+    K = R - 1 if extra_row else R
     dd = 0 if hd is None else hd.shape[2]
     V = W.shape[0] if w_layout == 0 else W.shape[1]
     assert tok.shape == (B, K) and w.shape == (d + dd,)
@@ -149,7 +152,7 @@ def verify(h_target, h_draft, W, draft_tok, judge_w, judge_b, tau, dtype: int, w
     )
     rc = _lib().ajo_verify(
         _ptr(ht), _ptr(hd), _ptr(W), _ptr(tok), _ptr(w), float(judge_b), float(tau), dtype, w_layout,
-        B, K, d, dd, V, _ptr(res.accept_len), _ptr(res.next_tok), _ptr(res.target_tok),
+        B, K, d, dd, V, 1 if extra_row else 0, _ptr(res.accept_len), _ptr(res.next_tok), _ptr(res.target_tok),
         _ptr(res.top1), _ptr(res.gap), _ptr(res.judge_p),
     )
     if rc:

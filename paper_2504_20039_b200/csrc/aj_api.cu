@@ -129,6 +129,10 @@ aj_status check_call(aj_handle h, const void *h_target, const void *h_draft, con
     return AJ_OK;
 }
 
+// rows of hidden states per sequence: the last accepted token and the K draft tokens, or without
+// the last draft token when the caller does not encode it
+int rows_per_seq(aj_handle h, int K) { return (h->flags & AJ_FLAG_NO_EXTRA_ROW) ? K : K + 1; }
+
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
 }  // namespace
@@ -157,7 +161,8 @@ aj_status aj_create(aj_handle *out, int device, int max_B, int max_K, int d, int
     if (device < 0 || max_B < 1 || max_K < 1 || max_K > 1024 || d < 1 || d_draft < 0 || V < 1) return AJ_ERR_INVALID_ARG;
     if (dtype != AJ_BF16 && dtype != AJ_F32) return AJ_ERR_INVALID_ARG;
     if (layout != AJ_W_VD && layout != AJ_W_DV) return AJ_ERR_INVALID_ARG;
-    if (flags & ~(AJ_FLAG_FORCE_SIMT | AJ_FLAG_TIME_KERNELS | AJ_FLAG_ROW_TILES | AJ_FLAG_ONE_SM)) return AJ_ERR_INVALID_ARG;
+    if (flags & ~(AJ_FLAG_FORCE_SIMT | AJ_FLAG_TIME_KERNELS | AJ_FLAG_ROW_TILES | AJ_FLAG_ONE_SM | AJ_FLAG_NO_EXTRA_ROW))
+        return AJ_ERR_INVALID_ARG;
     if ((long long)max_B * (max_K + 1) > (1ll << 24)) return AJ_ERR_INVALID_ARG;
     if (dtype == AJ_BF16 && (d % 8 != 0 || d_draft % 8 != 0)) return AJ_ERR_UNSUPPORTED;
 
@@ -239,7 +244,7 @@ aj_status aj_destroy(aj_handle h) {
 
 // Enqueue the projection + argmax kernel of one cycle (and, on a sharded handle, its exchange).
 static aj_status enqueue_project(aj_handle h, const void *h_target, const void *W_lm, int B, int K, cudaStream_t stream) {
-    const int M = B * (K + 1);
+    const int M = B * rows_per_seq(h, K);
     const int d = h->d;
     const int V = h->world ? h->v_count : h->V;  // vocabulary entries this GPU projects
     h->last_launches = 0;
@@ -361,6 +366,7 @@ static aj_status enqueue_finish(aj_handle h, const void *h_target, const void *h
     j.d = h->d;
     j.d_draft = h->d_draft;
     j.dtype = h->dtype;
+    j.no_extra_row = (h->flags & AJ_FLAG_NO_EXTRA_ROW) ? 1 : 0;
     j.accept_len = accept_len;
     j.next_tok = next_tok;
     j.target_tok = target_tok;
@@ -399,7 +405,7 @@ aj_status aj_verify_host(aj_handle h, const void *h_target_host, const void *h_d
     DeviceGuard guard(h->device);
     if (!guard.ok()) return AJ_ERR_CUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    const size_t M = (size_t)B * (K + 1), esz = elem_size(h->dtype);
+    const size_t M = (size_t)B * rows_per_seq(h, K), esz = elem_size(h->dtype);
     bool ok = cudaMemcpyAsync(h->st_ht, h_target_host, M * d * esz, cudaMemcpyHostToDevice, stream) == cudaSuccess &&
               (h->d_draft == 0 ||
                cudaMemcpyAsync(h->st_hd, h_draft_host, M * h->d_draft * esz, cudaMemcpyHostToDevice, stream) == cudaSuccess) &&

@@ -159,6 +159,7 @@ struct JudgeArgs {
     const float *judge_w;            // [d_draft + d]
     float judge_b, tau;
     int B, K, d, d_draft, dtype;
+    int no_extra_row = 0;            // 1: K rows per sequence instead of K + 1
     int32_t *accept_len, *next_tok, *target_tok;
     float *top1_val, *judge_p;
 };

@@ -100,7 +100,7 @@ __device__ inline float scalar_dot(const void *x, const float *w, int n, int dty
 
 __global__ void __maxnreg__(96) judge_scan_kernel(JudgeArgs a) {
     extern __shared__ int smem[];
-    const int K = a.K, R = a.K + 1;
+    const int K = a.K, R = a.K + 1 - a.no_extra_row;  // without the extra row the last draft token is not encoded
     int *y_s = smem;                                          // [K+1]
     int *rej_s = smem + R;                                    // [K]: 1 = mismatch not forgiven
     int *mis_s = rej_s + K;                                   // [K]
@@ -125,7 +125,7 @@ __global__ void __maxnreg__(96) judge_scan_kernel(JudgeArgs a) {
         if ((long long)gridDim.x * K <= 256) {
             const size_t lt = (row_bytes_t + 127) / 128, ld = a.h_draft ? (row_bytes_d + 127) / 128 : 0;
             const size_t per_row = lt + ld;
-            for (size_t l = threadIdx.x; l < per_row * K; l += blockDim.x) {
+            for (size_t l = threadIdx.x; l < per_row * (R - 1); l += blockDim.x) {
                 const size_t row = (size_t)b * R + 1 + l / per_row, o = l % per_row;
                 const char *src = o < lt ? reinterpret_cast<const char *>(a.h_target) + row * row_bytes_t + o * 128
                                          : reinterpret_cast<const char *>(a.h_draft) + row * row_bytes_d + (o - lt) * 128;
@@ -190,7 +190,7 @@ __global__ void __maxnreg__(96) judge_scan_kernel(JudgeArgs a) {
     const int chunks = (a.d_draft + a.d) / epc;
     for (int it = warp; it < K * SEGS; it += nwarps) {
         const int i = it / SEGS, seg = it % SEGS;
-        if (!mis_s[i]) continue;                        // the judge is consulted at mismatches only
+        if (!mis_s[i] || i + 1 >= R) continue;          // at mismatches only, and only where the features exist
         const size_t row = (size_t)b * R + (i + 1);     // the hidden states that encode draft token i
         const char *xd = a.h_draft ? reinterpret_cast<const char *>(a.h_draft) + row * row_bytes_d : nullptr;
         const char *xt = reinterpret_cast<const char *>(a.h_target) + row * row_bytes_t;
@@ -213,7 +213,9 @@ __global__ void __maxnreg__(96) judge_scan_kernel(JudgeArgs a) {
     for (int i = threadIdx.x; i < K; i += blockDim.x) {
         float p = __int_as_float(0x7fc00000);  // NaN where the judge is not consulted
         int rej = 0;
-        if (mis_s[i]) {
+        if (mis_s[i] && i + 1 >= R) {
+            rej = 1;  // the states that encode the last draft token were not computed: rejected unjudged
+        } else if (mis_s[i]) {
             float z = a.judge_b;
 #pragma unroll
             for (int seg = 0; seg < SEGS; seg++) z += part_s[i * SEGS + seg];
@@ -238,7 +240,7 @@ __global__ void __maxnreg__(96) judge_scan_kernel(JudgeArgs a) {
         }
         if (lane == 0) {
             a.accept_len[b] = first;
-            a.next_tok[b] = y_s[first];
+            a.next_tok[b] = first < R ? y_s[first] : -1;  // all K accepted and no row K: nothing to predict from
         }
     }
 }

@@ -50,6 +50,7 @@ class DeviceCase:
         self.ht = to_device(ht, cfg.dtype)
         self.hd = to_device(hd, cfg.dtype)
         self.w = to_device(w, gen.F32)
+        self.extra_row = not (flags & aj.AJ_FLAG_NO_EXTRA_ROW)  # K + 1 rows per sequence, or K
         self.handle = aj.Handle(0, max_B or cfg.B, max_K or cfg.K, cfg.d, cfg.d_draft, cfg.V, cfg.dtype, layout, flags)
 
     def run(self, tok: np.ndarray, tau: float, judge_b: float | None = None, B=None, K=None, seqs=slice(None), fill=None) -> GpuResult:
@@ -65,8 +66,9 @@ class DeviceCase:
         fill_i = -7 if fill is None else fill
         acc = torch.full((B,), fill_i, **i32)
         nxt = torch.full((B,), fill_i, **i32)
-        tt = torch.full((B, K + 1), fill_i, **i32)
-        top1 = torch.full((B, K + 1), 12345.0, **f32)
+        R = K + 1 if self.extra_row else K
+        tt = torch.full((B, R), fill_i, **i32)
+        top1 = torch.full((B, R), 12345.0, **f32)
         jp = torch.full((B, K), 12345.0, **f32)
         stream = torch.cuda.current_stream().cuda_stream
         self.handle.verify(ht.contiguous(), None if hd is None else hd.contiguous(), self.W, tok_d, self.w,
@@ -104,8 +106,8 @@ def check_parity(orc_res, gpu: GpuResult, tok: np.ndarray, tau: float, seqs=None
     rep = ParityReport()
     idx = np.arange(gpu.accept_len.shape[0]) if seqs is None else np.asarray(seqs)
     B, R = orc_res.target_tok.shape
-    K = R - 1
     tok = np.asarray(tok)
+    K = tok.shape[1]  # R is K + 1, or K when the last draft token is not encoded
     for r, b in enumerate(idx):
         y_o, y_g = orc_res.target_tok[r], gpu.target_tok[b]
         close = orc_res.gap[r] <= GAP_EXEMPT
@@ -137,7 +139,7 @@ def check_parity(orc_res, gpu: GpuResult, tok: np.ndarray, tau: float, seqs=None
             assert gpu.next_tok[b] == orc_res.next_tok[r], f"seq {b}: next_tok {gpu.next_tok[b]} != {orc_res.next_tok[r]}"
         # what must hold regardless: the device is consistent with its own tokens
         assert 0 <= gpu.accept_len[b] <= K
-        assert gpu.next_tok[b] == gpu.target_tok[b, gpu.accept_len[b]]
+        assert gpu.next_tok[b] == (gpu.target_tok[b, gpu.accept_len[b]] if gpu.accept_len[b] < R else -1)
     return rep
 
 

@@ -120,6 +120,36 @@ def test_bf16_dv_layout_runs_on_cuda_cores():
     _full_parity(cfg, (0.5,), layout=1, expect_path="simt")
 
 
+@pytest.mark.parametrize("shape", [("ne_small", 3, 9, 256, 128, 3000), ("ne_pair", 6, 50, 128, 64, 1500), ("ne_k1", 5, 1, 64, 0, 300)],
+                         ids=lambda s: s[0])
+def test_without_the_extra_row(shape):
+    """AJ_FLAG_NO_EXTRA_ROW: K rows per sequence, a last-position mismatch is rejected without the judge."""
+    import paper_2504_20039_b200 as aj
+
+    orc = _oracle()
+    name, B, K, d, dd, V = shape
+    cfg = gen.Config(name, B=B, K=K, d=d, d_draft=dd, V=V, sigma_W=0.2, sigma_w=0.05, match_lo=0.6, match_hi=0.95, seed=13)
+    W, ht, hd, w = _host_case(cfg)
+    ht = ht[:, :K].copy()
+    hd = None if hd is None else hd[:, :K].copy()
+    y = np.stack([[orc.argmax(r)[0] for r in orc.logits(ht[b], W, cfg.dtype)] for b in range(B)])  # [B, K]
+    tok = gen.plant_draft_tokens(cfg, np.concatenate([y, y[:, :1]], axis=1))
+    tok[0, K - 1] = (y[0, K - 1] + 1) % V   # a sure mismatch at the last position
+    tok[1, :] = y[1, :K]                    # and a sequence that passes everywhere
+    case = DeviceCase(cfg, W, ht, hd, w, flags=aj.AJ_FLAG_NO_EXTRA_ROW)
+    try:
+        for tau in (0.0, 0.5, 1.0):
+            o = orc.verify(ht, hd, W, tok, w, cfg.judge_b, tau, cfg.dtype, extra_row=False)
+            g = case.run(tok, tau)
+            assert g.target_tok.shape == (B, K) and g.launches == 2
+            check_parity(o, g, tok, tau)
+            assert np.isnan(g.judge_p[:, K - 1]).all()
+            assert g.accept_len[1] == K and g.next_tok[1] == -1
+            assert g.accept_len[0] <= K - 1
+    finally:
+        case.close()
+
+
 # -------------------------------------------------------------------------------- edge cases
 
 

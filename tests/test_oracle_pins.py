@@ -308,3 +308,57 @@ def test_expected_accept_len_matches_closed_form(tau):
     se = math.sqrt(var / cfg.B)
     assert abs(float(r.accept_len.mean()) - want) < 4 * se
     assert abs(float((tok == y[:, :K]).mean()) - r_match) < 4 * math.sqrt(r_match * (1 - r_match) / (cfg.B * K))
+
+
+# ---------------------------------------------------- variant: the last draft token is not encoded
+
+
+@pytest.mark.parametrize("tau", [0.0, 0.4, 1.0])
+def test_without_the_extra_row_the_last_mismatch_is_rejected_unjudged(tau):
+    """Section 3.2, design choice 1, second way: with K rows instead of K + 1 the states that encode the
+    last draft token do not exist, so a mismatch there is discarded without the classifier.  Everything
+    before the last position must be decided exactly as with the extra row."""
+    g = np.random.default_rng(101)
+    B, K, d, dd, V = 40, 5, 32, 16, 50
+    cfg = gen.Config("noextra", B=B, K=K, d=d, d_draft=dd, V=V, sigma_W=0.3, sigma_w=0.3, match_lo=0.6, match_hi=0.9, seed=77)
+    W = gen.make_W(cfg)
+    ht, hd = gen.make_hidden(cfg)
+    w = gen.make_judge(cfg)
+    y = np.stack([[orc.argmax(r)[0] for r in orc.logits(ht[b], W, cfg.dtype)] for b in range(B)])
+    tok = gen.plant_draft_tokens(cfg, y)
+    tok[:8, K - 1] = y[:8, K - 1]                    # some sequences surely match at the last position
+    tok[8:16, K - 1] = (y[8:16, K - 1] + 1) % V      # and some surely do not
+    full = orc.verify(ht, hd, W, tok, w, 0.0, tau, cfg.dtype)
+    ne = orc.verify(ht[:, :K].copy(), hd[:, :K].copy(), W, tok, w, 0.0, tau, cfg.dtype, extra_row=False)
+    assert ne.target_tok.shape == (B, K)
+    np.testing.assert_array_equal(ne.target_tok, full.target_tok[:, :K])
+    np.testing.assert_array_equal(ne.top1, full.top1[:, :K])
+    np.testing.assert_array_equal(ne.judge_p[:, : K - 1], full.judge_p[:, : K - 1])  # same rows, same values
+    assert np.isnan(ne.judge_p[:, K - 1]).all()     # never judged at the last position
+    seen = set()
+    for b in range(B):
+        last_mismatch = tok[b, K - 1] != y[b, K - 1]
+        if full.accept_len[b] < K - 1:               # stopped earlier: nothing changes
+            want_len, want_next, kind = full.accept_len[b], full.next_tok[b], "early"
+        elif last_mismatch:                          # reached the last position and it mismatches
+            want_len, want_next, kind = K - 1, y[b, K - 1], "last_rejected"
+        else:                                        # reached it and it matches: all K pass, nothing to predict from
+            want_len, want_next, kind = K, -1, "all_pass"
+        seen.add(kind)
+        assert (ne.accept_len[b], ne.next_tok[b]) == (want_len, want_next), (b, kind)
+    assert "last_rejected" in seen and "all_pass" in seen and ("early" in seen or tau >= 1.0)
+
+
+def test_without_the_extra_row_single_token_window():
+    # K = 1: one row per sequence; the only position is the last one
+    cfg = gen.Config("noextra1", B=6, K=1, d=16, d_draft=0, V=9, sigma_W=0.5, seed=5)
+    W = gen.make_W(cfg)
+    ht, _ = gen.make_hidden(cfg)
+    ht = ht[:, :1].copy()
+    w = gen.make_judge(cfg)
+    y = np.array([orc.argmax(orc.logits(ht[b], W, cfg.dtype)[0])[0] for b in range(cfg.B)])
+    tok = y.copy().reshape(-1, 1).astype(np.int32)
+    tok[::2, 0] = (tok[::2, 0] + 1) % cfg.V
+    r = orc.verify(ht, None, W, tok, w, 0.0, 1.0, cfg.dtype, extra_row=False)
+    np.testing.assert_array_equal(r.accept_len, np.where(np.arange(cfg.B) % 2 == 0, 0, 1))
+    np.testing.assert_array_equal(r.next_tok, np.where(np.arange(cfg.B) % 2 == 0, y, -1))

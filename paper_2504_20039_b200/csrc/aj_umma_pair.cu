@@ -95,6 +95,7 @@ __device__ inline Tile decode_tile(const PairSched &sc, int t) {
     return r;
 }
 
+template <bool DUAL>  // DUAL: every tile uses two accumulators that share the staged block of W
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_h,
                  int M, int V, int d, PairSched sc, int stream_w, int v_offset,
@@ -119,7 +120,7 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
     const int num_pairs = gridDim.x >> 1;
     const int num_kb = d / BK;
     const int num_tiles = sc.n_n * sc.n_v;
-    const int n_acc = sc.dual ? 2 : 1;
+    constexpr int n_acc = DUAL ? 2 : 1;
     const int stages = sc.stages;
     const uint32_t b_bytes = (uint32_t)sc.box_rows * BK * 2;       // one accumulator's rows of h staged by this CTA
     const uint32_t stage_bytes = A_BYTES + n_acc * b_bytes;         // a multiple of 1024
@@ -154,8 +155,8 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
     // Accumulator hand-over.  Single mode: the two 256-column buffers alternate from tile to tile
     // (buffer it & 1, each with its own pair of barriers).  Dual mode: every tile uses both buffers
     // as two accumulators that share the staged block of W, and one pair of barriers.
-    auto acc_slot = [&](int it) { return sc.dual ? 0 : (it & 1); };
-    auto acc_phase = [&](int it) { return (uint32_t)(sc.dual ? it : (it >> 1)) & 1u; };
+    auto acc_slot = [&](int it) { return DUAL ? 0 : (it & 1); };
+    auto acc_phase = [&](int it) { return (uint32_t)(DUAL ? it : (it >> 1)) & 1u; };
 
     if (warp == 0) {
         if (lane == 0) {
@@ -285,7 +286,7 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
                     if (c * 32 < n_inst) {  // warp-uniform
                         const float thr = cur[u];
                         float v[32];
-                        tmem_ld32(tbase + (uint32_t)((sc.dual ? a : slot) * BN + c * 32), v);
+                        tmem_ld32(tbase + (uint32_t)((DUAL ? a : slot) * BN + c * 32), v);
                         bool hit = false;
 #pragma unroll
                         for (int j = 0; j < 32; j++) hit |= v[j] >= __shfl_sync(0xffffffffu, thr, j);
@@ -342,7 +343,9 @@ int g_max_pairs = 0;
 }  // namespace
 
 cudaError_t umma_pair_prepare(int num_sms) {
-    cudaError_t e = cudaFuncSetAttribute(umma_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    cudaError_t e = cudaFuncSetAttribute(umma_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(umma_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e != cudaSuccess) return e;
     // how many CTA pairs can be resident at once (pairs need both SMs of a pair free)
     cudaLaunchConfig_t cfg = {};
@@ -357,7 +360,7 @@ cudaError_t umma_pair_prepare(int num_sms) {
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     int clusters = 0;
-    e = cudaOccupancyMaxActiveClusters(&clusters, umma_pair_kernel, &cfg);
+    e = cudaOccupancyMaxActiveClusters(&clusters, umma_pair_kernel<false>, &cfg);
     if (e != cudaSuccess) return e;
     if (clusters < 1) return cudaErrorInvalidConfiguration;
     g_max_pairs = clusters < num_sms / 2 ? clusters : num_sms / 2;
@@ -410,8 +413,11 @@ cudaError_t launch_umma_pair(const GemmArgs &a, const UmmaPlan &p, cudaStream_t 
     attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    return cudaLaunchKernelEx(&cfg, umma_pair_kernel, p.tmap_w, p.tmap_h, a.M, a.V, a.d, sc, stream_w, a.v_offset, a.keys,
-                              a.status, a.pub);
+    if (sc.dual)
+        return cudaLaunchKernelEx(&cfg, umma_pair_kernel<true>, p.tmap_w, p.tmap_h, a.M, a.V, a.d, sc, stream_w, a.v_offset,
+                                  a.keys, a.status, a.pub);
+    return cudaLaunchKernelEx(&cfg, umma_pair_kernel<false>, p.tmap_w, p.tmap_h, a.M, a.V, a.d, sc, stream_w, a.v_offset,
+                              a.keys, a.status, a.pub);
 }
 
 }  // namespace aj

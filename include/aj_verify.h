@@ -153,9 +153,9 @@ int aj_last_launch_count(aj_handle h);
  *   [4] rows of h_target each SM of a pair stages per 64-column block and accumulator
  *   [5] groups the row tiles are walked in (each group against the whole vocabulary, so that a
  *       group's rows of h_target stay in L2)    [6],[7] group g holds out[6] + (g < out[7]) row tiles
- *   [8] 1 if each tile uses two accumulators that share the staged block of W_lm (257..512 rows: one
- *       pass over W_lm for all rows, a tile then holds up to 512 rows), else 0 (tiles of at most 256
- *       rows on one accumulator, double-buffered)      [9] depth of the shared-memory ring
+ *   [8] 1 if each tile uses two accumulators that share the staged block of W_lm (a tile then holds up
+ *       to 512 rows; chosen for 257..448 rows, and from 1024 rows on when d >= 8192), else 0 (tiles of
+ *       at most 256 rows on one accumulator, double-buffered)      [9] depth of the shared-memory ring
  * Errors: AJ_ERR_INVALID_ARG.
  */
 aj_status aj_pair_schedule(int M, int d, int V, int32_t out[10]);

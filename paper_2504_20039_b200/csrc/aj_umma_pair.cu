@@ -372,10 +372,14 @@ int umma_pair_max_pairs() { return g_max_pairs; }
 PairSched pair_schedule(int M, int V, int d) {
     PairSched sc;
     const int units = (M + 15) / 16;  // rows in units of 16 (the UMMA N granule)
-    // Between 257 and 512 rows one tile takes all rows on two accumulators that share each staged
-    // block of W (no second pass over W, no accumulator double-buffering); otherwise the fewest
-    // tiles of at most 256 rows, one accumulator each, double-buffered.
-    sc.dual = (units > 16 && units <= 32) ? 1 : 0;
+    // Two accumulators per tile (up to 512 rows share each staged block of W; 25 % less operand
+    // traffic, but the epilogue is no longer hidden under the next tile's MMAs) or one (at most 256
+    // rows, double-buffered)?  Measured on the same GPU: two win from 257 to about 450 rows, where
+    // they save a second pass over W (-10 % at 264 and 400 rows, +4 % at 512), and for deep
+    // contractions with many rows, where the exposed epilogue is a small share of a tile and the
+    // operand traffic weighs most (d = 8192: -1.5 % at 1056 rows, -6 % at 2080, -9 % at 4160; but
+    // +1.5 % at 528, and +3 ... +8 % for every batch at d = 4096).
+    sc.dual = (units > 16 && (units <= 28 || (d >= 8192 && units >= 64))) ? 1 : 0;
     const int cap = sc.dual ? 32 : 16;
     sc.n_n = (units + cap - 1) / cap;
     sc.u_base = units / sc.n_n;

@@ -80,7 +80,7 @@ def test_two_sm_schedule_covers_every_row_once(built):
         s = aj.pair_schedule(M, d, 128256)
         assert s["n_v"] == 501
         units = (M + 15) // 16
-        assert s["dual"] == (1 if 256 < M <= 512 else 0)
+        assert s["dual"] == (1 if (256 < M <= 448 or (d >= 8192 and M > 1008)) else 0)
         cap = 32 if s["dual"] else 16                         # units per tile: two accumulators or one
         sizes = [s["u_base"] + (i < s["u_rem"]) for i in range(s["n_n"])]
         assert sum(sizes) == units and max(sizes) <= cap and min(sizes) >= (2 if s["dual"] else 1)

@@ -94,9 +94,11 @@ SHAPES = [
     ("window_above_64", 2, 100, 64, 0, 700),      # K > 64: several ballots; target-only features
     ("pair_ragged_rows", 9, 63, 320, 64, 3000),   # M = 576 = 2*256 + 64: a 64-row tail tile on the two-SM kernel; V = 11*256 + 184
     ("pair_odd_tail", 3, 86, 192, 0, 1111),       # M = 261: 17 units of 16 rows on two accumulators (144 + 128), 3 k-blocks
-    ("pair_dual_full", 8, 63, 128, 64, 2000),     # M = 512: two full accumulators of 256 rows
+    ("pair_two_full_tiles", 8, 63, 128, 64, 2000),  # M = 512: two tiles of 256 rows, one accumulator each
+    ("pair_dual_448", 7, 63, 128, 64, 2000),      # M = 448: the largest batch on two accumulators (224 + 224)
     ("pair_dual_mid", 7, 56, 256, 0, 1500),       # M = 399: 25 units -> 208 + 192 rows
     ("pair_three_tiles", 11, 47, 128, 64, 1300),  # M = 528: just past the two-accumulator range, 3 tiles of 176 rows
+    ("pair_dual_deep", 16, 64, 8192, 0, 700),     # M = 1040, d = 8192: deep contraction, two accumulators per tile (3 tiles)
 ]
 
 

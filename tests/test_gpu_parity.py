@@ -341,3 +341,43 @@ def test_host_buffer_entry_point_matches_device_entry_point():
         np.testing.assert_array_equal(tt.numpy(), g.target_tok)
     finally:
         case.close()
+
+
+def test_a_cycle_captured_in_a_cuda_graph_replays_with_new_inputs():
+    """aj_verify only enqueues (two kernel launches, no allocation, no synchronisation), so a cycle can be
+    captured in a CUDA graph and replayed: the replay reads whatever the input buffers hold then."""
+    import torch
+
+    orc = _oracle()
+    cfg = gen.Config("graph", B=3, K=12, d=256, d_draft=128, V=4000, sigma_W=0.2, sigma_w=0.05, match_lo=0.5, match_hi=0.9, seed=14)
+    W, ht, hd, w = _host_case(cfg)
+    y = _oracle_y(cfg, W, ht)
+    tok = gen.plant_draft_tokens(cfg, y)
+    case = DeviceCase(cfg, W, ht, hd, w)
+    try:
+        case.run(tok, 0.5)  # warms the handle up (tensor maps cached) before the capture
+        i32 = dict(dtype=torch.int32, device="cuda")
+        tok_d = torch.zeros((cfg.B, cfg.K), **i32)
+        acc, nxt, tt = torch.zeros(cfg.B, **i32), torch.zeros(cfg.B, **i32), torch.zeros((cfg.B, cfg.K + 1), **i32)
+        graph = torch.cuda.CUDAGraph()
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            with torch.cuda.graph(graph, stream=side):
+                case.handle.verify(case.ht, case.hd, case.W, tok_d, case.w, cfg.judge_b, 0.5, cfg.B, cfg.K, acc, nxt, tt,
+                                   stream=torch.cuda.current_stream().cuda_stream)
+        torch.cuda.current_stream().wait_stream(side)
+        for trial in range(3):
+            cur = tok if trial != 1 else np.roll(tok, 1, axis=1)  # other draft tokens on the second replay
+            tok_d.copy_(torch.from_numpy(np.ascontiguousarray(cur)))
+            graph.replay()
+            torch.cuda.synchronize()
+            got = (tt.cpu().numpy(), acc.cpu().numpy(), nxt.cpu().numpy())
+            direct = case.run(cur, 0.5)  # the same cycle enqueued directly
+            np.testing.assert_array_equal(got[0], direct.target_tok)
+            np.testing.assert_array_equal(got[1], direct.accept_len)
+            np.testing.assert_array_equal(got[2], direct.next_tok)
+            check_parity(orc.verify(ht, hd, W, cur, w, cfg.judge_b, 0.5, cfg.dtype), direct, cur, 0.5)
+        assert case.handle.last_status() == case.aj.AJ_OK
+    finally:
+        case.close()

@@ -208,3 +208,43 @@ def test_sharded_argument_checks():
         assert plain.shard_project(buf, buf, 1, 1, check=False) == aj.AJ_ERR_INVALID_ARG  # not a sharded handle
     finally:
         plain.destroy()
+
+
+def test_a_rank_that_never_publishes_is_reported_as_a_timeout_and_the_gpu_stays_usable():
+    """Failure detection without a fault: in a group of two, only rank 0 runs its cycle.  Nothing ever
+    sets rank 1's flag in rank 0's exchange buffer, so rank 0's judge kernel gives up after its bounded
+    wait (2 s), records AJ_ERR_TIMEOUT in the status word and returns normally."""
+    import time
+
+    import torch
+
+    import paper_2504_20039_b200 as aj
+
+    cfg = gen.Config("absent_peer", B=2, K=4, d=128, d_draft=64, V=1024, sigma_W=0.2, sigma_w=0.05, seed=24)
+    W = gen.make_W(cfg)
+    ht, hd = gen.make_hidden(cfg)
+    w = gen.make_judge(cfg)
+    tok = gen.random_draft_tokens(cfg)
+    one = DeviceCase(cfg, W, ht, hd, w)
+    grp = ShardedGroup(cfg, one, 2)
+    try:
+        want = one.run(tok, 0.5)
+        h0 = grp.handles[0]
+        i32 = dict(dtype=torch.int32, device="cuda")
+        acc, nxt = torch.full((cfg.B,), -7, **i32), torch.full((cfg.B,), -7, **i32)
+        t0 = time.time()
+        h0.verify(one.ht, one.hd, grp.shards[0], torch.from_numpy(tok).cuda(), one.w, cfg.judge_b, 0.5, cfg.B, cfg.K, acc, nxt)
+        torch.cuda.synchronize()  # returns: the wait is bounded
+        waited = time.time() - t0
+        assert 1.5 < waited < 20.0
+        assert h0.last_status() == aj.AJ_ERR_TIMEOUT
+        assert h0.last_status() == aj.AJ_OK  # reading the status clears it
+        assert ((acc.cpu() >= 0) & (acc.cpu() <= cfg.K)).all()  # outputs are invalid but in range: nothing ran wild
+    finally:
+        grp.close()
+    try:
+        again = one.run(tok, 0.5)  # the context is intact: an ordinary cycle gives what it gave before
+        np.testing.assert_array_equal(again.target_tok, want.target_tok)
+        np.testing.assert_array_equal(again.accept_len, want.accept_len)
+    finally:
+        one.close()

@@ -76,7 +76,8 @@ enum {
  * The handle owns a small device workspace: 8 bytes per row (max_B*(max_K+1)) for the per-row
  * packed (max, argmax) keys, a status word, and staging buffers for aj_verify_host.  This is the
  * only place memory is allocated.  AJ_BF16 needs d % 8 == 0 and d_draft % 8 == 0; the tensor-core
- * path needs AJ_BF16, AJ_W_VD and d % 64 == 0, anything else runs on the CUDA-core kernel.
+ * path needs AJ_BF16 and d % 64 == 0, and for AJ_W_DV also V % 8 == 0 (rows of [d, V] must be 16-byte
+ * aligned); anything else runs on the CUDA-core kernel.
  * Errors: AJ_ERR_INVALID_ARG, AJ_ERR_UNSUPPORTED, AJ_ERR_CUDA, AJ_ERR_NOT_SM100.
  */
 aj_status aj_create(aj_handle *out, int device, int max_B, int max_K, int d, int d_draft, int V,

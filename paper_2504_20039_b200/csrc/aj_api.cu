@@ -19,7 +19,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
 struct TmapSlot {
     const void *ptr = nullptr;
     long long rows = 0;
-    int box_rows = 0;
+    int box_rows = 0;  // -1: the [d, V] map of W_lm (64 entries x 64 k-rows per box)
     unsigned long long stamp = 0;
     CUtensorMap map;
 };
@@ -97,6 +97,12 @@ const CUtensorMap *get_tmap(aj_handle h, const void *ptr, long long rows, int bo
     cuuint64_t dims[2] = {(cuuint64_t)h->d, (cuuint64_t)rows};
     cuuint64_t strides[1] = {(cuuint64_t)h->d * 2};
     cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
+    if (box_rows < 0) {  // W_lm stored [d, V]: `rows` vocabulary entries are the inner dimension
+        dims[0] = (cuuint64_t)rows;
+        dims[1] = (cuuint64_t)h->d;
+        strides[0] = (cuuint64_t)rows * 2;
+        box[1] = 64;
+    }
     cuuint32_t estr[2] = {1, 1};
     CUresult r = h->encode(&victim->map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), dims, strides, box,
                            estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -189,7 +195,10 @@ aj_status aj_create(aj_handle *out, int device, int max_B, int max_K, int d, int
     h->layout = layout;
     h->flags = flags;
     h->num_sms = prop.multiProcessorCount;
-    h->umma_ok = dtype == AJ_BF16 && layout == AJ_W_VD && d % 64 == 0 && !(flags & AJ_FLAG_FORCE_SIMT);
+    // tensor-core path: bf16, d a multiple of 64; W_lm as [V, d], or as [d, V] with a row pitch that
+    // TMA accepts (a multiple of 16 bytes) on the vocabulary-major kernels
+    h->umma_ok = dtype == AJ_BF16 && d % 64 == 0 && !(flags & AJ_FLAG_FORCE_SIMT) &&
+                 (layout == AJ_W_VD || (V % 8 == 0 && !(flags & AJ_FLAG_ROW_TILES)));
 
     const size_t max_M = (size_t)max_B * (max_K + 1);
     const size_t esz = elem_size(dtype);
@@ -289,7 +298,7 @@ static aj_status enqueue_project(aj_handle h, const void *h_target, const void *
         UmmaPlan p;
         p.bn = 256;
         const PairSched sc = pair_schedule(M, V, d);
-        const CUtensorMap *tw = get_tmap(h, W_lm, V, 128);
+        const CUtensorMap *tw = get_tmap(h, W_lm, V, h->layout == AJ_W_DV ? -1 : 128);
         const CUtensorMap *th = get_tmap(h, h_target, M, sc.box_rows);
         if (!th || !tw) return AJ_ERR_CUDA;
         p.tmap_h = *th;
@@ -302,7 +311,7 @@ static aj_status enqueue_project(aj_handle h, const void *h_target, const void *
     } else if (h->umma_ok && !(h->flags & AJ_FLAG_ROW_TILES)) {
         UmmaPlan p;
         p.bn = vm_choose_bn(M);
-        const CUtensorMap *tw = get_tmap(h, W_lm, V, 128);
+        const CUtensorMap *tw = get_tmap(h, W_lm, V, h->layout == AJ_W_DV ? -1 : 128);
         const CUtensorMap *th = get_tmap(h, h_target, M, p.bn);
         if (!th || !tw) return AJ_ERR_CUDA;
         p.tmap_h = *th;
@@ -497,6 +506,7 @@ aj_status aj_create_sharded(aj_handle *out, int device, int max_B, int max_K, in
         if (!exchange[r] || (reinterpret_cast<uintptr_t>(exchange[r]) & 255)) return AJ_ERR_INVALID_ARG;
     if (flags & AJ_FLAG_ROW_TILES) return AJ_ERR_UNSUPPORTED;
     aj_handle h = nullptr;
+    if (layout == AJ_W_DV && v_count % 8 != 0) flags |= AJ_FLAG_FORCE_SIMT;  // the shard's row pitch is not TMA-loadable
     aj_status st = aj_create(&h, device, max_B, max_K, d, d_draft, V, dtype, layout, flags);
     if (st != AJ_OK) return st;
     h->world = world;

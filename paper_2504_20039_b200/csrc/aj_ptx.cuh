@@ -106,6 +106,22 @@ __device__ inline unsigned long long smem_desc_sw128(uint32_t addr) {
     return d;
 }
 
+// Shared-memory matrix descriptor for an A operand stored MN-major (W_lm kept as [d, V]: vocabulary
+// entries contiguous): the tile is two blocks of 64 entries (128 bytes per k-row, 128-byte swizzle),
+// each block 64 k-rows = 8 groups of 8 rows, 1024 bytes per group; the blocks are 8192 bytes apart.
+// One MMA (16 k-rows) spans two groups, so the k-step advances the start address by 2048 bytes.
+__device__ inline unsigned long long smem_desc_sw128_mn(uint32_t addr) {
+    unsigned long long d = 0;
+    d |= (unsigned long long)((addr & 0x3FFFF) >> 4);  // start address, 16-byte units
+    d |= (unsigned long long)(8192 >> 4) << 16;        // leading byte offset: next block of 64 entries
+    d |= (unsigned long long)(1024 >> 4) << 32;        // stride byte offset: next group of 8 k-rows
+    d |= (unsigned long long)1 << 46;                  // descriptor version for sm_100
+    d |= (unsigned long long)2 << 61;                  // 128-byte swizzle
+    return d;
+}
+constexpr unsigned long long MN_KSTEP = 2048 >> 4;     // descriptor increment per 16 k-rows
+constexpr uint32_t IDESC_A_MN_MAJOR = 1u << 15;       // instruction descriptor: A operand is MN-major
+
 // Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, UMMA shape m x n.
 __host__ __device__ constexpr uint32_t instr_desc(int m, int n) {
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);

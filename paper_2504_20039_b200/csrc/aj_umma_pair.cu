@@ -98,7 +98,7 @@ __device__ inline Tile decode_tile(const PairSched &sc, int t) {
 template <bool DUAL>  // DUAL: every tile uses two accumulators that share the staged block of W
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_h,
-                 int M, int V, int d, PairSched sc, int stream_w, int v_offset,
+                 int M, int V, int d, PairSched sc, int stream_w, int w_dv, int v_offset,
                  unsigned long long *__restrict__ keys, int *__restrict__ status, const Publish pub) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -180,7 +180,12 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
                     const uint32_t leader_full = map_to_cta(full_bar(s), 0);
                     if (rank == 0) mbar_expect_tx(full_bar(s), stage_tx);
                     const uint32_t a_dst = base + s * stage_bytes;
-                    tma_load_2d_pair(a_dst, &tmap_w, kb * BK, w_row, leader_full, pol_w);
+                    if (w_dv) {  // W stored [d, V]: two boxes of 64 entries x 64 k-rows
+                        tma_load_2d_pair(a_dst, &tmap_w, w_row, kb * BK, leader_full, pol_w);
+                        tma_load_2d_pair(a_dst + A_BYTES / 2, &tmap_w, w_row + 64, kb * BK, leader_full, pol_w);
+                    } else {
+                        tma_load_2d_pair(a_dst, &tmap_w, kb * BK, w_row, leader_full, pol_w);
+                    }
                     tma_load_2d_pair(a_dst + A_BYTES, &tmap_h, kb * BK, h_row0, leader_full, pol_h);
                     if (n_acc == 2) tma_load_2d_pair(a_dst + A_BYTES + b_bytes, &tmap_h, kb * BK, h_row1, leader_full, pol_h);
                     if (++s == stages) {
@@ -199,8 +204,9 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
             int it = 0;
             for (int t = pair; ok && t < num_tiles; t += num_pairs, ++it) {
                 const Tile tl = decode_tile(sc, t);
-                const uint32_t idesc0 = instr_desc(BV, tl.n_inst[0]);
-                const uint32_t idesc1 = instr_desc(BV, tl.n_inst[1]);
+                const uint32_t a_major = w_dv ? IDESC_A_MN_MAJOR : 0u;
+                const uint32_t idesc0 = instr_desc(BV, tl.n_inst[0]) | a_major;
+                const uint32_t idesc1 = instr_desc(BV, tl.n_inst[1]) | a_major;
                 const int slot = acc_slot(it);
                 if (!mbar_wait(acc_empty_bar(slot), acc_phase(it) ^ 1u, abort_flag)) {
                     give_up();
@@ -217,16 +223,17 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
                     }
                     tc_fence_after();
                     const uint32_t a_addr = base + s * stage_bytes;
-                    const unsigned long long adesc = smem_desc_sw128(a_addr);
+                    const unsigned long long adesc = w_dv ? smem_desc_sw128_mn(a_addr) : smem_desc_sw128(a_addr);
+                    const unsigned long long a_step = w_dv ? MN_KSTEP : 2ull;
                     const unsigned long long bdesc0 = smem_desc_sw128(a_addr + A_BYTES);
 #pragma unroll
                     for (int k = 0; k < BK / UMMA_K; k++)
-                        umma_bf16_pair(d_tmem0, adesc + 2ull * k, bdesc0 + 2ull * k, idesc0, (uint32_t)((kb | k) != 0));
+                        umma_bf16_pair(d_tmem0, adesc + a_step * k, bdesc0 + 2ull * k, idesc0, (uint32_t)((kb | k) != 0));
                     if (n_acc == 2) {
                         const unsigned long long bdesc1 = smem_desc_sw128(a_addr + A_BYTES + b_bytes);
 #pragma unroll
                         for (int k = 0; k < BK / UMMA_K; k++)
-                            umma_bf16_pair(d_tmem1, adesc + 2ull * k, bdesc1 + 2ull * k, idesc1, (uint32_t)((kb | k) != 0));
+                            umma_bf16_pair(d_tmem1, adesc + a_step * k, bdesc1 + 2ull * k, idesc1, (uint32_t)((kb | k) != 0));
                     }
                     umma_commit_pair(empty_bar(s));  // frees the stage in both CTAs
                     if (++s == stages) {
@@ -418,9 +425,9 @@ cudaError_t launch_umma_pair(const GemmArgs &a, const UmmaPlan &p, cudaStream_t 
     cfg.attrs = attr;
     cfg.numAttrs = 2;
     if (sc.dual)
-        return cudaLaunchKernelEx(&cfg, umma_pair_kernel<true>, p.tmap_w, p.tmap_h, a.M, a.V, a.d, sc, stream_w, a.v_offset,
+        return cudaLaunchKernelEx(&cfg, umma_pair_kernel<true>, p.tmap_w, p.tmap_h, a.M, a.V, a.d, sc, stream_w, a.w_layout, a.v_offset,
                                   a.keys, a.status, a.pub);
-    return cudaLaunchKernelEx(&cfg, umma_pair_kernel<false>, p.tmap_w, p.tmap_h, a.M, a.V, a.d, sc, stream_w, a.v_offset,
+    return cudaLaunchKernelEx(&cfg, umma_pair_kernel<false>, p.tmap_w, p.tmap_h, a.M, a.V, a.d, sc, stream_w, a.w_layout, a.v_offset,
                               a.keys, a.status, a.pub);
 }
 

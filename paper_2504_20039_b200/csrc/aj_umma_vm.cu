@@ -63,7 +63,7 @@ __device__ inline uint32_t warp_max_u32(uint32_t x) {
 template <int BN>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 umma_vm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_h,
-               int M, int V, int d, int n_n, int n_v, int stream_w, int v_offset,
+               int M, int V, int d, int n_n, int n_v, int stream_w, int w_dv, int v_offset,
                unsigned long long *__restrict__ keys, int *__restrict__ status, const Publish pub) {
     using C = VCfg<BN>;
     constexpr int STAGES = C::STAGES;
@@ -131,7 +131,12 @@ umma_vm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                     }
                     mbar_expect_tx(full_bar(s), C::STAGE_BYTES);
                     const uint32_t a_dst = base + s * C::STAGE_BYTES;
-                    tma_load_2d(a_dst, &tmap_w, kb * BK, v_tile * BV, full_bar(s), pol_w);
+                    if (w_dv) {  // W stored [d, V]: two boxes of 64 entries x 64 k-rows
+                        tma_load_2d(a_dst, &tmap_w, v_tile * BV, kb * BK, full_bar(s), pol_w);
+                        tma_load_2d(a_dst + A_BYTES / 2, &tmap_w, v_tile * BV + 64, kb * BK, full_bar(s), pol_w);
+                    } else {
+                        tma_load_2d(a_dst, &tmap_w, kb * BK, v_tile * BV, full_bar(s), pol_w);
+                    }
                     tma_load_2d(a_dst + A_BYTES, &tmap_h, kb * BK, n_tile * BN, full_bar(s), pol_h);
                     if (++s == STAGES) {
                         s = 0;
@@ -151,7 +156,7 @@ umma_vm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                 const int n_tile = t % n_n;
                 const int rows_valid = min(BN, M - n_tile * BN);
                 const int n_inst = max(16, (rows_valid + 15) & ~15);  // UMMA N: a multiple of 16
-                const uint32_t idesc = instr_desc(BV, n_inst);
+                const uint32_t idesc = instr_desc(BV, n_inst) | (w_dv ? IDESC_A_MN_MAJOR : 0u);
                 const int ab = it & 1;
                 const uint32_t aph = (uint32_t)(it >> 1) & 1u;
                 if (!mbar_wait(acc_empty_bar(ab), aph ^ 1u, abort_flag)) {
@@ -168,11 +173,12 @@ umma_vm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                     }
                     tc_fence_after();
                     const uint32_t a_addr = base + s * C::STAGE_BYTES;
-                    const unsigned long long adesc = smem_desc_sw128(a_addr);
+                    const unsigned long long adesc = w_dv ? smem_desc_sw128_mn(a_addr) : smem_desc_sw128(a_addr);
+                    const unsigned long long a_step = w_dv ? MN_KSTEP : 2ull;
                     const unsigned long long bdesc = smem_desc_sw128(a_addr + A_BYTES);
 #pragma unroll
                     for (int k = 0; k < BK / UMMA_K; k++)
-                        umma_bf16(d_tmem, adesc + 2ull * k, bdesc + 2ull * k, idesc, (uint32_t)((kb | k) != 0));
+                        umma_bf16(d_tmem, adesc + a_step * k, bdesc + 2ull * k, idesc, (uint32_t)((kb | k) != 0));
                     umma_commit(empty_bar(s));  // the stage is free once these MMAs have read it
                     if (++s == STAGES) {
                         s = 0;
@@ -276,7 +282,7 @@ cudaError_t launch_vm(const GemmArgs &a, const UmmaPlan &p, cudaStream_t stream)
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, umma_vm_kernel<BN>, p.tmap_w, p.tmap_h, a.M, a.V, a.d, n_n, n_v, stream_w, a.v_offset,
+    return cudaLaunchKernelEx(&cfg, umma_vm_kernel<BN>, p.tmap_w, p.tmap_h, a.M, a.V, a.d, n_n, n_v, stream_w, a.w_layout, a.v_offset,
                               a.keys, a.status, a.pub);
 }
 

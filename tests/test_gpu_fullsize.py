@@ -94,3 +94,25 @@ def test_c5_sweep_points_on_the_8b_shape():
 def test_c4_70b_sampled_sequences_tau_sweep():
     reps = _run_workload(gen.C4, gen.C4_TAUS, 4, "umma_pair_256x256")
     assert len(reps) == 9 and all(r.seqs >= 4 for r in reps)
+
+
+def test_c2_with_the_lm_head_stored_d_by_v_gives_the_same_bits():
+    """The [d, V] layout of W_lm (tensor-core path, MN-major operand) against the [V, d] layout, which the
+    tests above check against the oracle: same tokens, same winning logits, at the full vocabulary."""
+    cfg = gen.C2
+    Wh, Wd = _W(cfg)
+    ht, hd = gen.make_hidden(cfg)
+    w = gen.make_judge(cfg)
+    tok = gen.random_draft_tokens(cfg)
+    a = DeviceCase(cfg, Wd, ht, hd, w, layout=0)
+    b = DeviceCase(cfg, Wd.t().contiguous(), ht, hd, w, layout=1)
+    try:
+        ra, rb = a.run(tok, 0.5), b.run(tok, 0.5)
+        assert ra.path == rb.path == "umma_vm_128x32"
+        np.testing.assert_array_equal(ra.target_tok, rb.target_tok)
+        np.testing.assert_array_equal(ra.top1, rb.top1)
+        np.testing.assert_array_equal(ra.accept_len, rb.accept_len)
+        np.testing.assert_array_equal(ra.next_tok, rb.next_tok)
+    finally:
+        a.close()
+        b.close()

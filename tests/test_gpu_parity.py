@@ -117,7 +117,33 @@ def test_fp32_storage_and_both_layouts(layout):
     _full_parity(cfg, (0.0, 0.5, 1.0), layout=layout, expect_path="simt")
 
 
+@pytest.mark.parametrize("shape", [("dv_one_sm", 1, 16, 256, 128, 3000, "umma_vm_128x32"),
+                                   ("dv_one_sm_wide", 6, 20, 192, 64, 1000, "umma_vm_128x128"),
+                                   ("dv_pair_dual", 5, 60, 256, 128, 5000, "umma_pair_256x256"),
+                                   ("dv_pair_single", 9, 63, 128, 64, 2000, "umma_pair_256x256")], ids=lambda s: s[0])
+def test_bf16_dv_layout_on_the_tensor_cores(shape):
+    """W_lm stored [d, V] (vocabulary entries contiguous) with V a multiple of 8: the tensor-core kernels
+    read it as an MN-major operand; results must equal those of the [V, d] layout bit for bit."""
+    name, B, K, d, dd, V, path = shape
+    cfg = gen.Config(name, B=B, K=K, d=d, d_draft=dd, V=V, sigma_W=0.2, sigma_w=0.05, match_lo=0.5, match_hi=0.95, seed=15)
+    reps = _full_parity(cfg, (0.0, 0.5, 1.0), layout=1, expect_path=path)
+    assert all(r.seqs_exempt <= r.seqs // 2 + 1 for r in reps)
+    W, ht, hd, w = _host_case(cfg, 0)
+    tok = gen.random_draft_tokens(cfg)
+    a = DeviceCase(cfg, W, ht, hd, w, layout=0)
+    b = DeviceCase(cfg, np.ascontiguousarray(W.T), ht, hd, w, layout=1)
+    try:
+        ra, rb = a.run(tok, 0.5), b.run(tok, 0.5)
+        np.testing.assert_array_equal(ra.target_tok, rb.target_tok)
+        np.testing.assert_array_equal(ra.top1, rb.top1)
+        np.testing.assert_array_equal(ra.accept_len, rb.accept_len)
+    finally:
+        a.close()
+        b.close()
+
+
 def test_bf16_dv_layout_runs_on_cuda_cores():
+    # V = 999: the rows of a [d, V] matrix are then not 16-byte aligned, which TMA needs
     cfg = gen.Config("dv", B=2, K=5, d=128, d_draft=64, V=999, sigma_w=0.05, seed=5)
     _full_parity(cfg, (0.5,), layout=1, expect_path="simt")
 

@@ -38,6 +38,22 @@ __device__ inline float key_value(unsigned long long key) {
 
 __device__ inline int key_index(unsigned long long key) { return (int)(~(uint32_t)key); }
 
+#ifdef __CUDACC__
+// The high half of a key, branch-free, for the epilogues: an order-preserving map of a float onto
+// unsigned integers in which the two zeros map to one value (equal to ordered_from_float).
+__device__ inline uint32_t ordered_image(float x) {
+    const uint32_t b = __float_as_uint(x + 0.0f);  // -0.0 + 0.0 = +0.0
+    return b ^ ((uint32_t)((int32_t)b >> 31) | 0x80000000u);
+}
+
+// Maximum of x over the 32 lanes of the warp.
+__device__ inline uint32_t warp_max_u32(uint32_t x) {
+    uint32_t r;
+    asm volatile("redux.sync.max.u32 %0, %1, 0xffffffff;" : "=r"(r) : "r"(x));
+    return r;
+}
+#endif
+
 // Device status word values (mirrors aj_status where they overlap).
 enum : int { DEV_OK = 0, DEV_TIMEOUT = 5 };
 

@@ -50,17 +50,6 @@ constexpr int TMEM_COLS = 2 * BN;
 constexpr int BAR_BYTES = 8 * (2 * MAX_STAGES + 4) + 16;
 constexpr int SMEM_BYTES = RING_BYTES + BAR_BYTES + 1024;
 
-__device__ inline uint32_t ordered_image(float x) {
-    const uint32_t b = __float_as_uint(x + 0.0f);  // -0.0 + 0.0 = +0.0: the two zeros tie
-    return b ^ ((uint32_t)((int32_t)b >> 31) | 0x80000000u);
-}
-
-__device__ inline uint32_t warp_max(uint32_t x) {
-    uint32_t r;
-    asm volatile("redux.sync.max.u32 %0, %1, 0xffffffff;" : "=r"(r) : "r"(x));
-    return r;
-}
-
 struct Tile {
     int v_tile;     // block of 256 vocabulary entries
     int row0[2];    // first row of h of each accumulator
@@ -303,7 +292,7 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
 #pragma unroll
                             for (int j = 0; j < 32; j++) {
                                 const uint32_t x = v_ok ? ordered_image(v[j]) : 0u;
-                                const uint32_t m = warp_max(x);
+                                const uint32_t m = warp_max_u32(x);
                                 const uint32_t who = __ballot_sync(0xffffffffu, x == m);
                                 if (lane == j) {
                                     best_u = m;

@@ -48,18 +48,6 @@ template <int BN> struct VCfg {
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + BAR_BYTES + 1024;  // + alignment slack
 };
 
-// order-preserving map of a float onto unsigned integers; the two zeros map to one value
-__device__ inline uint32_t ordered_u32(float x) {
-    const uint32_t b = __float_as_uint(x + 0.0f);  // -0.0 + 0.0 = +0.0
-    return b ^ ((uint32_t)((int32_t)b >> 31) | 0x80000000u);
-}
-
-__device__ inline uint32_t warp_max_u32(uint32_t x) {
-    uint32_t r;
-    asm volatile("redux.sync.max.u32 %0, %1, 0xffffffff;" : "=r"(r) : "r"(x));
-    return r;
-}
-
 template <int BN>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 umma_vm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_h,
@@ -232,7 +220,7 @@ umma_vm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                     // latencies overlap instead of adding up
                     uint32_t u[32], m[32];
 #pragma unroll
-                    for (int j = 0; j < 32; j++) u[j] = v_ok ? ordered_u32(v[j]) : 0u;
+                    for (int j = 0; j < 32; j++) u[j] = v_ok ? ordered_image(v[j]) : 0u;
 #pragma unroll
                     for (int j = 0; j < 32; j++) m[j] = warp_max_u32(u[j]);
 #pragma unroll

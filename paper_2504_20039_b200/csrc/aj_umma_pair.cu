@@ -84,10 +84,11 @@ __device__ inline Tile decode_tile(const PairSched &sc, int t) {
     return r;
 }
 
-template <bool DUAL>  // DUAL: every tile uses two accumulators that share the staged block of W
+// DUAL: every tile uses two accumulators that share the staged block of W.  WDV: W is stored [d, V].
+template <bool DUAL, bool WDV>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_h,
-                 int M, int V, int d, PairSched sc, int stream_w, int w_dv, int v_offset,
+                 int M, int V, int d, PairSched sc, int stream_w, int v_offset,
                  unsigned long long *__restrict__ keys, int *__restrict__ status, const Publish pub) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -169,7 +170,7 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
                     const uint32_t leader_full = map_to_cta(full_bar(s), 0);
                     if (rank == 0) mbar_expect_tx(full_bar(s), stage_tx);
                     const uint32_t a_dst = base + s * stage_bytes;
-                    if (w_dv) {  // W stored [d, V]: two boxes of 64 entries x 64 k-rows
+                    if (WDV) {  // W stored [d, V]: two boxes of 64 entries x 64 k-rows
                         tma_load_2d_pair(a_dst, &tmap_w, w_row, kb * BK, leader_full, pol_w);
                         tma_load_2d_pair(a_dst + A_BYTES / 2, &tmap_w, w_row + 64, kb * BK, leader_full, pol_w);
                     } else {
@@ -187,13 +188,17 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
     } else if (warp == 1) {
         if (lane == 0 && rank == 0) {
             // ------------------------------------------- MMA issuer (leader CTA only)
+            // (rebuilding the descriptors per k-block measured slightly faster than stepping them
+            // from stage to stage, which chains every k-block's issue to the previous one)
+            const unsigned long long acc_step = b_bytes >> 4;
+            constexpr unsigned long long a_step = WDV ? MN_KSTEP : 2ull;
             int s = 0;
             uint32_t ph = 0;
             bool ok = true;
             int it = 0;
             for (int t = pair; ok && t < num_tiles; t += num_pairs, ++it) {
                 const Tile tl = decode_tile(sc, t);
-                const uint32_t a_major = w_dv ? IDESC_A_MN_MAJOR : 0u;
+                constexpr uint32_t a_major = WDV ? IDESC_A_MN_MAJOR : 0u;
                 const uint32_t idesc0 = instr_desc(BV, tl.n_inst[0]) | a_major;
                 const uint32_t idesc1 = instr_desc(BV, tl.n_inst[1]) | a_major;
                 const int slot = acc_slot(it);
@@ -212,14 +217,13 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
                     }
                     tc_fence_after();
                     const uint32_t a_addr = base + s * stage_bytes;
-                    const unsigned long long adesc = w_dv ? smem_desc_sw128_mn(a_addr) : smem_desc_sw128(a_addr);
-                    const unsigned long long a_step = w_dv ? MN_KSTEP : 2ull;
+                    const unsigned long long adesc = WDV ? smem_desc_sw128_mn(a_addr) : smem_desc_sw128(a_addr);
                     const unsigned long long bdesc0 = smem_desc_sw128(a_addr + A_BYTES);
 #pragma unroll
                     for (int k = 0; k < BK / UMMA_K; k++)
                         umma_bf16_pair(d_tmem0, adesc + a_step * k, bdesc0 + 2ull * k, idesc0, (uint32_t)((kb | k) != 0));
                     if (n_acc == 2) {
-                        const unsigned long long bdesc1 = smem_desc_sw128(a_addr + A_BYTES + b_bytes);
+                        const unsigned long long bdesc1 = bdesc0 + acc_step;
 #pragma unroll
                         for (int k = 0; k < BK / UMMA_K; k++)
                             umma_bf16_pair(d_tmem1, adesc + a_step * k, bdesc1 + 2ull * k, idesc1, (uint32_t)((kb | k) != 0));
@@ -339,9 +343,13 @@ int g_max_pairs = 0;
 }  // namespace
 
 cudaError_t umma_pair_prepare(int num_sms) {
-    cudaError_t e = cudaFuncSetAttribute(umma_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    cudaError_t e = cudaFuncSetAttribute(umma_pair_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(umma_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    e = cudaFuncSetAttribute(umma_pair_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(umma_pair_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(umma_pair_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e != cudaSuccess) return e;
     // how many CTA pairs can be resident at once (pairs need both SMs of a pair free)
     cudaLaunchConfig_t cfg = {};
@@ -356,7 +364,7 @@ cudaError_t umma_pair_prepare(int num_sms) {
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     int clusters = 0;
-    e = cudaOccupancyMaxActiveClusters(&clusters, umma_pair_kernel<false>, &cfg);
+    e = cudaOccupancyMaxActiveClusters(&clusters, umma_pair_kernel<false, false>, &cfg);
     if (e != cudaSuccess) return e;
     if (clusters < 1) return cudaErrorInvalidConfiguration;
     g_max_pairs = clusters < num_sms / 2 ? clusters : num_sms / 2;
@@ -413,11 +421,10 @@ cudaError_t launch_umma_pair(const GemmArgs &a, const UmmaPlan &p, cudaStream_t 
     attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    if (sc.dual)
-        return cudaLaunchKernelEx(&cfg, umma_pair_kernel<true>, p.tmap_w, p.tmap_h, a.M, a.V, a.d, sc, stream_w, a.w_layout, a.v_offset,
-                                  a.keys, a.status, a.pub);
-    return cudaLaunchKernelEx(&cfg, umma_pair_kernel<false>, p.tmap_w, p.tmap_h, a.M, a.V, a.d, sc, stream_w, a.w_layout, a.v_offset,
-                              a.keys, a.status, a.pub);
+    auto kernel = sc.dual ? (a.w_layout ? umma_pair_kernel<true, true> : umma_pair_kernel<true, false>)
+                          : (a.w_layout ? umma_pair_kernel<false, true> : umma_pair_kernel<false, false>);
+    return cudaLaunchKernelEx(&cfg, kernel, p.tmap_w, p.tmap_h, a.M, a.V, a.d, sc, stream_w, a.v_offset, a.keys, a.status,
+                              a.pub);
 }
 
 }  // namespace aj

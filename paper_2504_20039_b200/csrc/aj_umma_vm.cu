@@ -48,10 +48,10 @@ template <int BN> struct VCfg {
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + BAR_BYTES + 1024;  // + alignment slack
 };
 
-template <int BN>
+template <int BN, bool WDV>  // WDV: W is stored [d, V]
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 umma_vm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_h,
-               int M, int V, int d, int n_n, int n_v, int stream_w, int w_dv, int v_offset,
+               int M, int V, int d, int n_n, int n_v, int stream_w, int v_offset,
                unsigned long long *__restrict__ keys, int *__restrict__ status, const Publish pub) {
     using C = VCfg<BN>;
     constexpr int STAGES = C::STAGES;
@@ -119,7 +119,7 @@ umma_vm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                     }
                     mbar_expect_tx(full_bar(s), C::STAGE_BYTES);
                     const uint32_t a_dst = base + s * C::STAGE_BYTES;
-                    if (w_dv) {  // W stored [d, V]: two boxes of 64 entries x 64 k-rows
+                    if (WDV) {  // W stored [d, V]: two boxes of 64 entries x 64 k-rows
                         tma_load_2d(a_dst, &tmap_w, v_tile * BV, kb * BK, full_bar(s), pol_w);
                         tma_load_2d(a_dst + A_BYTES / 2, &tmap_w, v_tile * BV + 64, kb * BK, full_bar(s), pol_w);
                     } else {
@@ -144,7 +144,7 @@ umma_vm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                 const int n_tile = t % n_n;
                 const int rows_valid = min(BN, M - n_tile * BN);
                 const int n_inst = max(16, (rows_valid + 15) & ~15);  // UMMA N: a multiple of 16
-                const uint32_t idesc = instr_desc(BV, n_inst) | (w_dv ? IDESC_A_MN_MAJOR : 0u);
+                const uint32_t idesc = instr_desc(BV, n_inst) | (WDV ? IDESC_A_MN_MAJOR : 0u);
                 const int ab = it & 1;
                 const uint32_t aph = (uint32_t)(it >> 1) & 1u;
                 if (!mbar_wait(acc_empty_bar(ab), aph ^ 1u, abort_flag)) {
@@ -161,8 +161,8 @@ umma_vm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                     }
                     tc_fence_after();
                     const uint32_t a_addr = base + s * C::STAGE_BYTES;
-                    const unsigned long long adesc = w_dv ? smem_desc_sw128_mn(a_addr) : smem_desc_sw128(a_addr);
-                    const unsigned long long a_step = w_dv ? MN_KSTEP : 2ull;
+                    const unsigned long long adesc = WDV ? smem_desc_sw128_mn(a_addr) : smem_desc_sw128(a_addr);
+                    constexpr unsigned long long a_step = WDV ? MN_KSTEP : 2ull;
                     const unsigned long long bdesc = smem_desc_sw128(a_addr + A_BYTES);
 #pragma unroll
                     for (int k = 0; k < BK / UMMA_K; k++)
@@ -270,8 +270,9 @@ cudaError_t launch_vm(const GemmArgs &a, const UmmaPlan &p, cudaStream_t stream)
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, umma_vm_kernel<BN>, p.tmap_w, p.tmap_h, a.M, a.V, a.d, n_n, n_v, stream_w, a.w_layout, a.v_offset,
-                              a.keys, a.status, a.pub);
+    auto kernel = a.w_layout ? umma_vm_kernel<BN, true> : umma_vm_kernel<BN, false>;
+    return cudaLaunchKernelEx(&cfg, kernel, p.tmap_w, p.tmap_h, a.M, a.V, a.d, n_n, n_v, stream_w, a.v_offset, a.keys,
+                              a.status, a.pub);
 }
 
 }  // namespace
@@ -280,13 +281,21 @@ int vm_choose_bn(int M) { return M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : 
 
 cudaError_t umma_vm_prepare() {
     cudaError_t e;
-    e = cudaFuncSetAttribute(umma_vm_kernel<32>, cudaFuncAttributeMaxDynamicSharedMemorySize, VCfg<32>::SMEM_BYTES);
+    e = cudaFuncSetAttribute(umma_vm_kernel<32, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, VCfg<32>::SMEM_BYTES);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(umma_vm_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, VCfg<64>::SMEM_BYTES);
+    e = cudaFuncSetAttribute(umma_vm_kernel<32, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, VCfg<32>::SMEM_BYTES);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(umma_vm_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, VCfg<128>::SMEM_BYTES);
+    e = cudaFuncSetAttribute(umma_vm_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, VCfg<64>::SMEM_BYTES);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(umma_vm_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, VCfg<256>::SMEM_BYTES);
+    e = cudaFuncSetAttribute(umma_vm_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, VCfg<64>::SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(umma_vm_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, VCfg<128>::SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(umma_vm_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, VCfg<128>::SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(umma_vm_kernel<256, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, VCfg<256>::SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(umma_vm_kernel<256, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, VCfg<256>::SMEM_BYTES);
     return e;
 }
 

@@ -212,9 +212,9 @@ class GpuWorkload:
 CSRC = os.path.join(ROOT, "paper_2504_20039_b200", "csrc")
 NCU_TRAFFIC = {
     # (workload, kernel configuration): (bytes per launch, kernel source files, sha1 of those files)
-    ("c2_8b_b1_k16", "umma_vm_128x32"): (1.0547e9, ["aj_umma_vm.cu"], "9f104a6d84b1"),        # profiles/umma_vm_128x32_c2_8b_b1_k16.md
-    ("c3_8b_b64_k32", "umma_pair_256x256"): (1.0735e9, ["aj_umma_pair.cu"], "50125b50fbb8"),  # profiles/umma_pair_256x256_c3_8b_b64_k32.md
-    ("c4_70b_b32_k64", "umma_pair_256x256"): (3.1872e9, ["aj_umma_pair.cu"], "50125b50fbb8"),  # profiles/umma_pair_256x256_c4_70b_b32_k64.md
+    ("c2_8b_b1_k16", "umma_vm_128x32"): (1.0547e9, ["aj_umma_vm.cu"], "b95ca07c429b"),        # profiles/umma_vm_128x32_c2_8b_b1_k16.md
+    ("c3_8b_b64_k32", "umma_pair_256x256"): (1.3295e9, ["aj_umma_pair.cu"], "b57c867d6820"),  # profiles/umma_pair_256x256_c3_8b_b64_k32.md
+    ("c4_70b_b32_k64", "umma_pair_256x256"): (3.5888e9, ["aj_umma_pair.cu"], "b57c867d6820"),  # profiles/umma_pair_256x256_c4_70b_b32_k64.md
 }
 
 

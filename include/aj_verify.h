@@ -114,7 +114,9 @@ aj_status aj_verify(aj_handle h, const void *h_target, const void *h_draft, cons
  * draft_tok are HOST pointers and are copied to the handle's staging buffers; accept_len and
  * next_tok (and target_tok, if not NULL) are HOST pointers and are copied back.  W_lm and judge_w
  * are model parameters and stay DEVICE pointers.  The call synchronises `cuda_stream` before it
- * returns, so the host outputs are valid on return.
+ * returns, so the host outputs are valid on return.  draft_tok and the outputs are used in place,
+ * without a copy, when they are pinned host memory (cudaHostAlloc / cudaHostRegister); pageable
+ * buffers work too and are copied.
  */
 aj_status aj_verify_host(aj_handle h, const void *h_target_host, const void *h_draft_host,
                          const void *W_lm, const int32_t *draft_tok_host, const float *judge_w,

@@ -139,6 +139,17 @@ aj_status check_call(aj_handle h, const void *h_target, const void *h_draft, con
 // the last draft token when the caller does not encode it
 int rows_per_seq(aj_handle h, int K) { return (h->flags & AJ_FLAG_NO_EXTRA_ROW) ? K : K + 1; }
 
+// The address at which the current device can read and write a HOST buffer directly, or nullptr
+// if the buffer is ordinary pageable memory (then it has to be copied).
+void *device_view(const void *host_ptr) {
+    cudaPointerAttributes attr;
+    if (cudaPointerGetAttributes(&attr, host_ptr) != cudaSuccess) {
+        cudaGetLastError();
+        return nullptr;
+    }
+    return attr.type == cudaMemoryTypeHost ? attr.devicePointer : nullptr;
+}
+
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
 }  // namespace
@@ -415,18 +426,28 @@ aj_status aj_verify_host(aj_handle h, const void *h_target_host, const void *h_d
     if (!guard.ok()) return AJ_ERR_CUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const size_t M = (size_t)B * rows_per_seq(h, K), esz = elem_size(h->dtype);
+    // Small host buffers that are pinned (and therefore mapped into the device's address space) are
+    // used in place by the judge kernel: it reads the draft tokens and writes the results over PCIe,
+    // which saves three copy operations per cycle.  The hidden states are always copied: the
+    // projection kernel reads them a thousand times over.
+    int32_t *tok_dev = static_cast<int32_t *>(device_view(draft_tok_host));
+    int32_t *acc_dev = static_cast<int32_t *>(device_view(accept_len_host));
+    int32_t *next_dev = static_cast<int32_t *>(device_view(next_tok_host));
+    int32_t *tt_dev = target_tok_host ? static_cast<int32_t *>(device_view(target_tok_host)) : nullptr;
     bool ok = cudaMemcpyAsync(h->st_ht, h_target_host, M * d * esz, cudaMemcpyHostToDevice, stream) == cudaSuccess &&
               (h->d_draft == 0 ||
                cudaMemcpyAsync(h->st_hd, h_draft_host, M * h->d_draft * esz, cudaMemcpyHostToDevice, stream) == cudaSuccess) &&
-              cudaMemcpyAsync(h->st_tok, draft_tok_host, (size_t)B * K * 4, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+              (tok_dev || cudaMemcpyAsync(h->st_tok, draft_tok_host, (size_t)B * K * 4, cudaMemcpyHostToDevice, stream) == cudaSuccess);
     if (!ok) return AJ_ERR_CUDA;
-    st = aj_verify(h, h->st_ht, h->d_draft ? h->st_hd : nullptr, W_lm, h->st_tok, judge_w, judge_b, tau, B, K, d, V, h->st_acc,
-                   h->st_next, target_tok_host ? h->st_tt : nullptr, nullptr, nullptr, cuda_stream);
+    st = aj_verify(h, h->st_ht, h->d_draft ? h->st_hd : nullptr, W_lm, tok_dev ? tok_dev : h->st_tok, judge_w, judge_b, tau, B, K,
+                   d, V, acc_dev ? acc_dev : h->st_acc, next_dev ? next_dev : h->st_next,
+                   target_tok_host ? (tt_dev ? tt_dev : h->st_tt) : nullptr, nullptr, nullptr, cuda_stream);
     if (st != AJ_OK) return st;
     const int launches = h->last_launches;
-    ok = cudaMemcpyAsync(accept_len_host, h->st_acc, (size_t)B * 4, cudaMemcpyDeviceToHost, stream) == cudaSuccess &&
-         cudaMemcpyAsync(next_tok_host, h->st_next, (size_t)B * 4, cudaMemcpyDeviceToHost, stream) == cudaSuccess &&
-         (!target_tok_host || cudaMemcpyAsync(target_tok_host, h->st_tt, M * 4, cudaMemcpyDeviceToHost, stream) == cudaSuccess) &&
+    ok = (acc_dev || cudaMemcpyAsync(accept_len_host, h->st_acc, (size_t)B * 4, cudaMemcpyDeviceToHost, stream) == cudaSuccess) &&
+         (next_dev || cudaMemcpyAsync(next_tok_host, h->st_next, (size_t)B * 4, cudaMemcpyDeviceToHost, stream) == cudaSuccess) &&
+         (!target_tok_host || tt_dev ||
+          cudaMemcpyAsync(target_tok_host, h->st_tt, M * 4, cudaMemcpyDeviceToHost, stream) == cudaSuccess) &&
          cudaStreamSynchronize(stream) == cudaSuccess;
     h->last_launches = launches;
     return ok ? AJ_OK : AJ_ERR_CUDA;

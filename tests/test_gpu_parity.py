@@ -365,6 +365,13 @@ def test_host_buffer_entry_point_matches_device_entry_point():
         np.testing.assert_array_equal(acc.numpy(), g.accept_len)
         np.testing.assert_array_equal(nxt.numpy(), g.next_tok)
         np.testing.assert_array_equal(tt.numpy(), g.target_tok)
+        # pageable host buffers (plain numpy arrays) take the copying route and give the same
+        acc2, nxt2, tt2 = np.full(cfg.B, -1, np.int32), np.full(cfg.B, -1, np.int32), np.full((cfg.B, cfg.K + 1), -1, np.int32)
+        case.handle.verify_host(ht.copy(), hd.copy(), case.W, tok.copy(), case.w, 0.0, 0.5, cfg.B, cfg.K, acc2, nxt2, tt2,
+                                stream=torch.cuda.current_stream().cuda_stream)
+        np.testing.assert_array_equal(acc2, g.accept_len)
+        np.testing.assert_array_equal(nxt2, g.next_tok)
+        np.testing.assert_array_equal(tt2, g.target_tok)
     finally:
         case.close()
 

@@ -399,8 +399,8 @@ def main():
     if "e2e_s_per_step" in r:
         line["e2e"] = {"value": positions / r["e2e_s_per_step"], "unit": UNIT, "h2d_bytes_per_step": r["h2d"],
                        "d2h_bytes_per_step": r["d2h"], "us_per_cycle": r["e2e_s_per_step"] * 1e6,
-                       "note": "aj_verify_host: hidden states and draft tokens from pinned host memory, results read back; "
-                               "W_lm and judge_w are resident parameters"}
+                       "note": "aj_verify_host: hidden states copied from pinned host memory, draft tokens read and results "
+                               "written in place over PCIe by the judge kernel; W_lm and judge_w are resident parameters"}
 
     extra = []
     if not args.no_extra:

@@ -33,6 +33,12 @@
  * the classifier, and when all K positions pass there is no row to predict a further token from
  * (next_tok = -1).
  *
+ * Top-K rule (Section 4.1, the lossy baseline the paper compares with): instead of consulting the
+ * classifier, a mismatching draft token is accepted iff it is among the top_k most likely tokens of
+ * the target, i.e. iff its rank (number of vocabulary entries with a larger logit; among equal
+ * logits the lower index ranks first) is below top_k.  A draft token outside the vocabulary is
+ * never accepted.  See ajo_verify_topk.
+ *
  * All inputs are converted exactly to double; every sum is accumulated in double.
  *
  * parity pins: see tests/test_oracle_pins.py (library matmul special case, one-hot
@@ -209,6 +215,72 @@ int ajo_verify(const void *h_target, const void *h_draft, const void *W,
         }
         accept_len[b] = n;
         next_tok[b] = n < R ? y[n] : -1;
+    }
+    free(logits);
+    return 0;
+}
+
+/*
+ * Rank of entry `tok` in one row of logits: how many entries come before it when the row is sorted
+ * by decreasing logit, ties by increasing index.  *near receives the number of OTHER entries whose
+ * logit lies within `band` of logit[tok] (a device that rounds differently may order those otherwise).
+ */
+int ajo_rank(const double *row, int V, int tok, double band, int32_t *near)
+{
+    int rank = 0, n = 0;
+    const double t = row[tok];
+    for (int v = 0; v < V; v++) {
+        if (v == tok) continue;
+        if (row[v] > t || (row[v] == t && v < tok)) rank++;
+        if (fabs(row[v] - t) <= band) n++;
+    }
+    if (near) *near = n;
+    return rank;
+}
+
+/*
+ * The whole step under the top-K rule for B sequences, K + 1 rows each (layouts as ajo_verify).
+ * Outputs: accept_len [B], next_tok [B], target_tok [B][K+1], top1 [B][K+1], gap [B][K+1],
+ *   rank [B][K]  rank of the draft token at every mismatching position (-1 where it matched, V where
+ *                the draft token is outside the vocabulary),
+ *   near [B][K]  entries within `band` of the draft token's logit there (0 where it matched).
+ */
+int ajo_verify_topk(const void *h_target, const void *W, const int32_t *draft_tok, int top_k, double band,
+                    int dtype, int w_layout, int B, int K, int d, int V,
+                    int32_t *accept_len, int32_t *next_tok, int32_t *target_tok,
+                    double *top1, double *gap, int32_t *rank, int32_t *near)
+{
+    if (!h_target || !W || !draft_tok || B < 1 || K < 1 || d < 1 || V < 1 || top_k < 1) return 1;
+    size_t esz = (dtype == AJO_BF16) ? 2 : 4;
+    int R = K + 1;
+    double *logits = (double *)malloc((size_t)R * V * sizeof(double));
+    if (!logits) return 2;
+    for (int b = 0; b < B; b++) {
+        const char *ht = (const char *)h_target + (size_t)b * R * d * esz;
+        int rc = ajo_logits(ht, W, dtype, w_layout, R, d, V, logits);
+        if (rc) { free(logits); return rc; }
+        int32_t *y = target_tok + (size_t)b * R;
+        for (int j = 0; j < R; j++)
+            ajo_argmax(logits + (size_t)j * V, V, &y[j], &top1[(size_t)b * R + j], &gap[(size_t)b * R + j]);
+        for (int i = 0; i < K; i++) {
+            int tok = draft_tok[(size_t)b * K + i];
+            int32_t r = -1, n = 0;
+            if (tok != y[i]) {
+                if (tok < 0 || tok >= V) r = V;
+                else r = ajo_rank(logits + (size_t)i * V, V, tok, band, &n);
+            }
+            rank[(size_t)b * K + i] = r;
+            near[(size_t)b * K + i] = n;
+        }
+        int n = 0;
+        while (n < K) {
+            int32_t r = rank[(size_t)b * K + n];
+            int t = draft_tok[(size_t)b * K + n];
+            if (r >= 0 && (t < 0 || t >= V || !(r < top_k))) break; /* a mismatch outside the target's top_k */
+            n++;
+        }
+        accept_len[b] = n;
+        next_tok[b] = y[n];
     }
     free(logits);
     return 0;

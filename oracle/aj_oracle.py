@@ -66,6 +66,10 @@ def _lib():
         L.ajo_judge_p.restype = ctypes.c_double
         L.ajo_verify.argtypes = [vp, vp, vp, ip, fp, cf, cf, ci, ci, ci, ci, ci, ci, ci, ci, ip, ip, ip, dp, dp, dp]
         L.ajo_verify.restype = ci
+        L.ajo_rank.argtypes = [dp, ci, ci, ctypes.c_double, ip]
+        L.ajo_rank.restype = ci
+        L.ajo_verify_topk.argtypes = [vp, vp, ip, ci, ctypes.c_double, ci, ci, ci, ci, ci, ci, ip, ip, ip, dp, dp, ip, ip]
+        L.ajo_verify_topk.restype = ci
         _LIB = L
     return _LIB
 
@@ -183,3 +187,40 @@ def rewalk(target_tok, draft_tok, judge_p_all, tau):
         acc[b] = n
         nxt[b] = target_tok[b, n]
     return acc, nxt
+
+
+def rank(row: np.ndarray, tok: int, band: float = 0.0):
+    """(rank of entry tok by decreasing logit, ties by index; number of other entries within band of it)."""
+    row = np.ascontiguousarray(row, dtype=np.float64)
+    near = ctypes.c_int32()
+    r = _lib().ajo_rank(_ptr(row), row.shape[0], int(tok), float(band), ctypes.byref(near))
+    return int(r), int(near.value)
+
+
+@dataclass
+class TopKResult:
+    accept_len: np.ndarray  # [B]
+    next_tok: np.ndarray  # [B]
+    target_tok: np.ndarray  # [B, K+1]
+    top1: np.ndarray  # [B, K+1]
+    gap: np.ndarray  # [B, K+1]
+    rank: np.ndarray  # [B, K]: -1 where the draft token matched
+    near: np.ndarray  # [B, K]
+
+
+def verify_topk(h_target, W, draft_tok, top_k: int, dtype: int, w_layout: int = 0, band: float = 1e-2) -> TopKResult:
+    """The step under the top-K rule of Section 4.1 (see aj_oracle.c)."""
+    ht = _check_storage(h_target, dtype, "h_target")
+    W = _check_storage(W, dtype, "W")
+    tok = np.ascontiguousarray(draft_tok, dtype=np.int32)
+    B, R, d = ht.shape
+    K = R - 1
+    V = W.shape[0] if w_layout == 0 else W.shape[1]
+    res = TopKResult(np.empty(B, np.int32), np.empty(B, np.int32), np.empty((B, R), np.int32), np.empty((B, R), np.float64),
+                     np.empty((B, R), np.float64), np.empty((B, K), np.int32), np.empty((B, K), np.int32))
+    rc = _lib().ajo_verify_topk(_ptr(ht), _ptr(W), _ptr(tok), int(top_k), float(band), dtype, w_layout, B, K, d, V,
+                                _ptr(res.accept_len), _ptr(res.next_tok), _ptr(res.target_tok), _ptr(res.top1), _ptr(res.gap),
+                                _ptr(res.rank), _ptr(res.near))
+    if rc:
+        raise RuntimeError(f"ajo_verify_topk failed: {rc}")
+    return res

@@ -362,3 +362,62 @@ def test_without_the_extra_row_single_token_window():
     r = orc.verify(ht, None, W, tok, w, 0.0, 1.0, cfg.dtype, extra_row=False)
     np.testing.assert_array_equal(r.accept_len, np.where(np.arange(cfg.B) % 2 == 0, 0, 1))
     np.testing.assert_array_equal(r.next_tok, np.where(np.arange(cfg.B) % 2 == 0, y, -1))
+
+
+# ------------------------------------------------------------------- the top-K rule (Section 4.1)
+
+
+def test_rank_equals_position_in_a_stable_sort():
+    g = np.random.default_rng(5)
+    row = np.round(g.standard_normal(300), 1)            # rounded: plenty of exact ties
+    order = np.argsort(-row, kind="stable")              # decreasing logit, ties by increasing index
+    pos = np.empty_like(order)
+    pos[order] = np.arange(row.size)
+    for tok in (0, 7, 150, 299, int(order[0]), int(order[-1])):
+        r, near = orc.rank(row, tok, band=0.05)
+        assert r == pos[tok]
+        assert near == int((np.abs(row - row[tok]) <= 0.05).sum()) - 1
+    assert orc.rank(row, int(order[0]))[0] == 0
+
+
+@pytest.mark.parametrize("dtype", [BF16, F32])
+def test_top_k_rule_extremes_monotonicity_and_brute_force(dtype):
+    B, K, d, V = 12, 6, 32, 40
+    cfg = gen.Config("topk", B=B, K=K, d=d, d_draft=0, V=V, dtype=dtype, sigma_W=0.3, match_lo=0.3, match_hi=0.7, seed=61)
+    W = gen.make_W(cfg)
+    ht, _ = gen.make_hidden(cfg)
+    lg = np.stack([orc.logits(ht[b], W, dtype) for b in range(B)])      # [B, K+1, V]
+    y = np.stack([[orc.argmax(r)[0] for r in lg[b]] for b in range(B)])
+    tok = gen.plant_draft_tokens(cfg, y)
+    tok[0, 2] = -3                                                        # outside the vocabulary: never accepted
+    tok[1, 1] = V + 5
+    vanilla = np.array([int(np.argmax(np.append(tok[b] != y[b, :K], True))) for b in range(B)])
+    prev = None
+    for k in (1, 2, 3, 5, 10, V, V + 7):
+        r = orc.verify_topk(ht, W, tok, k, dtype)
+        np.testing.assert_array_equal(r.target_tok, y)
+        # brute force from a full sort of every row
+        for b in range(B):
+            n = 0
+            while n < K:
+                t = tok[b, n]
+                if t != y[b, n]:
+                    if not (0 <= t < V):
+                        break
+                    order = np.argsort(-lg[b, n], kind="stable")
+                    if int(np.nonzero(order == t)[0][0]) >= k:
+                        break
+                n += 1
+            assert r.accept_len[b] == n and r.next_tok[b] == y[b, n]
+        if k == 1:  # only the argmax itself is in the top 1, and a mismatch is not the argmax: plain greedy verification
+            np.testing.assert_array_equal(r.accept_len, vanilla)
+        if k >= V:  # every token of the vocabulary is in the top V
+            in_vocab_everywhere = np.array([((tok[b] >= 0) & (tok[b] < V)).all() for b in range(B)])
+            assert (r.accept_len[in_vocab_everywhere] == K).all()
+            assert r.accept_len[0] == 2 and r.accept_len[1] == 1  # stops exactly at the ids outside the vocabulary
+        assert (r.accept_len >= vanilla).all()
+        if prev is not None:
+            assert (r.accept_len >= prev).all()  # a larger K accepts more (Section 4.1)
+        prev = r.accept_len.copy()
+    r = orc.verify_topk(ht, W, tok, V, dtype)
+    assert r.accept_len[0] == 2 and r.accept_len[1] == 1 and r.rank[0, 2] == V

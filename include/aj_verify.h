@@ -110,6 +110,20 @@ aj_status aj_verify(aj_handle h, const void *h_target, const void *h_draft, cons
                     float *top1_val, float *judge_p, void *cuda_stream);
 
 /*
+ * Switch the acceptance rule of a handle to the top-K rule of the paper's Section 4.1 (the lossy
+ * baseline it compares with): a mismatching draft token is accepted iff it is among the top_k most
+ * likely tokens of the target, i.e. iff fewer than top_k vocabulary entries have a larger logit
+ * (among equal logits the lower index ranks first; a draft token outside the vocabulary is never
+ * accepted).  The classifier is then not consulted: judge_w and h_draft may be NULL and judge_b, tau
+ * are ignored; judge_p, if given, receives the draft token's rank (as a float, 0 = the target's own
+ * token) at every mismatching position and NaN elsewhere.  A cycle then launches three kernels (the
+ * draft tokens' own logits, the projection with the count fused into its epilogue, the scan).
+ * top_k = 0 switches back to the classifier.  Not available on vocabulary-parallel handles, with
+ * AJ_FLAG_ROW_TILES or with AJ_FLAG_NO_EXTRA_ROW (AJ_ERR_UNSUPPORTED).  Errors: AJ_ERR_INVALID_ARG.
+ */
+aj_status aj_set_top_k(aj_handle h, int top_k);
+
+/*
  * The same cycle for a caller whose per-cycle tensors live in host memory: h_target, h_draft and
  * draft_tok are HOST pointers and are copied to the handle's staging buffers; accept_len and
  * next_tok (and target_tok, if not NULL) are HOST pointers and are copied back.  W_lm and judge_w

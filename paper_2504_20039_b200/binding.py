@@ -19,7 +19,7 @@ AJ_FLAG_FORCE_SIMT, AJ_FLAG_TIME_KERNELS, AJ_FLAG_ROW_TILES, AJ_FLAG_ONE_SM, AJ_
 
 EXPORTS = (
     "aj_create", "aj_verify", "aj_verify_host", "aj_last_status", "aj_last_gemm_ms", "aj_gemm_ms_stats", "aj_last_launch_count",
-    "aj_last_gemm_path", "aj_pair_schedule", "aj_destroy", "aj_shard_exchange_bytes", "aj_shard_exchange_alloc", "aj_shard_exchange_free", "aj_shard_range", "aj_create_sharded",
+    "aj_last_gemm_path", "aj_pair_schedule", "aj_destroy", "aj_set_top_k", "aj_shard_exchange_bytes", "aj_shard_exchange_alloc", "aj_shard_exchange_free", "aj_shard_range", "aj_create_sharded",
     "aj_shard_project", "aj_shard_finish", "aj_ipc_export", "aj_ipc_import", "aj_ipc_close", "aj_status_string", "aj_version", "aj_verify_static",
 )
 
@@ -87,6 +87,8 @@ def lib() -> ctypes.CDLL:
         L.aj_ipc_import.restype = ci
         L.aj_ipc_close.argtypes = [vp]
         L.aj_ipc_close.restype = ci
+        L.aj_set_top_k.argtypes = [vp, ci]
+        L.aj_set_top_k.restype = ci
         L.aj_version.argtypes = []
         L.aj_version.restype = ctypes.c_char_p
         _lib = L
@@ -252,6 +254,13 @@ class Handle:
                                   _ptr(target_tok), stream or None)
         if check and st != AJ_OK:
             raise AjError(st, "aj_verify_host")
+        return st
+
+    def set_top_k(self, top_k: int, check: bool = True) -> int:
+        """aj_set_top_k: accept a mismatch iff the draft token is among the target's top_k (0: back to the classifier)."""
+        st = lib().aj_set_top_k(self._h, int(top_k))
+        if check and st != AJ_OK:
+            raise AjError(st, "aj_set_top_k")
         return st
 
     def last_status(self) -> int:

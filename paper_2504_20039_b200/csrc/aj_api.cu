@@ -56,6 +56,11 @@ struct aj_handle_s {
     unsigned long long *exchange[MAX_SHARD_WORLD] = {};  // every GPU's exchange buffer, as mapped on this device
     unsigned long long epoch = 0;    // cycles started; the same on every rank, which call in step
     bool projected = false;          // aj_shard_project was enqueued and its aj_shard_finish is still due
+    // top-K rule (aj_set_top_k)
+    int top_k = 0;                   // 0: the classifier decides
+    float *rk_thr = nullptr;         // [max_M] the draft tokens' own logits
+    int *rk_tok = nullptr;           // [max_M]
+    unsigned *rk_cnt = nullptr;      // [max_M] entries that outrank them
 };
 
 // Exchange buffer of one GPU: 256 bytes of flags (one 8-byte epoch per source GPU), then two slot
@@ -128,8 +133,10 @@ aj_status check_call(aj_handle h, const void *h_target, const void *h_draft, con
                      const float *judge_w, int B, int K, int d, int V, const int32_t *accept_len,
                      const int32_t *next_tok) {
     if (!h) return AJ_ERR_INVALID_ARG;
-    if (!h_target || !W_lm || !draft_tok || !judge_w || !accept_len || !next_tok) return AJ_ERR_INVALID_ARG;
-    if ((h->d_draft > 0) != (h_draft != nullptr)) return AJ_ERR_INVALID_ARG;
+    if (!h_target || !W_lm || !draft_tok || !accept_len || !next_tok) return AJ_ERR_INVALID_ARG;
+    if (h->top_k == 0) {  // the classifier's operands are needed unless the top-K rule is in force
+        if (!judge_w || (h->d_draft > 0) != (h_draft != nullptr)) return AJ_ERR_INVALID_ARG;
+    }
     if (B < 1 || K < 1 || d != h->d || V != h->V) return AJ_ERR_INVALID_ARG;
     if (B > h->max_B || K > h->max_K) return AJ_ERR_WORKSPACE;
     return AJ_OK;
@@ -220,7 +227,9 @@ aj_status aj_create(aj_handle *out, int device, int max_B, int max_K, int d, int
               (d_draft == 0 || cudaMalloc(&h->st_hd, max_M * d_draft * esz) == cudaSuccess) &&
               cudaMalloc(&h->st_tok, (size_t)max_B * max_K * 4) == cudaSuccess &&
               cudaMalloc(&h->st_acc, (size_t)max_B * 4) == cudaSuccess &&
-              cudaMalloc(&h->st_next, (size_t)max_B * 4) == cudaSuccess && cudaMalloc(&h->st_tt, max_M * 4) == cudaSuccess;
+              cudaMalloc(&h->st_next, (size_t)max_B * 4) == cudaSuccess && cudaMalloc(&h->st_tt, max_M * 4) == cudaSuccess &&
+              cudaMalloc(&h->rk_thr, max_M * 4) == cudaSuccess && cudaMalloc(&h->rk_tok, max_M * 4) == cudaSuccess &&
+              cudaMalloc(&h->rk_cnt, max_M * 4) == cudaSuccess;
     if (ok && (flags & AJ_FLAG_TIME_KERNELS))
         for (int i = 0; ok && i < EVENT_RING; i++)
             ok = cudaEventCreate(&h->ev0[i]) == cudaSuccess && cudaEventCreate(&h->ev1[i]) == cudaSuccess;
@@ -254,6 +263,9 @@ aj_status aj_destroy(aj_handle h) {
     cudaFree(h->st_acc);
     cudaFree(h->st_next);
     cudaFree(h->st_tt);
+    cudaFree(h->rk_thr);
+    cudaFree(h->rk_tok);
+    cudaFree(h->rk_cnt);
     for (int i = 0; i < EVENT_RING; i++) {
         if (h->ev0[i]) cudaEventDestroy(h->ev0[i]);
         if (h->ev1[i]) cudaEventDestroy(h->ev1[i]);
@@ -263,7 +275,8 @@ aj_status aj_destroy(aj_handle h) {
 }
 
 // Enqueue the projection + argmax kernel of one cycle (and, on a sharded handle, its exchange).
-static aj_status enqueue_project(aj_handle h, const void *h_target, const void *W_lm, int B, int K, cudaStream_t stream) {
+static aj_status enqueue_project(aj_handle h, const void *h_target, const void *W_lm, const int32_t *draft_tok, int B, int K,
+                                 cudaStream_t stream) {
     const int M = B * rows_per_seq(h, K);
     const int d = h->d;
     const int V = h->world ? h->v_count : h->V;  // vocabulary entries this GPU projects
@@ -276,6 +289,28 @@ static aj_status enqueue_project(aj_handle h, const void *h_target, const void *
     h->keys_dirty = true;
 
     GemmArgs g;
+    if (h->top_k > 0) {
+        // top-K rule: the draft tokens' own logits first; the projection kernel counts against them
+        RankPrepArgs r;
+        r.h = h_target;
+        r.W = W_lm;
+        r.draft_tok = draft_tok;
+        r.B = B;
+        r.K = K;
+        r.R = rows_per_seq(h, K);
+        r.d = d;
+        r.V = V;
+        r.dtype = h->dtype;
+        r.w_layout = h->layout;
+        r.thr = h->rk_thr;
+        r.tok = h->rk_tok;
+        r.cnt = h->rk_cnt;
+        if (launch_rank_prepare(r, stream) != cudaSuccess) return AJ_ERR_CUDA;
+        h->last_launches++;
+        g.rank.thr = h->rk_thr;
+        g.rank.tok = h->rk_tok;
+        g.rank.cnt = h->rk_cnt;
+    }
     g.h = h_target;
     g.W = W_lm;
     g.M = M;
@@ -387,6 +422,9 @@ static aj_status enqueue_finish(aj_handle h, const void *h_target, const void *h
     j.d_draft = h->d_draft;
     j.dtype = h->dtype;
     j.no_extra_row = (h->flags & AJ_FLAG_NO_EXTRA_ROW) ? 1 : 0;
+    j.top_k = h->top_k;
+    j.V = h->V;
+    j.rank_cnt = h->rk_cnt;
     j.accept_len = accept_len;
     j.next_tok = next_tok;
     j.target_tok = target_tok;
@@ -409,7 +447,7 @@ aj_status aj_verify(aj_handle h, const void *h_target, const void *h_draft, cons
     DeviceGuard guard(h->device);
     if (!guard.ok()) return AJ_ERR_CUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    st = enqueue_project(h, h_target, W_lm, B, K, stream);
+    st = enqueue_project(h, h_target, W_lm, draft_tok, B, K, stream);
     if (st != AJ_OK) return st;
     return enqueue_finish(h, h_target, h_draft, draft_tok, judge_w, judge_b, tau, B, K, accept_len, next_tok, target_tok,
                           top1_val, judge_p, stream);
@@ -555,7 +593,7 @@ aj_status aj_shard_project(aj_handle h, const void *h_target, const void *W_shar
     if (h->dtype == AJ_BF16 && (!aligned16(h_target) || !aligned16(W_shard))) return AJ_ERR_UNSUPPORTED;
     DeviceGuard guard(h->device);
     if (!guard.ok()) return AJ_ERR_CUDA;
-    aj_status st = enqueue_project(h, h_target, W_shard, B, K, static_cast<cudaStream_t>(cuda_stream));
+    aj_status st = enqueue_project(h, h_target, W_shard, nullptr, B, K, static_cast<cudaStream_t>(cuda_stream));
     if (st == AJ_OK) h->projected = true;
     return st;
 }
@@ -630,6 +668,14 @@ aj_status aj_ipc_close(void *device_ptr) {
         cudaGetLastError();
         return AJ_ERR_CUDA;
     }
+    return AJ_OK;
+}
+
+aj_status aj_set_top_k(aj_handle h, int top_k) {
+    if (!h || top_k < 0) return AJ_ERR_INVALID_ARG;
+    // the count is kept per GPU and the row-tile kernel does not produce it
+    if (top_k > 0 && (h->world || (h->flags & (AJ_FLAG_ROW_TILES | AJ_FLAG_NO_EXTRA_ROW)))) return AJ_ERR_UNSUPPORTED;
+    h->top_k = top_k;
     return AJ_OK;
 }
 

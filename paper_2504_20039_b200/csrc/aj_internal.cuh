@@ -112,6 +112,53 @@ __device__ inline void publish_keys(const Publish &p, unsigned long long *keys) 
 }
 #endif
 
+// ------------------------------------------------------------------- top-K rule (rank counting)
+//
+// Under the top-K rule a mismatching draft token is accepted iff fewer than top_k vocabulary
+// entries outrank it.  A small kernel first computes, per row, the draft token's own logit (the
+// threshold); the projection kernels then also count, per row, the entries that outrank it
+// (larger logit, or equal logit and lower index), and the judge kernel compares the count with top_k.
+struct RankArgs {
+    const float *thr = nullptr;  // [M] the draft token's logit; +inf where the row has no draft token
+    const int *tok = nullptr;    // [M] the draft token, -1 where there is none or it is outside the vocabulary
+    unsigned *cnt = nullptr;     // [M] entries that outrank it (zeroed by the threshold kernel)
+};
+
+#ifdef __CUDACC__
+// Epilogue add-on for the vocabulary-major kernels: the warp holds 32 consecutive vocabulary entries
+// (lane = entry v_first + lane) of 32 columns (rows row_first .. + 32 of h) in v[]; lane j is
+// responsible for column j.
+__device__ inline void count_outranking(const RankArgs &rk, const float (&v)[32], int v_first, bool v_ok, int row_first,
+                                        int n_cols, int M, int lane) {
+    const int row = row_first + lane;
+    const bool valid = lane < n_cols && row < M;
+    const float th = valid ? __ldg(rk.thr + row) : INFINITY;
+    const int tk = valid ? __ldg(rk.tok + row) : -1;
+    const int vidx = v_first + lane;
+    unsigned mine = 0;
+#pragma unroll
+    for (int j = 0; j < 32; j++) {
+        const float t = __shfl_sync(0xffffffffu, th, j);
+        const int k = __shfl_sync(0xffffffffu, tk, j);
+        const bool ahead = v_ok && vidx != k && (v[j] > t || (v[j] == t && vidx < k));
+        const unsigned b = __ballot_sync(0xffffffffu, ahead);
+        if (lane == j) mine = __popc(b);
+    }
+    if (valid && mine) atomicAdd(rk.cnt + row, mine);
+}
+#endif
+
+struct RankPrepArgs {
+    const void *h;             // [M, d]
+    const void *W;             // LM head
+    const int32_t *draft_tok;  // [B, K]
+    int B, K, R, d, V, dtype, w_layout;
+    float *thr;
+    int *tok;
+    unsigned *cnt;
+};
+cudaError_t launch_rank_prepare(const RankPrepArgs &a, cudaStream_t stream);
+
 // ------------------------------------------------------------------------------ launchers
 
 struct GemmArgs {
@@ -124,6 +171,7 @@ struct GemmArgs {
     unsigned long long *keys;  // [M], must be zero on entry (the judge kernel clears what it reads)
     int *status;
     Publish pub;
+    RankArgs rank;       // thr != nullptr: also count, per row, the entries that outrank the draft token
 };
 
 // CUDA-core projection + argmax (any dtype / layout).
@@ -176,6 +224,9 @@ struct JudgeArgs {
     float judge_b, tau;
     int B, K, d, d_draft, dtype;
     int no_extra_row = 0;            // 1: K rows per sequence instead of K + 1
+    int top_k = 0;                   // > 0: the top-K rule replaces the classifier
+    int V = 0;                       // vocabulary size (top-K rule: ids outside it are never accepted)
+    unsigned *rank_cnt = nullptr;    // [B*R] counts from the projection kernel (top-K rule)
     int32_t *accept_len, *next_tok, *target_tok;
     float *top1_val, *judge_p;
 };

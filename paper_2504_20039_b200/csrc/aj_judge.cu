@@ -117,7 +117,7 @@ __global__ void __maxnreg__(96) judge_scan_kernel(JudgeArgs a) {
     // the judge weights (and, for small batches, the candidate feature rows) into L2.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     for (int i = threadIdx.x; i < K; i += blockDim.x) mis_s[i] = a.draft_tok[(size_t)b * K + i];
-    {
+    if (a.top_k == 0) {  // the classifier's operands; the top-K rule needs none of them
         const char *wbytes = reinterpret_cast<const char *>(a.judge_w);
         const size_t wlines = ((size_t)(a.d + a.d_draft) * 4 + 127) / 128;
         for (size_t l = threadIdx.x; l < wlines; l += blockDim.x)
@@ -190,7 +190,7 @@ __global__ void __maxnreg__(96) judge_scan_kernel(JudgeArgs a) {
     const int chunks = (a.d_draft + a.d) / epc;
     for (int it = warp; it < K * SEGS; it += nwarps) {
         const int i = it / SEGS, seg = it % SEGS;
-        if (!mis_s[i] || i + 1 >= R) continue;          // at mismatches only, and only where the features exist
+        if (!mis_s[i] || i + 1 >= R || a.top_k > 0) continue;  // at mismatches only, where the features exist; not under the top-K rule
         const size_t row = (size_t)b * R + (i + 1);     // the hidden states that encode draft token i
         const char *xd = a.h_draft ? reinterpret_cast<const char *>(a.h_draft) + row * row_bytes_d : nullptr;
         const char *xt = reinterpret_cast<const char *>(a.h_target) + row * row_bytes_t;
@@ -213,7 +213,14 @@ __global__ void __maxnreg__(96) judge_scan_kernel(JudgeArgs a) {
     for (int i = threadIdx.x; i < K; i += blockDim.x) {
         float p = __int_as_float(0x7fc00000);  // NaN where the judge is not consulted
         int rej = 0;
-        if (mis_s[i] && i + 1 >= R) {
+        if (mis_s[i] && a.top_k > 0) {
+            // top-K rule: accepted iff fewer than top_k entries outrank the draft token; p reports the rank
+            const int tk = a.draft_tok[(size_t)b * K + i];
+            const bool in_vocab = tk >= 0 && tk < a.V;
+            const unsigned ahead = in_vocab ? a.rank_cnt[(size_t)b * R + i] : (unsigned)a.V;
+            p = (float)ahead;
+            rej = (in_vocab && ahead < (unsigned)a.top_k) ? 0 : 1;
+        } else if (mis_s[i] && i + 1 >= R) {
             rej = 1;  // the states that encode the last draft token were not computed: rejected unjudged
         } else if (mis_s[i]) {
             float z = a.judge_b;

@@ -19,7 +19,8 @@ __device__ inline float load_as_float(const __nv_bfloat16 *p, size_t i) { return
 template <typename T>
 __global__ void __launch_bounds__(256) simt_gemm_argmax_kernel(const T *__restrict__ h, const T *__restrict__ W,
                                                                int M, int d, int V, int w_layout, int v_offset,
-                                                               unsigned long long *__restrict__ keys, const Publish pub) {
+                                                               unsigned long long *__restrict__ keys, const Publish pub,
+                                                               const RankArgs rk) {
     const int lane = threadIdx.x & 31;
     const int warps_per_block = blockDim.x >> 5;
     const long long warp = (long long)blockIdx.x * warps_per_block + (threadIdx.x >> 5);
@@ -32,10 +33,16 @@ __global__ void __launch_bounds__(256) simt_gemm_argmax_kernel(const T *__restri
     for (int m0 = 0; m0 < M && v0 < v1; m0 += ROWS) {
         float best[ROWS];
         int bidx[ROWS];
+        unsigned ahead[ROWS];  // top-K rule: entries of this slice that outrank the row's draft token
+        float thr[ROWS];
+        int tok[ROWS];
 #pragma unroll
         for (int r = 0; r < ROWS; r++) {
             best[r] = -INFINITY;
             bidx[r] = v0;
+            ahead[r] = 0;
+            thr[r] = (rk.thr && m0 + r < M) ? rk.thr[m0 + r] : INFINITY;
+            tok[r] = (rk.thr && m0 + r < M) ? rk.tok[m0 + r] : -1;
         }
         for (int v = v0; v < v1; v++) {
             float acc[ROWS];
@@ -59,12 +66,16 @@ __global__ void __launch_bounds__(256) simt_gemm_argmax_kernel(const T *__restri
                     best[r] = s;
                     bidx[r] = v;
                 }
+                if (v != tok[r] && (s > thr[r] || (s == thr[r] && v < tok[r]))) ahead[r]++;
             }
         }
         if (lane == 0) {
 #pragma unroll
             for (int r = 0; r < ROWS; r++)
-                if (m0 + r < M) atomicMax(&keys[m0 + r], pack_key(best[r], bidx[r] + v_offset));
+                if (m0 + r < M) {
+                    atomicMax(&keys[m0 + r], pack_key(best[r], bidx[r] + v_offset));
+                    if (rk.thr && ahead[r]) atomicAdd(rk.cnt + m0 + r, ahead[r]);
+                }
         }
     }
     publish_keys(pub, keys);
@@ -82,10 +93,10 @@ cudaError_t launch_simt_gemm_argmax(const GemmArgs &a, int num_sms, cudaStream_t
     if (blocks < 1) blocks = 1;
     if (a.dtype == 0)
         simt_gemm_argmax_kernel<__nv_bfloat16><<<(unsigned)blocks, threads, 0, stream>>>(
-            (const __nv_bfloat16 *)a.h, (const __nv_bfloat16 *)a.W, a.M, a.d, a.V, a.w_layout, a.v_offset, a.keys, a.pub);
+            (const __nv_bfloat16 *)a.h, (const __nv_bfloat16 *)a.W, a.M, a.d, a.V, a.w_layout, a.v_offset, a.keys, a.pub, a.rank);
     else
         simt_gemm_argmax_kernel<float><<<(unsigned)blocks, threads, 0, stream>>>(
-            (const float *)a.h, (const float *)a.W, a.M, a.d, a.V, a.w_layout, a.v_offset, a.keys, a.pub);
+            (const float *)a.h, (const float *)a.W, a.M, a.d, a.V, a.w_layout, a.v_offset, a.keys, a.pub, a.rank);
     return cudaGetLastError();
 }
 

@@ -48,11 +48,12 @@ template <int BN> struct VCfg {
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + BAR_BYTES + 1024;  // + alignment slack
 };
 
-template <int BN, bool WDV>  // WDV: W is stored [d, V]
+// WDV: W is stored [d, V].  CNT: also count, per row, the entries that outrank the draft token.
+template <int BN, bool WDV, bool CNT>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 umma_vm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_h,
                int M, int V, int d, int n_n, int n_v, int stream_w, int v_offset,
-               unsigned long long *__restrict__ keys, int *__restrict__ status, const Publish pub) {
+               unsigned long long *__restrict__ keys, int *__restrict__ status, const Publish pub, const RankArgs rk) {
     using C = VCfg<BN>;
     constexpr int STAGES = C::STAGES;
     extern __shared__ uint8_t smem_raw[];
@@ -216,6 +217,7 @@ umma_vm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                 if (c * 32 < n_inst) {  // warp-uniform
                     float v[32];
                     tmem_ld32(taddr + c * 32, v);
+                    if (CNT) count_outranking(rk, v, v_first, v_ok, n_tile * BN + c * 32, n_inst - c * 32, M, lane);
                     // all 32 reductions are issued before any result is used, so that their
                     // latencies overlap instead of adding up
                     uint32_t u[32], m[32];
@@ -270,32 +272,34 @@ cudaError_t launch_vm(const GemmArgs &a, const UmmaPlan &p, cudaStream_t stream)
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    auto kernel = a.w_layout ? umma_vm_kernel<BN, true> : umma_vm_kernel<BN, false>;
+    auto kernel = a.rank.thr ? (a.w_layout ? umma_vm_kernel<BN, true, true> : umma_vm_kernel<BN, false, true>)
+                             : (a.w_layout ? umma_vm_kernel<BN, true, false> : umma_vm_kernel<BN, false, false>);
     return cudaLaunchKernelEx(&cfg, kernel, p.tmap_w, p.tmap_h, a.M, a.V, a.d, n_n, n_v, stream_w, a.v_offset, a.keys,
-                              a.status, a.pub);
+                              a.status, a.pub, a.rank);
 }
 
 }  // namespace
 
 int vm_choose_bn(int M) { return M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : 256; }
 
+template <int BN> static cudaError_t set_smem() {
+    const int bytes = VCfg<BN>::SMEM_BYTES;
+    cudaError_t e = cudaFuncSetAttribute(umma_vm_kernel<BN, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(umma_vm_kernel<BN, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(umma_vm_kernel<BN, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(umma_vm_kernel<BN, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    return e;
+}
+
 cudaError_t umma_vm_prepare() {
     cudaError_t e;
-    e = cudaFuncSetAttribute(umma_vm_kernel<32, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, VCfg<32>::SMEM_BYTES);
+    e = set_smem<32>();
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(umma_vm_kernel<32, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, VCfg<32>::SMEM_BYTES);
+    e = set_smem<64>();
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(umma_vm_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, VCfg<64>::SMEM_BYTES);
+    e = set_smem<128>();
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(umma_vm_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, VCfg<64>::SMEM_BYTES);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(umma_vm_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, VCfg<128>::SMEM_BYTES);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(umma_vm_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, VCfg<128>::SMEM_BYTES);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(umma_vm_kernel<256, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, VCfg<256>::SMEM_BYTES);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(umma_vm_kernel<256, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, VCfg<256>::SMEM_BYTES);
+    e = set_smem<256>();
     return e;
 }
 

@@ -116,3 +116,30 @@ def test_c2_with_the_lm_head_stored_d_by_v_gives_the_same_bits():
     finally:
         a.close()
         b.close()
+
+
+def test_c2_under_the_top_k_rule():
+    """The batch-1 8B shape under the top-K rule (k = 1, 8, 1000): ranks over the full vocabulary."""
+    orc = _orc()
+    cfg = gen.C2
+    Wh, Wd = _W(cfg)
+    ht, hd = gen.make_hidden(cfg)
+    w = gen.make_judge(cfg)
+    y = np.stack([[orc.argmax(r)[0] for r in orc.logits(ht[b], Wh, cfg.dtype)] for b in range(cfg.B)])
+    tok = gen.plant_draft_tokens(cfg, y)
+    case = DeviceCase(cfg, Wd, ht, hd, w)
+    try:
+        for k in (1, 8, 1000):
+            case.handle.set_top_k(k)
+            o = orc.verify_topk(ht, Wh, tok, k, cfg.dtype, band=1e-2)
+            g = case.run(tok, 0.5)
+            assert g.path == "umma_vm_128x32" and g.launches == 3
+            np.testing.assert_array_equal(g.target_tok, o.target_tok)
+            mism = o.rank[0] >= 0
+            assert (np.abs(g.judge_p[0][mism] - o.rank[0][mism]) <= o.near[0][mism]).all()
+            n = int(o.accept_len[0])
+            shaky = (mism[: n + 1] & (np.abs(o.rank[0][: n + 1] - k) <= o.near[0][: n + 1]) & (o.near[0][: n + 1] > 0)).any()
+            if not shaky:
+                assert g.accept_len[0] == n and g.next_tok[0] == o.next_tok[0]
+    finally:
+        case.close()

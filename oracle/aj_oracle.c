@@ -33,6 +33,15 @@
  * the classifier, and when all K positions pass there is no row to predict a further token from
  * (next_tok = -1).
  *
+ * Sampling (Appendix A, "Generalization to sampling"): the target's token is drawn by the Gumbel-max
+ * trick, token = argmax_v (logit[v] + T * g[v]) with g standard Gumbel noise that is a deterministic
+ * function of a random state, so that the draw is reproducible; with temperature T this samples from
+ * softmax(logit / T).  The noise for row j (row index within the call), vocabulary entry v, cycle
+ * counter `step` and 64-bit `seed` is defined here as: x = word (j mod 4) of Philox4x32-10 with key
+ * (seed low, seed high) and counter (v, j div 4, step low, step high); u = ((x >> 9) + 0.5) * 2^-23;
+ * g = -ln(-ln(u)).  Everything downstream (mismatch test, classifier, prefix walk) uses the drawn
+ * token in place of the greedy one.  T = 0 is greedy verification.
+ *
  * Top-K rule (Section 4.1, the lossy baseline the paper compares with): instead of consulting the
  * classifier, a mismatching draft token is accepted iff it is among the top_k most likely tokens of
  * the target, i.e. iff its rank (number of vocabulary entries with a larger logit; among equal
@@ -75,6 +84,35 @@ int ajo_num_threads(void)
 #else
     return 1;
 #endif
+}
+
+/* Philox4x32-10 (Salmon, Moraes, Dror, Shaw: "Parallel random numbers: as easy as 1, 2, 3", 2011) */
+void ajo_philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4])
+{
+    uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3], k0 = key[0], k1 = key[1];
+    for (int r = 0; r < 10; r++) {
+        uint64_t p0 = (uint64_t)0xD2511F53u * c0, p1 = (uint64_t)0xCD9E8D57u * c2;
+        uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0, n1 = (uint32_t)p1;
+        uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1, n3 = (uint32_t)p0;
+        c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+        k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+/* the uniform variate in (0,1) behind the noise of (row j, entry v): exactly representable in fp32 */
+double ajo_noise_uniform(uint64_t seed, uint64_t step, int j, int v)
+{
+    uint32_t ctr[4] = {(uint32_t)v, (uint32_t)(j >> 2), (uint32_t)step, (uint32_t)(step >> 32)};
+    uint32_t key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)}, out[4];
+    ajo_philox4x32_10(ctr, key, out);
+    return ((double)(out[j & 3] >> 9) + 0.5) * (1.0 / 8388608.0);
+}
+
+/* standard Gumbel noise of (row j, entry v) */
+double ajo_gumbel(uint64_t seed, uint64_t step, int j, int v)
+{
+    return -log(-log(ajo_noise_uniform(seed, step, j, v)));
 }
 
 /*
@@ -171,11 +209,33 @@ static int forgiven(double p, float tau)
  *   accept_len [B], next_tok [B], target_tok [B][R], top1 [B][R], gap [B][R],
  *   judge_p [B][K]  (p at every mismatching position whose features exist, NaN elsewhere).
  */
+int ajo_verify_sampled(const void *h_target, const void *h_draft, const void *W,
+                       const int32_t *draft_tok, const float *judge_w, float judge_b, float tau,
+                       int dtype, int w_layout, int B, int K, int d, int d_draft, int V, int extra_row,
+                       double temperature, uint64_t seed, uint64_t step,
+                       int32_t *accept_len, int32_t *next_tok, int32_t *target_tok,
+                       double *top1, double *gap, double *judge_p);
+
 int ajo_verify(const void *h_target, const void *h_draft, const void *W,
                const int32_t *draft_tok, const float *judge_w, float judge_b, float tau,
                int dtype, int w_layout, int B, int K, int d, int d_draft, int V, int extra_row,
                int32_t *accept_len, int32_t *next_tok, int32_t *target_tok,
                double *top1, double *gap, double *judge_p)
+{
+    return ajo_verify_sampled(h_target, h_draft, W, draft_tok, judge_w, judge_b, tau, dtype, w_layout, B, K, d, d_draft,
+                              V, extra_row, 0.0, 0, 0, accept_len, next_tok, target_tok, top1, gap, judge_p);
+}
+
+/*
+ * The whole step with the target's tokens drawn by the Gumbel-max trick at the given temperature
+ * (0 = greedy); top1 and gap then refer to the noisy scores logit + temperature * g.
+ */
+int ajo_verify_sampled(const void *h_target, const void *h_draft, const void *W,
+                       const int32_t *draft_tok, const float *judge_w, float judge_b, float tau,
+                       int dtype, int w_layout, int B, int K, int d, int d_draft, int V, int extra_row,
+                       double temperature, uint64_t seed, uint64_t step,
+                       int32_t *accept_len, int32_t *next_tok, int32_t *target_tok,
+                       double *top1, double *gap, double *judge_p)
 {
     if (!h_target || !W || !draft_tok || !judge_w || B < 1 || K < 1 || d < 1 || V < 1 ||
         d_draft < 0 || (d_draft > 0 && !h_draft))
@@ -190,6 +250,12 @@ int ajo_verify(const void *h_target, const void *h_draft, const void *W,
         const char *hdr = h_draft ? (const char *)h_draft + (size_t)b * R * d_draft * esz : NULL;
         int rc = ajo_logits(ht, W, dtype, w_layout, R, d, V, logits);
         if (rc) { free(logits); return rc; }
+        if (temperature > 0.0) {
+#pragma omp parallel for schedule(static)
+            for (int v = 0; v < V; v++)
+                for (int j = 0; j < R; j++)
+                    logits[(size_t)j * V + v] += temperature * ajo_gumbel(seed, step, b * R + j, v);
+        }
 
         int32_t *y = target_tok + (size_t)b * R;
         for (int j = 0; j < R; j++)

@@ -66,6 +66,16 @@ def _lib():
         L.ajo_judge_p.restype = ctypes.c_double
         L.ajo_verify.argtypes = [vp, vp, vp, ip, fp, cf, cf, ci, ci, ci, ci, ci, ci, ci, ci, ip, ip, ip, dp, dp, dp]
         L.ajo_verify.restype = ci
+        u64 = ctypes.c_uint64
+        L.ajo_verify_sampled.argtypes = [vp, vp, vp, ip, fp, cf, cf, ci, ci, ci, ci, ci, ci, ci, ci, ctypes.c_double, u64, u64,
+                                         ip, ip, ip, dp, dp, dp]
+        L.ajo_verify_sampled.restype = ci
+        L.ajo_philox4x32_10.argtypes = [vp, vp, vp]
+        L.ajo_philox4x32_10.restype = None
+        L.ajo_noise_uniform.argtypes = [u64, u64, ci, ci]
+        L.ajo_noise_uniform.restype = ctypes.c_double
+        L.ajo_gumbel.argtypes = [u64, u64, ci, ci]
+        L.ajo_gumbel.restype = ctypes.c_double
         L.ajo_rank.argtypes = [dp, ci, ci, ctypes.c_double, ip]
         L.ajo_rank.restype = ci
         L.ajo_verify_topk.argtypes = [vp, vp, ip, ci, ctypes.c_double, ci, ci, ci, ci, ci, ci, ip, ip, ip, dp, dp, ip, ip]
@@ -134,8 +144,25 @@ class OracleResult:
     judge_p: np.ndarray  # [B, K] float64, NaN where the draft token matched
 
 
+def philox4x32_10(ctr, key):
+    """Philox4x32-10: four 32-bit counter words and two key words in, four words out."""
+    c = np.asarray(ctr, dtype=np.uint32)
+    k = np.asarray(key, dtype=np.uint32)
+    out = np.empty(4, dtype=np.uint32)
+    _lib().ajo_philox4x32_10(_ptr(c), _ptr(k), _ptr(out))
+    return out
+
+
+def noise_uniform(seed: int, step: int, j: int, v: int) -> float:
+    return float(_lib().ajo_noise_uniform(seed, step, j, v))
+
+
+def gumbel(seed: int, step: int, j: int, v: int) -> float:
+    return float(_lib().ajo_gumbel(seed, step, j, v))
+
+
 def verify(h_target, h_draft, W, draft_tok, judge_w, judge_b, tau, dtype: int, w_layout: int = 0,
-           extra_row: bool = True) -> OracleResult:
+           extra_row: bool = True, temperature: float = 0.0, seed: int = 0, step: int = 0) -> OracleResult:
     """The whole verify-and-judge step for B sequences (see aj_oracle.c for the definition).
 
     extra_row=False: the hidden states have K rows, not K + 1 (the last draft token is not encoded)."""
@@ -154,9 +181,9 @@ def verify(h_target, h_draft, W, draft_tok, judge_w, judge_b, tau, dtype: int, w
         np.empty(B, np.int32), np.empty(B, np.int32), np.empty((B, R), np.int32),
         np.empty((B, R), np.float64), np.empty((B, R), np.float64), np.empty((B, K), np.float64),
     )
-    rc = _lib().ajo_verify(
+    rc = _lib().ajo_verify_sampled(
         _ptr(ht), _ptr(hd), _ptr(W), _ptr(tok), _ptr(w), float(judge_b), float(tau), dtype, w_layout,
-        B, K, d, dd, V, 1 if extra_row else 0, _ptr(res.accept_len), _ptr(res.next_tok), _ptr(res.target_tok),
+        B, K, d, dd, V, 1 if extra_row else 0, float(temperature), int(seed), int(step), _ptr(res.accept_len), _ptr(res.next_tok), _ptr(res.target_tok),
         _ptr(res.top1), _ptr(res.gap), _ptr(res.judge_p),
     )
     if rc:

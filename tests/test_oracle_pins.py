@@ -421,3 +421,61 @@ def test_top_k_rule_extremes_monotonicity_and_brute_force(dtype):
         prev = r.accept_len.copy()
     r = orc.verify_topk(ht, W, tok, V, dtype)
     assert r.accept_len[0] == 2 and r.accept_len[1] == 1 and r.rank[0, 2] == V
+
+
+# ------------------------------------------------------ sampling by the Gumbel-max trick (Appendix A)
+
+
+def test_philox_known_answers():
+    """Known-answer vectors of Philox4x32-10 as published with the Random123 library."""
+    kat = [((0, 0, 0, 0), (0, 0), (0x6627E8D5, 0xE169C58D, 0xBC57AC4C, 0x9B00DBD8)),
+           ((0x243F6A88, 0x85A308D3, 0x13198A2E, 0x03707344), (0xA4093822, 0x299F31D0),
+            (0xD16CFE09, 0x94FDCCEB, 0x5001E420, 0x24126EA1))]
+    for ctr, key, want in kat:
+        assert tuple(int(x) for x in orc.philox4x32_10(ctr, key)) == want
+
+
+def test_noise_is_a_uniform_in_the_open_interval_and_exact_in_fp32():
+    us = np.array([orc.noise_uniform(7, 3, j, v) for j in range(8) for v in range(500)])
+    assert (us > 0).all() and (us < 1).all()
+    assert (us.astype(np.float32).astype(np.float64) == us).all()
+    assert 0.45 < us.mean() < 0.55 and len(np.unique(us)) > 3990
+    # rows 4q .. 4q+3 take the four words of one Philox call, and every argument matters
+    base = orc.noise_uniform(7, 3, 5, 11)
+    assert base == orc.noise_uniform(7, 3, 5, 11)
+    assert len({base, orc.noise_uniform(8, 3, 5, 11), orc.noise_uniform(7, 4, 5, 11), orc.noise_uniform(7, 3, 6, 11),
+                orc.noise_uniform(7, 3, 5, 12), orc.noise_uniform(7 + (1 << 32), 3, 5, 11), orc.noise_uniform(7, 3 + (1 << 32), 5, 11)}) == 7
+    w = orc.philox4x32_10((11, 1, 3, 0), (7, 0))
+    assert base == (float(int(w[1]) >> 9) + 0.5) / 8388608.0
+    assert orc.gumbel(7, 3, 5, 11) == pytest.approx(-np.log(-np.log(base)), rel=1e-15)
+
+
+def test_gumbel_max_draws_follow_the_softmax_and_zero_temperature_is_greedy():
+    """Appendix A: adding independent Gumbel noise to the logits and taking the argmax draws an index with
+    the softmax probabilities; at temperature T the distribution is softmax(logit / T)."""
+    V, d, T = 6, 8, 0.7
+    cfg = gen.Config("gumbel", B=1, K=3, d=d, d_draft=0, V=V, dtype=F32, sigma_W=0.6, seed=71)
+    W = gen.make_W(cfg)
+    ht, _ = gen.make_hidden(cfg)
+    w = gen.make_judge(cfg)
+    tok = np.zeros((1, 3), np.int32)
+    lg = orc.logits(ht[0], W, F32)                               # [4, V]
+    greedy = orc.verify(ht, None, W, tok, w, 0.0, 0.5, F32)
+    np.testing.assert_array_equal(greedy.target_tok[0], lg.argmax(1))
+    again = orc.verify(ht, None, W, tok, w, 0.0, 0.5, F32, temperature=0.0, seed=99, step=5)
+    np.testing.assert_array_equal(again.target_tok, greedy.target_tok)   # T = 0 ignores the random state
+    n = 6000
+    counts = np.zeros((4, V))
+    for step in range(n):
+        r = orc.verify(ht, None, W, tok, w, 0.0, 0.5, F32, temperature=T, seed=2024, step=step)
+        for j in range(4):
+            counts[j, r.target_tok[0, j]] += 1
+    p = np.exp(lg / T)
+    p /= p.sum(1, keepdims=True)
+    chi2 = ((counts - n * p) ** 2 / (n * p)).sum(1)              # 5 degrees of freedom per row
+    assert (chi2 < 25.0).all(), chi2                             # P(chi2_5 > 25) = 1.4e-4
+    same = orc.verify(ht, None, W, tok, w, 0.0, 0.5, F32, temperature=T, seed=2024, step=17)
+    np.testing.assert_array_equal(same.target_tok, orc.verify(ht, None, W, tok, w, 0.0, 0.5, F32, temperature=T, seed=2024, step=17).target_tok)
+    # the reported winner is the noisy score
+    j, y = 2, int(same.target_tok[0, 2])
+    assert same.top1[0, j] == pytest.approx(lg[j, y] + T * orc.gumbel(2024, 17, j, y), abs=1e-12)

@@ -124,6 +124,27 @@ aj_status aj_verify(aj_handle h, const void *h_target, const void *h_draft, cons
 aj_status aj_set_top_k(aj_handle h, int top_k);
 
 /*
+ * Sampled verification (the paper's Appendix A, "Generalization to sampling"): the target's token of
+ * every row is drawn from softmax(logit / temperature) instead of being the greedy argmax, by the
+ * Gumbel-max trick with noise that is a deterministic function of the random state, so that a draw
+ * can be reproduced: token = argmax_v (logit[v] + temperature * g[v]).  For row j of the call
+ * (j = b * rows per sequence + position) and vocabulary entry v:
+ *     x = word (j mod 4) of Philox4x32-10 with key (seed low word, seed high word) and counter
+ *         (v, j div 4, step low word, step high word);
+ *     u = ((x >> 9) + 0.5) * 2^-23;   g = -ln(-ln u)      (fp32 on the device).
+ * The noise is added in the projection kernels' epilogues before the argmax; logits are still never
+ * written.  Everything downstream (mismatch test, classifier, accepted prefix, next token) uses the
+ * drawn tokens; top1_val receives the winning noisy score.  `step` is the cycle counter of the next
+ * cycle enqueued on the handle and advances by one with every cycle, so that consecutive cycles
+ * draw independent noise; set it again to replay a cycle.  The draw does not depend on the kernel
+ * chosen, on tiling or on vocabulary sharding (the ranks of a vocabulary-parallel group must be
+ * given the same temperature, seed and step).  temperature = 0 switches back to greedy
+ * verification.  Errors: AJ_ERR_INVALID_ARG (NULL handle, negative or non-finite temperature),
+ * AJ_ERR_UNSUPPORTED (together with the top-K rule, or with AJ_FLAG_ROW_TILES).
+ */
+aj_status aj_set_sampling(aj_handle h, float temperature, uint64_t seed, uint64_t step);
+
+/*
  * The same cycle for a caller whose per-cycle tensors live in host memory: h_target, h_draft and
  * draft_tok are HOST pointers and are copied to the handle's staging buffers; accept_len and
  * next_tok (and target_tok, if not NULL) are HOST pointers and are copied back.  W_lm and judge_w

@@ -19,7 +19,7 @@ AJ_FLAG_FORCE_SIMT, AJ_FLAG_TIME_KERNELS, AJ_FLAG_ROW_TILES, AJ_FLAG_ONE_SM, AJ_
 
 EXPORTS = (
     "aj_create", "aj_verify", "aj_verify_host", "aj_last_status", "aj_last_gemm_ms", "aj_gemm_ms_stats", "aj_last_launch_count",
-    "aj_last_gemm_path", "aj_pair_schedule", "aj_destroy", "aj_set_top_k", "aj_shard_exchange_bytes", "aj_shard_exchange_alloc", "aj_shard_exchange_free", "aj_shard_range", "aj_create_sharded",
+    "aj_last_gemm_path", "aj_pair_schedule", "aj_destroy", "aj_set_top_k", "aj_set_sampling", "aj_shard_exchange_bytes", "aj_shard_exchange_alloc", "aj_shard_exchange_free", "aj_shard_range", "aj_create_sharded",
     "aj_shard_project", "aj_shard_finish", "aj_ipc_export", "aj_ipc_import", "aj_ipc_close", "aj_status_string", "aj_version", "aj_verify_static",
 )
 
@@ -89,6 +89,8 @@ def lib() -> ctypes.CDLL:
         L.aj_ipc_close.restype = ci
         L.aj_set_top_k.argtypes = [vp, ci]
         L.aj_set_top_k.restype = ci
+        L.aj_set_sampling.argtypes = [vp, ctypes.c_float, ctypes.c_uint64, ctypes.c_uint64]
+        L.aj_set_sampling.restype = ci
         L.aj_version.argtypes = []
         L.aj_version.restype = ctypes.c_char_p
         _lib = L
@@ -261,6 +263,14 @@ class Handle:
         st = lib().aj_set_top_k(self._h, int(top_k))
         if check and st != AJ_OK:
             raise AjError(st, "aj_set_top_k")
+        return st
+
+    def set_sampling(self, temperature: float, seed: int = 0, step: int = 0, check: bool = True) -> int:
+        """aj_set_sampling: draw the target's tokens from softmax(logit / temperature) by the Gumbel-max trick
+        (0: back to greedy); `step` is the next cycle's counter and advances by one per cycle."""
+        st = lib().aj_set_sampling(self._h, float(temperature), int(seed) & (2**64 - 1), int(step) & (2**64 - 1))
+        if check and st != AJ_OK:
+            raise AjError(st, "aj_set_sampling")
         return st
 
     def last_status(self) -> int:

@@ -58,6 +58,9 @@ struct aj_handle_s {
     bool projected = false;          // aj_shard_project was enqueued and its aj_shard_finish is still due
     // top-K rule (aj_set_top_k)
     int top_k = 0;                   // 0: the classifier decides
+    // sampled verification (aj_set_sampling)
+    float temperature = 0.0f;        // 0: greedy
+    unsigned long long seed = 0, step = 0;
     float *rk_thr = nullptr;         // [max_M] the draft tokens' own logits
     int *rk_tok = nullptr;           // [max_M]
     unsigned *rk_cnt = nullptr;      // [max_M] entries that outrank them
@@ -310,6 +313,14 @@ static aj_status enqueue_project(aj_handle h, const void *h_target, const void *
         g.rank.thr = h->rk_thr;
         g.rank.tok = h->rk_tok;
         g.rank.cnt = h->rk_cnt;
+    }
+    if (h->temperature > 0.0f) {
+        g.noise.temperature = h->temperature;
+        g.noise.key0 = (uint32_t)h->seed;
+        g.noise.key1 = (uint32_t)(h->seed >> 32);
+        g.noise.step0 = (uint32_t)h->step;
+        g.noise.step1 = (uint32_t)(h->step >> 32);
+        ++h->step;
     }
     g.h = h_target;
     g.W = W_lm;
@@ -675,7 +686,18 @@ aj_status aj_set_top_k(aj_handle h, int top_k) {
     if (!h || top_k < 0) return AJ_ERR_INVALID_ARG;
     // the count is kept per GPU and the row-tile kernel does not produce it
     if (top_k > 0 && (h->world || (h->flags & (AJ_FLAG_ROW_TILES | AJ_FLAG_NO_EXTRA_ROW)))) return AJ_ERR_UNSUPPORTED;
+    if (top_k > 0 && h->temperature > 0.0f) return AJ_ERR_UNSUPPORTED;  // the rule ranks the plain logits
     h->top_k = top_k;
+    return AJ_OK;
+}
+
+aj_status aj_set_sampling(aj_handle h, float temperature, uint64_t seed, uint64_t step) {
+    if (!h || !(temperature >= 0.0f) || !(temperature <= 3.0e38f)) return AJ_ERR_INVALID_ARG;
+    // the row-tile kernel's epilogue does not add the noise
+    if (temperature > 0.0f && (h->top_k > 0 || (h->flags & AJ_FLAG_ROW_TILES))) return AJ_ERR_UNSUPPORTED;
+    h->temperature = temperature;
+    h->seed = seed;
+    h->step = step;
     return AJ_OK;
 }
 

@@ -148,6 +148,66 @@ __device__ inline void count_outranking(const RankArgs &rk, const float (&v)[32]
 }
 #endif
 
+// ------------------------------------------------------- sampling by the Gumbel-max trick
+//
+// With a temperature T > 0 the target's token of a row is argmax_v (logit[v] + T * g[v]) with g
+// standard Gumbel noise, which draws from softmax(logit / T); the noise is a deterministic
+// function of (seed, cycle counter, row, vocabulary entry), so that a draw can be reproduced and
+// does not depend on how the work was tiled or sharded.  For row j and entry v: x = word (j mod 4)
+// of Philox4x32-10 with key (seed low, seed high) and counter (v, j div 4, step low, step high);
+// u = ((x >> 9) + 0.5) * 2^-23 (exact in fp32, never 0 or 1); g = -ln(-ln u).
+struct Noise {
+    float temperature = 0.0f;  // 0: greedy, no noise
+    uint32_t key0 = 0, key1 = 0;    // seed
+    uint32_t step0 = 0, step1 = 0;  // cycle counter
+};
+
+#ifdef __CUDACC__
+__device__ inline void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0, uint32_t k1,
+                                     uint32_t (&out)[4]) {
+#pragma unroll
+    for (int r = 0; r < 10; r++) {
+        const uint32_t h0 = __umulhi(0xD2511F53u, c0), l0 = 0xD2511F53u * c0;
+        const uint32_t h1 = __umulhi(0xCD9E8D57u, c2), l1 = 0xCD9E8D57u * c2;
+        c0 = h1 ^ c1 ^ k0;
+        c1 = l1;
+        c2 = h0 ^ c3 ^ k1;
+        c3 = l0;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    out[0] = c0;
+    out[1] = c1;
+    out[2] = c2;
+    out[3] = c3;
+}
+
+__device__ inline float gumbel_from_bits(uint32_t x) {
+    const float u = ((float)(x >> 9) + 0.5f) * 1.1920928955078125e-07f;  // 2^-23
+    return -logf(-logf(u));
+}
+
+// The noisy score of one element.
+__device__ inline float noisy_score(const Noise &nz, float logit, int row, int v) {
+    uint32_t w[4];
+    philox4x32_10((uint32_t)v, (uint32_t)(row >> 2), nz.step0, nz.step1, nz.key0, nz.key1, w);
+    const uint32_t x = (row & 2) ? ((row & 1) ? w[3] : w[2]) : ((row & 1) ? w[1] : w[0]);
+    return fmaf(nz.temperature, gumbel_from_bits(x), logit);
+}
+
+// Epilogue add-on for the vocabulary-major kernels: this thread holds entry v of the 32 rows
+// row_first .. + 32 (row_first a multiple of 4) in x[]; one Philox call serves four rows.
+__device__ inline void add_gumbel_noise(const Noise &nz, float (&x)[32], int v, int row_first) {
+#pragma unroll
+    for (int q = 0; q < 8; q++) {
+        uint32_t w[4];
+        philox4x32_10((uint32_t)v, (uint32_t)((row_first >> 2) + q), nz.step0, nz.step1, nz.key0, nz.key1, w);
+#pragma unroll
+        for (int i = 0; i < 4; i++) x[4 * q + i] = fmaf(nz.temperature, gumbel_from_bits(w[i]), x[4 * q + i]);
+    }
+}
+#endif
+
 struct RankPrepArgs {
     const void *h;             // [M, d]
     const void *W;             // LM head
@@ -172,7 +232,11 @@ struct GemmArgs {
     int *status;
     Publish pub;
     RankArgs rank;       // thr != nullptr: also count, per row, the entries that outrank the draft token
+    Noise noise;         // temperature > 0: the argmax is taken over logit + temperature * Gumbel noise
 };
+
+// What a projection kernel's epilogue does besides the argmax.
+enum : int { EPI_PLAIN = 0, EPI_COUNT = 1, EPI_SAMPLE = 2 };
 
 // CUDA-core projection + argmax (any dtype / layout).
 cudaError_t launch_simt_gemm_argmax(const GemmArgs &a, int num_sms, cudaStream_t stream);

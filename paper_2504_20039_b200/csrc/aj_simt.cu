@@ -20,7 +20,7 @@ template <typename T>
 __global__ void __launch_bounds__(256) simt_gemm_argmax_kernel(const T *__restrict__ h, const T *__restrict__ W,
                                                                int M, int d, int V, int w_layout, int v_offset,
                                                                unsigned long long *__restrict__ keys, const Publish pub,
-                                                               const RankArgs rk) {
+                                                               const RankArgs rk, const Noise nz) {
     const int lane = threadIdx.x & 31;
     const int warps_per_block = blockDim.x >> 5;
     const long long warp = (long long)blockIdx.x * warps_per_block + (threadIdx.x >> 5);
@@ -62,6 +62,7 @@ __global__ void __launch_bounds__(256) simt_gemm_argmax_kernel(const T *__restri
                 float s = acc[r];
 #pragma unroll
                 for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
+                if (nz.temperature > 0.0f) s = noisy_score(nz, s, min(m0 + r, M - 1), v + v_offset);
                 if (s > best[r]) {  // strict: the first (lowest) index keeps a tie
                     best[r] = s;
                     bidx[r] = v;
@@ -93,10 +94,11 @@ cudaError_t launch_simt_gemm_argmax(const GemmArgs &a, int num_sms, cudaStream_t
     if (blocks < 1) blocks = 1;
     if (a.dtype == 0)
         simt_gemm_argmax_kernel<__nv_bfloat16><<<(unsigned)blocks, threads, 0, stream>>>(
-            (const __nv_bfloat16 *)a.h, (const __nv_bfloat16 *)a.W, a.M, a.d, a.V, a.w_layout, a.v_offset, a.keys, a.pub, a.rank);
+            (const __nv_bfloat16 *)a.h, (const __nv_bfloat16 *)a.W, a.M, a.d, a.V, a.w_layout, a.v_offset, a.keys, a.pub, a.rank,
+            a.noise);
     else
         simt_gemm_argmax_kernel<float><<<(unsigned)blocks, threads, 0, stream>>>(
-            (const float *)a.h, (const float *)a.W, a.M, a.d, a.V, a.w_layout, a.v_offset, a.keys, a.pub, a.rank);
+            (const float *)a.h, (const float *)a.W, a.M, a.d, a.V, a.w_layout, a.v_offset, a.keys, a.pub, a.rank, a.noise);
     return cudaGetLastError();
 }
 

@@ -87,12 +87,14 @@ __device__ inline Tile decode_tile(const PairSched &sc, int t) {
 }
 
 // DUAL: every tile uses two accumulators that share the staged block of W.  WDV: W is stored [d, V].
-// CNT: also count, per row, the entries that outrank the draft token (top-K rule).
-template <bool DUAL, bool WDV, bool CNT>
+// EPI: EPI_COUNT also counts, per row, the entries that outrank the draft token (top-K rule);
+// EPI_SAMPLE adds Gumbel noise to the logits before the argmax.
+template <bool DUAL, bool WDV, int EPI>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_h,
                  int M, int V, int d, PairSched sc, int stream_w, int v_offset,
-                 unsigned long long *__restrict__ keys, int *__restrict__ status, const Publish pub, const RankArgs rk) {
+                 unsigned long long *__restrict__ keys, int *__restrict__ status, const Publish pub, const RankArgs rk,
+                 const Noise nz) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;  // the same offset in both CTAs: one descriptor serves both
@@ -290,8 +292,9 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
                         const float thr = cur[u];
                         float v[32];
                         tmem_ld32(tbase + (uint32_t)((DUAL ? a : slot) * BN + c * 32), v);
-                        if (CNT)
+                        if (EPI == EPI_COUNT)
                             count_outranking(rk, v, v_first, v_ok, (a ? tl.row0[1] : tl.row0[0]) + c * 32, n_inst - c * 32, M, lane);
+                        if (EPI == EPI_SAMPLE) add_gumbel_noise(nz, v, v_first + lane + v_offset, (a ? tl.row0[1] : tl.row0[0]) + c * 32);
                         bool hit = false;
 #pragma unroll
                         for (int j = 0; j < 32; j++) hit |= v[j] >= __shfl_sync(0xffffffffu, thr, j);
@@ -349,10 +352,13 @@ int g_max_pairs = 0;
 
 cudaError_t umma_pair_prepare(int num_sms) {
     cudaError_t e = cudaSuccess;
-    const void *kernels[8] = {(const void *)umma_pair_kernel<false, false, false>, (const void *)umma_pair_kernel<true, false, false>,
-                              (const void *)umma_pair_kernel<false, true, false>,  (const void *)umma_pair_kernel<true, true, false>,
-                              (const void *)umma_pair_kernel<false, false, true>,  (const void *)umma_pair_kernel<true, false, true>,
-                              (const void *)umma_pair_kernel<false, true, true>,   (const void *)umma_pair_kernel<true, true, true>};
+    const void *kernels[12] = {
+        (const void *)umma_pair_kernel<false, false, EPI_PLAIN>,  (const void *)umma_pair_kernel<true, false, EPI_PLAIN>,
+        (const void *)umma_pair_kernel<false, true, EPI_PLAIN>,   (const void *)umma_pair_kernel<true, true, EPI_PLAIN>,
+        (const void *)umma_pair_kernel<false, false, EPI_COUNT>,  (const void *)umma_pair_kernel<true, false, EPI_COUNT>,
+        (const void *)umma_pair_kernel<false, true, EPI_COUNT>,   (const void *)umma_pair_kernel<true, true, EPI_COUNT>,
+        (const void *)umma_pair_kernel<false, false, EPI_SAMPLE>, (const void *)umma_pair_kernel<true, false, EPI_SAMPLE>,
+        (const void *)umma_pair_kernel<false, true, EPI_SAMPLE>,  (const void *)umma_pair_kernel<true, true, EPI_SAMPLE>};
     for (const void *k : kernels) {
         e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
         if (e != cudaSuccess) return e;
@@ -370,7 +376,7 @@ cudaError_t umma_pair_prepare(int num_sms) {
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     int clusters = 0;
-    e = cudaOccupancyMaxActiveClusters(&clusters, umma_pair_kernel<false, false, false>, &cfg);
+    e = cudaOccupancyMaxActiveClusters(&clusters, umma_pair_kernel<false, false, EPI_PLAIN>, &cfg);
     if (e != cudaSuccess) return e;
     if (clusters < 1) return cudaErrorInvalidConfiguration;
     g_max_pairs = clusters < num_sms / 2 ? clusters : num_sms / 2;
@@ -427,14 +433,16 @@ cudaError_t launch_umma_pair(const GemmArgs &a, const UmmaPlan &p, cudaStream_t 
     attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
-    auto pick = [&](auto cnt) {
-        constexpr bool C = decltype(cnt)::value;
-        return sc.dual ? (a.w_layout ? umma_pair_kernel<true, true, C> : umma_pair_kernel<true, false, C>)
-                       : (a.w_layout ? umma_pair_kernel<false, true, C> : umma_pair_kernel<false, false, C>);
+    auto pick = [&](auto epi) {
+        constexpr int E = decltype(epi)::value;
+        return sc.dual ? (a.w_layout ? umma_pair_kernel<true, true, E> : umma_pair_kernel<true, false, E>)
+                       : (a.w_layout ? umma_pair_kernel<false, true, E> : umma_pair_kernel<false, false, E>);
     };
-    auto kernel = a.rank.thr ? pick(std::true_type{}) : pick(std::false_type{});
+    auto kernel = a.noise.temperature > 0.0f ? pick(std::integral_constant<int, EPI_SAMPLE>{})
+                  : a.rank.thr               ? pick(std::integral_constant<int, EPI_COUNT>{})
+                                             : pick(std::integral_constant<int, EPI_PLAIN>{});
     return cudaLaunchKernelEx(&cfg, kernel, p.tmap_w, p.tmap_h, a.M, a.V, a.d, sc, stream_w, a.v_offset, a.keys, a.status,
-                              a.pub, a.rank);
+                              a.pub, a.rank, a.noise);
 }
 
 }  // namespace aj

@@ -26,6 +26,8 @@
 #include "aj_internal.cuh"
 #include "aj_ptx.cuh"
 
+#include <type_traits>
+
 namespace aj {
 
 namespace {
@@ -48,12 +50,14 @@ template <int BN> struct VCfg {
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + BAR_BYTES + 1024;  // + alignment slack
 };
 
-// WDV: W is stored [d, V].  CNT: also count, per row, the entries that outrank the draft token.
-template <int BN, bool WDV, bool CNT>
+// WDV: W is stored [d, V].  EPI: EPI_COUNT also counts, per row, the entries that outrank the draft
+// token; EPI_SAMPLE adds Gumbel noise to the logits before the argmax.
+template <int BN, bool WDV, int EPI>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 umma_vm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_h,
                int M, int V, int d, int n_n, int n_v, int stream_w, int v_offset,
-               unsigned long long *__restrict__ keys, int *__restrict__ status, const Publish pub, const RankArgs rk) {
+               unsigned long long *__restrict__ keys, int *__restrict__ status, const Publish pub, const RankArgs rk,
+               const Noise nz) {
     using C = VCfg<BN>;
     constexpr int STAGES = C::STAGES;
     extern __shared__ uint8_t smem_raw[];
@@ -217,7 +221,8 @@ umma_vm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                 if (c * 32 < n_inst) {  // warp-uniform
                     float v[32];
                     tmem_ld32(taddr + c * 32, v);
-                    if (CNT) count_outranking(rk, v, v_first, v_ok, n_tile * BN + c * 32, n_inst - c * 32, M, lane);
+                    if (EPI == EPI_COUNT) count_outranking(rk, v, v_first, v_ok, n_tile * BN + c * 32, n_inst - c * 32, M, lane);
+                    if (EPI == EPI_SAMPLE) add_gumbel_noise(nz, v, v_first + lane + v_offset, n_tile * BN + c * 32);
                     // all 32 reductions are issued before any result is used, so that their
                     // latencies overlap instead of adding up
                     uint32_t u[32], m[32];
@@ -272,10 +277,15 @@ cudaError_t launch_vm(const GemmArgs &a, const UmmaPlan &p, cudaStream_t stream)
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    auto kernel = a.rank.thr ? (a.w_layout ? umma_vm_kernel<BN, true, true> : umma_vm_kernel<BN, false, true>)
-                             : (a.w_layout ? umma_vm_kernel<BN, true, false> : umma_vm_kernel<BN, false, false>);
+    auto pick = [&](auto epi) {
+        constexpr int E = decltype(epi)::value;
+        return a.w_layout ? umma_vm_kernel<BN, true, E> : umma_vm_kernel<BN, false, E>;
+    };
+    auto kernel = a.noise.temperature > 0.0f ? pick(std::integral_constant<int, EPI_SAMPLE>{})
+                  : a.rank.thr               ? pick(std::integral_constant<int, EPI_COUNT>{})
+                                             : pick(std::integral_constant<int, EPI_PLAIN>{});
     return cudaLaunchKernelEx(&cfg, kernel, p.tmap_w, p.tmap_h, a.M, a.V, a.d, n_n, n_v, stream_w, a.v_offset, a.keys,
-                              a.status, a.pub, a.rank);
+                              a.status, a.pub, a.rank, a.noise);
 }
 
 }  // namespace
@@ -284,11 +294,14 @@ int vm_choose_bn(int M) { return M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : 
 
 template <int BN> static cudaError_t set_smem() {
     const int bytes = VCfg<BN>::SMEM_BYTES;
-    cudaError_t e = cudaFuncSetAttribute(umma_vm_kernel<BN, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(umma_vm_kernel<BN, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(umma_vm_kernel<BN, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(umma_vm_kernel<BN, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
-    return e;
+    const void *kernels[6] = {(const void *)umma_vm_kernel<BN, false, EPI_PLAIN>,  (const void *)umma_vm_kernel<BN, true, EPI_PLAIN>,
+                              (const void *)umma_vm_kernel<BN, false, EPI_COUNT>,  (const void *)umma_vm_kernel<BN, true, EPI_COUNT>,
+                              (const void *)umma_vm_kernel<BN, false, EPI_SAMPLE>, (const void *)umma_vm_kernel<BN, true, EPI_SAMPLE>};
+    for (const void *k : kernels) {
+        const cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+        if (e != cudaSuccess) return e;
+    }
+    return cudaSuccess;
 }
 
 cudaError_t umma_vm_prepare() {

@@ -107,7 +107,7 @@ class ClockSampler:
 class GpuWorkload:
     """One workload resident on the device: rotating copies of W_lm, inputs, outputs, handles."""
 
-    def __init__(self, cfg: gen.Config, device: int, w_copies: int, W_host=None, flags: int = 0, group=None):
+    def __init__(self, cfg: gen.Config, device: int, w_copies: int, W_host=None, flags: int = 0, group=None, rule=None):
         import torch
 
         import paper_2504_20039_b200 as aj
@@ -143,6 +143,11 @@ class GpuWorkload:
         self.handle = aj.Handle(device, cfg.B, cfg.K, cfg.d, cfg.d_draft, cfg.V, aj.AJ_BF16, aj.AJ_W_VD, flags, shard=shard[0])
         self.handle_t = aj.Handle(device, cfg.B, cfg.K, cfg.d, cfg.d_draft, cfg.V, aj.AJ_BF16, aj.AJ_W_VD,
                                   flags | aj.AJ_FLAG_TIME_KERNELS, shard=shard[1])
+        for h in (self.handle, self.handle_t):  # the variants of the acceptance step: top-K rule, sampled target tokens
+            if rule and rule.get("top_k"):
+                h.set_top_k(rule["top_k"])
+            if rule and rule.get("temperature"):
+                h.set_sampling(rule["temperature"], seed=20250420, step=0)
         for ex in self.exchanges:
             ex.ready()
         # draft tokens planted against the device's own greedy tokens (a benchmark input, never an oracle input)
@@ -258,8 +263,8 @@ def roofline_of(cfg: gen.Config, gemm_ms: float, pk, v_count=None):
             "kernel_ms": gemm_ms, "algorithmic_flops": flops}
 
 
-def bench_one(cfg, device, steps, warmup, barrier, reduce_max, pk, w_copies, W_host=None, with_e2e=True, flags=0, group=None):
-    wl = GpuWorkload(cfg, device, w_copies, W_host, flags, group)
+def bench_one(cfg, device, steps, warmup, barrier, reduce_max, pk, w_copies, W_host=None, with_e2e=True, flags=0, group=None, rule=None):
+    wl = GpuWorkload(cfg, device, w_copies, W_host, flags, group, rule)
     try:
         wl.run(wl.handle, warmup)
         with ClockSampler(device) as cs:
@@ -275,7 +280,7 @@ def bench_one(cfg, device, steps, warmup, barrier, reduce_max, pk, w_copies, W_h
         assert wl.handle.last_status() == wl.aj.AJ_OK and wl.handle_t.last_status() == wl.aj.AJ_OK
         res = {
             "ms_per_step": ms / steps, "clocks": clocks, "path": wl.handle.last_gemm_path(),
-            "roofline": dict(roofline_of(cfg, gemm_mean, pk, wl.v_count), traffic=None if group is not None else traffic_of(cfg, wl.handle.last_gemm_path())),
+            "roofline": dict(roofline_of(cfg, gemm_mean, pk, wl.v_count), traffic=None if (group is not None or rule) else traffic_of(cfg, wl.handle.last_gemm_path())),
             "gemm_ms_min": gemm_min, "gemm_launches_timed": n,
             "launches_per_step": wl.handle.last_launch_count(),
             "mean_accept_len": float(wl.acc.float().mean().item()),
@@ -355,6 +360,8 @@ def main():
     ap.add_argument("--sharding", default="batch", choices=["batch", "vocab"],
                     help="batch: every rank its own batch and its own W_lm (default); vocab: W_lm split by vocabulary over the ranks")
     ap.add_argument("--flags", type=int, default=0, help="extra aj_create flags (kernel selection switches, for comparisons)")
+    ap.add_argument("--top-k", type=int, default=0, help="time the top-K acceptance rule (paper Section 4.1) instead of the classifier")
+    ap.add_argument("--temperature", type=float, default=0.0, help="time sampled verification (paper Appendix A) at this temperature instead of greedy")
     ap.add_argument("--w-copies", type=int, default=None, help="copies of W_lm to rotate over (default 3, or 2 for the 70B shape)")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -378,11 +385,12 @@ def main():
     copies = args.w_copies or (3 if head.d * head.V * 2 < 1.5e9 else 2)
 
     vocab = args.sharding == "vocab"
+    rule = {k: v for k, v in (("top_k", args.top_k), ("temperature", args.temperature)) if v}
     if not vocab:
         head = ajd.rank_config(head, rank)  # every rank verifies its own sequences
     W_host = gen.make_W(head)
     r = bench_one(head, local, steps, warmup, barrier, reduce_max, pk, copies, W_host, with_e2e=not args.no_e2e, flags=args.flags,
-                  group=group if vocab else None)
+                  group=group if vocab else None, rule=rule)
     positions = head.B * head.K if vocab else ajd.job_positions(head, world)
     line = {
         "metric": METRIC, "value": positions / (r["ms_per_step"] * 1e-3), "unit": UNIT, "n_gpus": world, "steps": steps,
@@ -392,7 +400,8 @@ def main():
                    "tau": head.tau, "match_rate": [head.match_lo, head.match_hi], "parallelism": (f"W_lm split by vocabulary over {world} GPU(s), one batch, keys exchanged by peer stores inside the kernels"
                                    if vocab else f"replicated W, batch per rank x{world}"),
                    "l2": f"W_lm rotates over {copies} copies of {head.d * head.V * 2 / 1e9:.2f} GB each (inputs larger than the 126 MB L2)",
-                   "gemm_path": r["path"], "mean_accept_len": r["mean_accept_len"]},
+                   "gemm_path": r["path"], "mean_accept_len": r["mean_accept_len"],
+                   "rule": rule or "classifier at tau on greedy target tokens"},
         "clocks": r["clocks"], "roofline": r["roofline"],
         "gpu_launches": r["launches_per_step"] * steps,
     }
@@ -413,7 +422,7 @@ def main():
             cfg = ajd.rank_config(cfg, rank)
             same_W = cfg.d == head.d and cfg.V == head.V
             n = max(20, int(0.4 / max(2.0 * cfg.M * cfg.d * cfg.V / 1.2e15, 1.7e-4)))
-            rr = bench_one(cfg, local, n, 5, barrier, reduce_max, pk, 2 if not same_W else copies, W_host if same_W else None, with_e2e=False, flags=args.flags)
+            rr = bench_one(cfg, local, n, 5, barrier, reduce_max, pk, 2 if not same_W else copies, W_host if same_W else None, with_e2e=False, flags=args.flags, rule=rule)
             extra.append({"workload": cfg.name, "B": cfg.B, "K": cfg.K, "d": cfg.d, "V": cfg.V, "steps": n,
                           "ms_per_step": rr["ms_per_step"], "value": cfg.B * cfg.K * world / (rr["ms_per_step"] * 1e-3), "unit": UNIT,
                           "gemm_path": rr["path"], "roofline": rr["roofline"], "clocks": rr["clocks"]})

@@ -167,12 +167,12 @@ __device__ inline void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint
                                      uint32_t (&out)[4]) {
 #pragma unroll
     for (int r = 0; r < 10; r++) {
-        const uint32_t h0 = __umulhi(0xD2511F53u, c0), l0 = 0xD2511F53u * c0;
-        const uint32_t h1 = __umulhi(0xCD9E8D57u, c2), l1 = 0xCD9E8D57u * c2;
-        c0 = h1 ^ c1 ^ k0;
-        c1 = l1;
-        c2 = h0 ^ c3 ^ k1;
-        c3 = l0;
+        const unsigned long long p0 = (unsigned long long)0xD2511F53u * c0;  // one wide multiply gives both halves
+        const unsigned long long p1 = (unsigned long long)0xCD9E8D57u * c2;
+        c0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
+        c1 = (uint32_t)p1;
+        c2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+        c3 = (uint32_t)p0;
         k0 += 0x9E3779B9u;
         k1 += 0xBB67AE85u;
     }
@@ -182,28 +182,48 @@ __device__ inline void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint
     out[3] = c3;
 }
 
-__device__ inline float gumbel_from_bits(uint32_t x) {
-    const float u = ((float)(x >> 9) + 0.5f) * 1.1920928955078125e-07f;  // 2^-23
-    return -logf(-logf(u));
+// lg2(-ln u) for u = (k + 0.5) * 2^-23, k = x >> 9; the Gumbel noise is g = -ln 2 * that, to about
+// 2e-6 absolute.  Built on the hardware's base-2 logarithm, whose absolute error (about 2e-7 on the
+// logarithm of the mantissa) is not enough for -ln u where u is close to 1, which is where the
+// largest noise values, the ones that win, come from: for t = 1 - u <= 1/16 (exact in fp32) the
+// series t + t^2/2 + ... + t^6/6 is used instead (the first term left out is below 1e-8 relative).
+// No integer-to-float conversion, no division, no branch: u is assembled from the bits.
+__device__ inline float lg2_approx(float x) {
+    float y;
+    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
 }
+
+__device__ inline float lg2_neg_ln_uniform(uint32_t x) {
+    const float f = __uint_as_float(0x3F800000u | (x >> 9));  // 1 + k 2^-23
+    const float u = f - __uint_as_float(0x3F7FFFFFu);         // minus (1 - 2^-24): (k + 0.5) 2^-23, exact
+    const float t = 1.0f - u;                                 // exact
+    const float near_one =
+        t * fmaf(t, fmaf(t, fmaf(t, fmaf(t, fmaf(t, 1.0f / 6.0f, 0.2f), 0.25f), 1.0f / 3.0f), 0.5f), 1.0f);
+    const float far = -0.693147180559945f * lg2_approx(u);
+    return lg2_approx(t <= 0.0625f ? near_one : far);
+}
+
+__device__ inline float gumbel_from_bits(uint32_t x) { return -0.693147180559945f * lg2_neg_ln_uniform(x); }
 
 // The noisy score of one element.
 __device__ inline float noisy_score(const Noise &nz, float logit, int row, int v) {
     uint32_t w[4];
     philox4x32_10((uint32_t)v, (uint32_t)(row >> 2), nz.step0, nz.step1, nz.key0, nz.key1, w);
     const uint32_t x = (row & 2) ? ((row & 1) ? w[3] : w[2]) : ((row & 1) ? w[1] : w[0]);
-    return fmaf(nz.temperature, gumbel_from_bits(x), logit);
+    return fmaf(nz.temperature * -0.693147180559945f, lg2_neg_ln_uniform(x), logit);
 }
 
 // Epilogue add-on for the vocabulary-major kernels: this thread holds entry v of the 32 rows
 // row_first .. + 32 (row_first a multiple of 4) in x[]; one Philox call serves four rows.
 __device__ inline void add_gumbel_noise(const Noise &nz, float (&x)[32], int v, int row_first) {
+    const float scale = nz.temperature * -0.693147180559945f;
 #pragma unroll
     for (int q = 0; q < 8; q++) {
         uint32_t w[4];
         philox4x32_10((uint32_t)v, (uint32_t)((row_first >> 2) + q), nz.step0, nz.step1, nz.key0, nz.key1, w);
 #pragma unroll
-        for (int i = 0; i < 4; i++) x[4 * q + i] = fmaf(nz.temperature, gumbel_from_bits(w[i]), x[4 * q + i]);
+        for (int i = 0; i < 4; i++) x[4 * q + i] = fmaf(scale, lg2_neg_ln_uniform(w[i]), x[4 * q + i]);
     }
 }
 #endif

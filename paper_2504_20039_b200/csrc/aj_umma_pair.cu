@@ -262,7 +262,10 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
             const unsigned long long k = __ldcg(keys + row);
             return k == 0ull ? -INFINITY : key_value(k);
         };
-        constexpr int GRP = 4;  // thresholds are fetched four chunks ahead of their use: an L2 round trip
+        // thresholds are fetched GRP chunks ahead of their use, an L2 round trip: four chunks, or one
+        // where the noise makes a chunk take that long by itself (and one copy of its code, not four,
+        // then stays within the instruction cache)
+        constexpr int GRP = EPI == EPI_SAMPLE ? 1 : 4;
         int it = 0;
         for (int t = pair; t < num_tiles; t += num_pairs, ++it) {
             const Tile tl = decode_tile(sc, t);

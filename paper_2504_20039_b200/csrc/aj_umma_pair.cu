@@ -44,7 +44,13 @@ constexpr int BV_CTA = 128;
 constexpr int BN = 256;       // rows of h per accumulator (half of them staged by each CTA)
 constexpr int BK = 64;        // bf16 elements per k-block = 128 bytes = one swizzle span
 constexpr int UMMA_K = 16;
-constexpr int NUM_THREADS = 192;
+// Warp 0 loads, warp 1 issues the MMAs, the rest drain the accumulators: one warp per TMEM lane quadrant,
+// or two (which take alternate chunks of columns) where the epilogue also generates the noise and, with
+// two accumulators per tile, is not hidden under the next tile's MMAs.  (Measured on one GPU against four
+// warps, sampled mode: 3 % and 4 % faster with two accumulators at 2080 x 8192 and 264 x 4096, 3 % slower
+// with one at 2112 and 528 rows x 4096.)
+__host__ __device__ constexpr int epilogue_warps(int epi, bool dual) { return epi == EPI_SAMPLE && dual ? 8 : 4; }
+__host__ __device__ constexpr int num_threads(int epi, bool dual) { return 64 + 32 * epilogue_warps(epi, dual); }
 constexpr int A_BYTES = BV_CTA * BK * 2;   // 16 KB: this CTA's 128 rows of W, one k-block
 constexpr int RING_BYTES = 224 * 1024;     // shared memory given to the stage ring (the SM has 227 KB per CTA)
 constexpr int MAX_STAGES = 8;
@@ -90,7 +96,7 @@ __device__ inline Tile decode_tile(const PairSched &sc, int t) {
 // EPI: EPI_COUNT also counts, per row, the entries that outrank the draft token (top-K rule);
 // EPI_SAMPLE adds Gumbel noise to the logits before the argmax.
 template <bool DUAL, bool WDV, int EPI>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+__global__ void __launch_bounds__(num_threads(EPI, DUAL), 1)
 umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_h,
                  int M, int V, int d, PairSched sc, int stream_w, int v_offset,
                  unsigned long long *__restrict__ keys, int *__restrict__ status, const Publish pub, const RankArgs rk,
@@ -128,7 +134,7 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
         }
         for (int a = 0; a < 2; a++) {
             mbar_init(acc_full_bar(a), 1);
-            mbar_init(acc_empty_bar(a), 8);  // four epilogue warps in each of the two CTAs
+            mbar_init(acc_empty_bar(a), 2 * epilogue_warps(EPI, DUAL));  // the epilogue warps of the two CTAs
         }
         *abort_flag = 0;
         fence_barrier_init();
@@ -252,6 +258,8 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
         // column by redux.sync, lowest lane by ballot, 64-bit atomic max into the key).  After the
         // first few vocabulary blocks nearly every chunk is skipped.
         const int q = warp & 3;  // TMEM lane quadrant this warp may read
+        constexpr int SPLIT = epilogue_warps(EPI, DUAL) / 4;           // warps per quadrant
+        const int part = SPLIT == 1 ? 0 : (warp - 2) >> 2;        // which of them this one is
         const float never = __int_as_float(0x7fc00000);  // NaN: no comparison with it is ever true
         // Chunk g of a tile is columns 32 (g & 7) .. + 32 of accumulator g >> 3.  Its threshold for
         // lane j is the best value the row of column 32 (g & 7) + j has so far, read from the key.
@@ -272,7 +280,7 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
             const int slot = acc_slot(it);
             float cur[GRP], nxt[GRP];
 #pragma unroll
-            for (int u = 0; u < GRP; u++) cur[u] = load_thr(tl, u);  // in flight while the accumulators are being computed
+            for (int u = 0; u < GRP; u++) cur[u] = load_thr(tl, part * GRP + u);  // in flight while the accumulators are being computed
             // the whole warp takes one decision, so the aligned TMEM loads below stay converged
             if (!__all_sync(0xffffffffu, mbar_wait(acc_full_bar(slot), acc_phase(it), abort_flag))) {
                 give_up();
@@ -284,9 +292,9 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
             const uint32_t tbase = tmem_base + ((uint32_t)(q * 32) << 16);
             // the group loop is kept rolled: one copy of the code stays in the instruction cache
 #pragma unroll 1
-            for (int g0 = 0; g0 < 8 * n_acc; g0 += GRP) {
+            for (int g0 = part * GRP; g0 < 8 * n_acc; g0 += GRP * SPLIT) {
 #pragma unroll
-                for (int u = 0; u < GRP; u++) nxt[u] = (g0 + GRP < 8 * n_acc) ? load_thr(tl, g0 + GRP + u) : never;
+                for (int u = 0; u < GRP; u++) nxt[u] = (g0 + GRP * SPLIT < 8 * n_acc) ? load_thr(tl, g0 + GRP * SPLIT + u) : never;
 #pragma unroll
                 for (int u = 0; u < GRP; u++) {
                     const int g = g0 + u, a = g >> 3, c = g & 7;
@@ -369,7 +377,7 @@ cudaError_t umma_pair_prepare(int num_sms) {
     // how many CTA pairs can be resident at once (pairs need both SMs of a pair free)
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(num_sms & ~1));
-    cfg.blockDim = dim3(NUM_THREADS);
+    cfg.blockDim = dim3(num_threads(EPI_SAMPLE, true));  // the largest block: residency is the same, one CTA per SM
     cfg.dynamicSmemBytes = SMEM_BYTES;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -379,7 +387,7 @@ cudaError_t umma_pair_prepare(int num_sms) {
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     int clusters = 0;
-    e = cudaOccupancyMaxActiveClusters(&clusters, umma_pair_kernel<false, false, EPI_PLAIN>, &cfg);
+    e = cudaOccupancyMaxActiveClusters(&clusters, umma_pair_kernel<true, false, EPI_SAMPLE>, &cfg);
     if (e != cudaSuccess) return e;
     if (clusters < 1) return cudaErrorInvalidConfiguration;
     g_max_pairs = clusters < num_sms / 2 ? clusters : num_sms / 2;
@@ -424,7 +432,7 @@ cudaError_t launch_umma_pair(const GemmArgs &a, const UmmaPlan &p, cudaStream_t 
     const int stream_w = (sc.n_n == 1) ? 1 : 0;  // W is read by one pair only: do not keep it in L2
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)p.grid);  // 2 CTAs per pair
-    cfg.blockDim = dim3(NUM_THREADS);
+    cfg.blockDim = dim3(num_threads(a.noise.temperature > 0.0f ? EPI_SAMPLE : EPI_PLAIN, sc.dual != 0));
     cfg.dynamicSmemBytes = SMEM_BYTES;
     cfg.stream = stream;
     cudaLaunchAttribute attr[2];

@@ -287,6 +287,94 @@ int ajo_verify_sampled(const void *h_target, const void *h_draft, const void *W,
 }
 
 /*
+ * Tree drafts (Section 3.3, "Generality": the method applies to tree-based speculative decoding;
+ * Appendix on EAGLE-2).  The draft is a tree of N nodes in topological order: parent[n] is -1 for a
+ * child of the root (the last accepted token, row 0) or the index (< n) of another node; row n + 1
+ * of the hidden states encodes node n.  The target's prediction after a node is the token of that
+ * node's row, so node n matches iff tok[n] == y[parent[n] + 1].  The acceptance rule of the paper,
+ * applied along every root-to-leaf path as it is applied to a window: a node is accepted iff its
+ * parent is accepted (the root always is) and it matches or its mismatch is forgiven (p < tau).  The
+ * result is the deepest accepted node (among equally deep ones the lowest index; -1 = the root),
+ * its depth as the accepted length, and the target's token after it.  A node whose parent index is
+ * outside [-1, n) is never accepted and never judged.
+ *
+ * This function is the rule alone, on given tokens and probabilities (p[n] is read only where node n
+ * mismatches).
+ */
+void ajo_tree_accept(int N, const int32_t *tok, const int32_t *parent, const int32_t *y, const double *p,
+                     float tau, int32_t *accept_len, int32_t *best_node, int32_t *next_tok)
+{
+    int best = -1, best_depth = 0;
+    int *ok = (int *)malloc((size_t)N * sizeof(int)), *depth = (int *)malloc((size_t)N * sizeof(int));
+    for (int n = 0; n < N; n++) {
+        const int q = parent[n];
+        ok[n] = 0;
+        depth[n] = 0;
+        if (q < -1 || q >= n) continue;
+        const int parent_ok = (q == -1) ? 1 : ok[q];
+        const int passes = (tok[n] == y[q + 1]) ? 1 : forgiven(p[n], tau);
+        depth[n] = (q == -1 ? 0 : depth[q]) + 1;
+        ok[n] = parent_ok && passes;
+        if (ok[n] && depth[n] > best_depth) {
+            best = n;
+            best_depth = depth[n];
+        }
+    }
+    free(ok);
+    free(depth);
+    *accept_len = best_depth;
+    *best_node = best;
+    *next_tok = y[best + 1];
+}
+
+/*
+ * The whole step for tree drafts: B sequences of N nodes (N + 1 rows each, layouts as ajo_verify),
+ * target tokens greedy or drawn (temperature as in ajo_verify_sampled), the classifier evaluated at
+ * every mismatching node with a valid parent, then ajo_tree_accept.
+ */
+int ajo_verify_tree(const void *h_target, const void *h_draft, const void *W, const int32_t *draft_tok,
+                    const int32_t *parent, const float *judge_w, float judge_b, float tau, int dtype, int w_layout,
+                    int B, int N, int d, int d_draft, int V, double temperature, uint64_t seed, uint64_t step,
+                    int32_t *accept_len, int32_t *next_tok, int32_t *best_node, int32_t *target_tok,
+                    double *top1, double *gap, double *judge_p)
+{
+    if (!h_target || !W || !draft_tok || !parent || !judge_w || B < 1 || N < 1 || d < 1 || V < 1 ||
+        d_draft < 0 || (d_draft > 0 && !h_draft))
+        return 1;
+    size_t esz = (dtype == AJO_BF16) ? 2 : 4;
+    int R = N + 1;
+    double *logits = (double *)malloc((size_t)R * V * sizeof(double));
+    if (!logits) return 2;
+    for (int b = 0; b < B; b++) {
+        const char *ht = (const char *)h_target + (size_t)b * R * d * esz;
+        const char *hdr = h_draft ? (const char *)h_draft + (size_t)b * R * d_draft * esz : NULL;
+        int rc = ajo_logits(ht, W, dtype, w_layout, R, d, V, logits);
+        if (rc) { free(logits); return rc; }
+        if (temperature > 0.0) {
+#pragma omp parallel for schedule(static)
+            for (int v = 0; v < V; v++)
+                for (int j = 0; j < R; j++)
+                    logits[(size_t)j * V + v] += temperature * ajo_gumbel(seed, step, b * R + j, v);
+        }
+        int32_t *y = target_tok + (size_t)b * R;
+        for (int j = 0; j < R; j++)
+            ajo_argmax(logits + (size_t)j * V, V, &y[j], &top1[(size_t)b * R + j], &gap[(size_t)b * R + j]);
+        const int32_t *tok = draft_tok + (size_t)b * N, *par = parent + (size_t)b * N;
+        double *p = judge_p + (size_t)b * N;
+        for (int n = 0; n < N; n++) {
+            p[n] = NAN;
+            if (par[n] < -1 || par[n] >= n) continue;
+            if (tok[n] != y[par[n] + 1]) /* row n + 1 encodes node n */
+                p[n] = ajo_judge_p(hdr ? hdr + (size_t)(n + 1) * d_draft * esz : NULL,
+                                   ht + (size_t)(n + 1) * d * esz, dtype, judge_w, judge_b, d_draft, d);
+        }
+        ajo_tree_accept(N, tok, par, y, p, tau, &accept_len[b], &best_node[b], &next_tok[b]);
+    }
+    free(logits);
+    return 0;
+}
+
+/*
  * Rank of entry `tok` in one row of logits: how many entries come before it when the row is sorted
  * by decreasing logit, ties by increasing index.  *near receives the number of OTHER entries whose
  * logit lies within `band` of logit[tok] (a device that rounds differently may order those otherwise).

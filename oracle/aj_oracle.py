@@ -144,6 +144,55 @@ class OracleResult:
     judge_p: np.ndarray  # [B, K] float64, NaN where the draft token matched
 
 
+def tree_accept(tok, parent, y, p, tau):
+    """The acceptance rule on a draft tree (one sequence): (accept_len, best_node, next_tok)."""
+    tok = np.ascontiguousarray(tok, dtype=np.int32)
+    parent = np.ascontiguousarray(parent, dtype=np.int32)
+    y = np.ascontiguousarray(y, dtype=np.int32)
+    p = np.ascontiguousarray(p, dtype=np.float64)
+    N = tok.shape[0]
+    assert parent.shape == (N,) and y.shape == (N + 1,) and p.shape == (N,)
+    out = [ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32()]
+    L = _lib()
+    L.ajo_tree_accept.argtypes = [ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_float,
+                                  ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+    L.ajo_tree_accept.restype = None
+    L.ajo_tree_accept(N, _ptr(tok), _ptr(parent), _ptr(y), _ptr(p), float(tau), *[ctypes.byref(o) for o in out])
+    return tuple(int(o.value) for o in out)
+
+
+def verify_tree(h_target, h_draft, W, draft_tok, parent, judge_w, judge_b, tau, dtype: int, w_layout: int = 0,
+                temperature: float = 0.0, seed: int = 0, step: int = 0) -> OracleResult:
+    """The whole step for tree drafts: h_target [B, N+1, d], draft_tok and parent [B, N]; the result also has best_node [B]."""
+    ht = np.ascontiguousarray(h_target)
+    B, R, d = ht.shape
+    N = R - 1
+    hd = None if h_draft is None else np.ascontiguousarray(h_draft)
+    dd = 0 if hd is None else hd.shape[2]
+    W = np.ascontiguousarray(W)
+    V = W.shape[0] if w_layout == 0 else W.shape[1]
+    tok = np.ascontiguousarray(draft_tok, dtype=np.int32)
+    par = np.ascontiguousarray(parent, dtype=np.int32)
+    assert tok.shape == (B, N) and par.shape == (B, N)
+    w = np.ascontiguousarray(judge_w, dtype=np.float32)
+    assert w.shape == (dd + d,)
+    res = OracleResult(np.empty(B, np.int32), np.empty(B, np.int32), np.empty((B, R), np.int32), np.empty((B, R), np.float64),
+                       np.empty((B, R), np.float64), np.empty((B, N), np.float64))
+    best = np.empty(B, np.int32)
+    L = _lib()
+    vp, ci, u64 = ctypes.c_void_p, ctypes.c_int, ctypes.c_uint64
+    L.ajo_verify_tree.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_float, ctypes.c_float, ci, ci, ci, ci, ci, ci, ci,
+                                  ctypes.c_double, u64, u64, vp, vp, vp, vp, vp, vp, vp]
+    L.ajo_verify_tree.restype = ci
+    rc = L.ajo_verify_tree(_ptr(ht), _ptr(hd), _ptr(W), _ptr(tok), _ptr(par), _ptr(w), float(judge_b), float(tau), dtype, w_layout,
+                           B, N, d, dd, V, float(temperature), int(seed), int(step), _ptr(res.accept_len), _ptr(res.next_tok),
+                           _ptr(best), _ptr(res.target_tok), _ptr(res.top1), _ptr(res.gap), _ptr(res.judge_p))
+    if rc:
+        raise RuntimeError(f"ajo_verify_tree failed ({rc})")
+    res.best_node = best
+    return res
+
+
 def philox4x32_10(ctr, key):
     """Philox4x32-10: four 32-bit counter words and two key words in, four words out."""
     c = np.asarray(ctr, dtype=np.uint32)

@@ -479,3 +479,119 @@ def test_gumbel_max_draws_follow_the_softmax_and_zero_temperature_is_greedy():
     # the reported winner is the noisy score
     j, y = 2, int(same.target_tok[0, 2])
     assert same.top1[0, j] == pytest.approx(lg[j, y] + T * orc.gumbel(2024, 17, j, y), abs=1e-12)
+
+
+# ------------------------------------------------------ tree drafts (Section 3.3 "Generality", EAGLE-2 appendix)
+
+
+def _random_tree(rng, N, shape="random"):
+    if shape == "chain":
+        return np.arange(-1, N - 1, dtype=np.int32)
+    if shape == "star":
+        return np.full(N, -1, np.int32)
+    return np.array([rng.integers(-1, n) for n in range(N)], dtype=np.int32)
+
+
+def _paths(parent):
+    """Root-to-node path (list of node indices, root excluded) of every node with a valid ancestry."""
+    out = {}
+    for n, q in enumerate(parent):
+        if q == -1:
+            out[n] = [n]
+        elif 0 <= q < n and q in out:
+            out[n] = out[q] + [n]
+    return out
+
+
+def test_tree_rule_is_the_window_rule_on_every_root_to_node_path():
+    """Brute force: a node is accepted iff the window rule (the pinned accept walk) accepts the whole window
+    formed by its root path; the result is the deepest such node, the lowest index among equals."""
+    rng = np.random.default_rng(5)
+    for trial in range(400):
+        N = int(rng.integers(1, 9))
+        parent = _random_tree(rng, N, ("random", "random", "chain", "star")[trial % 4])
+        if trial % 7 == 3 and N > 2:
+            parent[int(rng.integers(1, N))] = N + 3          # an invalid parent: that node and its subtree never count
+        y = rng.integers(0, 3, N + 1).astype(np.int32)
+        tok = rng.integers(0, 3, N).astype(np.int32)
+        p = rng.random(N)
+        tau = float(rng.choice([0.0, 0.3, 0.6, 1.0]))
+        best, best_len = -1, 0
+        for n, path in _paths(parent).items():
+            rows = [0] + [m + 1 for m in path]               # the rows along the path, root first
+            win_y = y[rows][None, :]                         # the window's target tokens
+            win_tok = tok[path][None, :]
+            win_p = p[path][None, :]
+            acc, _ = orc.rewalk(win_y, win_tok, win_p, tau)
+            if acc[0] == len(path) and len(path) > best_len:
+                best, best_len = n, len(path)
+        got = orc.tree_accept(tok, parent, y, p, tau)
+        assert got == (best_len, best, int(y[best + 1])), (trial, parent, tok, y, p, tau, got, best)
+
+
+def test_tree_rule_special_cases():
+    y = np.array([5, 6, 7, 8, 9], np.int32)
+    p = np.array([0.9, 0.2, 0.9, 0.2])
+    chain = np.array([-1, 0, 1, 2], np.int32)
+    # a chain is a window: stop at the first mismatch that is not forgiven
+    assert orc.tree_accept([5, 6, 0, 8], chain, y, p, 0.5) == (2, 1, 7)
+    assert orc.tree_accept([5, 0, 0, 8], chain, y, p, 0.5) == (2, 1, 7)     # node 1 forgiven (0.2 < 0.5), node 2 not
+    assert orc.tree_accept([5, 0, 0, 8], chain, y, p, 0.0) == (1, 0, 6)     # nothing forgiven
+    assert orc.tree_accept([0, 0, 0, 0], chain, y, p, 1.0) == (4, 3, 9)     # everything forgiven
+    assert orc.tree_accept([0, 6, 7, 8], chain, y, p, 0.5) == (0, -1, 5)    # the first node fails: the root stands
+    # a star: depth 1 at most, the first passing child wins
+    star = np.full(4, -1, np.int32)
+    assert orc.tree_accept([1, 2, 5, 5], star, y, p, 0.0) == (1, 2, 8)
+    assert orc.tree_accept([1, 2, 3, 4], star, y, p, 0.5) == (1, 1, 7)
+    # two branches: the deeper accepted one wins even if it comes later; equal depth: the lower index
+    par = np.array([-1, -1, 1, 2], np.int32)
+    assert orc.tree_accept([5, 5, 7, 8], par, y, p, 0.0) == (3, 3, 9)
+    assert orc.tree_accept([5, 5, 0, 7], par, y, np.array([0.9, 0.9, 0.9, 0.9]), 0.5) == (1, 0, 6)
+    # a match is tested against the PARENT's row: node 2 (child of node 1) must equal y[2]
+    assert orc.tree_accept([5, 5, 7, 0], par, y, p, 0.0) == (2, 2, 8)
+    assert orc.tree_accept([5, 5, 8, 0], par, y, np.array([0.9] * 4), 0.5) == (1, 0, 6)
+    # accept_len never decreases with tau
+    rng = np.random.default_rng(2)
+    for _ in range(50):
+        N = 7
+        parent = _random_tree(rng, N)
+        yy, tt, pp = rng.integers(0, 3, N + 1).astype(np.int32), rng.integers(0, 3, N).astype(np.int32), rng.random(N)
+        lens = [orc.tree_accept(tt, parent, yy, pp, t)[0] for t in (0.0, 0.2, 0.5, 0.8, 1.0)]
+        assert lens == sorted(lens)
+        depth = {n: len(path) for n, path in _paths(parent).items()}
+        assert lens[-1] == max(depth.values())
+
+
+@pytest.mark.parametrize("dtype", [BF16, F32])
+def test_tree_step_reduces_to_the_window_step_on_a_chain_and_composes_from_its_parts(dtype):
+    cfg = gen.Config("tree", B=3, K=6, d=40, d_draft=24, V=50, dtype=dtype, sigma_w=0.4, match_lo=0.4, match_hi=0.8, seed=81)
+    W = gen.make_W(cfg)
+    ht, hd = gen.make_hidden(cfg)
+    w = gen.make_judge(cfg)
+    y = np.stack([[orc.argmax(r)[0] for r in orc.logits(ht[b], W, dtype)] for b in range(cfg.B)])
+    tok = gen.plant_draft_tokens(cfg, y)
+    chain = np.tile(np.arange(-1, cfg.K - 1, dtype=np.int32), (cfg.B, 1))
+    for tau in (0.0, 0.4, 0.7, 1.0):
+        a = orc.verify(ht, hd, W, tok, w, cfg.judge_b, tau, dtype)
+        t = orc.verify_tree(ht, hd, W, tok, chain, w, cfg.judge_b, tau, dtype)
+        np.testing.assert_array_equal(t.accept_len, a.accept_len)
+        np.testing.assert_array_equal(t.next_tok, a.next_tok)
+        np.testing.assert_array_equal(t.target_tok, a.target_tok)
+        np.testing.assert_array_equal(t.best_node, a.accept_len - 1)
+        np.testing.assert_array_equal(t.judge_p, a.judge_p)
+    # a real tree: tokens planted against the parents' rows; the step equals argmax + judge_p + the rule
+    rng = np.random.default_rng(9)
+    parent = np.stack([_random_tree(rng, cfg.K) for _ in range(cfg.B)])
+    tok = np.stack([np.where(rng.random(cfg.K) < 0.7, y[b][parent[b] + 1], rng.integers(0, cfg.V, cfg.K)) for b in range(cfg.B)]).astype(np.int32)
+    t = orc.verify_tree(ht, hd, W, tok, parent, w, cfg.judge_b, 0.5, dtype)
+    np.testing.assert_array_equal(t.target_tok, y)
+    for b in range(cfg.B):
+        mism = tok[b] != y[b][parent[b] + 1]
+        assert mism.any() and (~mism).any()
+        assert (np.isnan(t.judge_p[b]) == ~mism).all()
+        for n in np.nonzero(mism)[0]:
+            assert t.judge_p[b, n] == orc.judge_p(hd[b, n + 1], ht[b, n + 1], dtype, w, cfg.judge_b)
+        assert (t.accept_len[b], t.best_node[b], t.next_tok[b]) == orc.tree_accept(tok[b], parent[b], y[b], np.nan_to_num(t.judge_p[b]), 0.5)
+    # sampled target tokens: the same rows and noise as the window step
+    s = orc.verify_tree(ht, hd, W, tok, chain, w, cfg.judge_b, 0.5, dtype, temperature=0.8, seed=3, step=2)
+    np.testing.assert_array_equal(s.target_tok, orc.verify(ht, hd, W, tok, w, cfg.judge_b, 0.5, dtype, temperature=0.8, seed=3, step=2).target_tok)

@@ -145,6 +145,30 @@ aj_status aj_set_top_k(aj_handle h, int top_k);
 aj_status aj_set_sampling(aj_handle h, float temperature, uint64_t seed, uint64_t step);
 
 /*
+ * The cycle for a tree draft (the paper's Section 3.3, "Generality": the method applies to tree-based
+ * speculative decoding; its appendix integrates it with EAGLE-2).  The N draft tokens of a sequence are
+ * the nodes of a tree in topological order: parent[b, n] is -1 for a child of the root (the last
+ * accepted token) or the index, below n, of another node.  Row 0 of h_target / h_draft encodes the
+ * root and row n + 1 encodes node n (the caller computed them under the tree's attention mask).  Node
+ * n matches iff draft_tok[b, n] equals the target's token of its parent's row; a mismatching node
+ * is scored by the classifier on row n + 1 exactly as a window position is.  A node is accepted iff
+ * its parent is accepted (the root always is) and it matches or p < tau.  Outputs: accept_len[b] =
+ * depth of the deepest accepted node (0 if none; among equally deep nodes the lowest index wins),
+ * best_node[b] = that node (-1 = the root; optional, may be NULL; its ancestors are the accepted
+ * path), next_tok[b] = the target's token of that node's row.  A node whose parent index is outside
+ * [-1, n) is never accepted and never scored.  With parent[b, n] = n - 1 this is aj_verify.
+ * All other arguments, their layouts, asynchrony and errors as aj_verify (N in place of K: N <= max_K;
+ * draft_tok, parent and judge_p are [B, N], target_tok and top1_val [B, N + 1]); parent is a device
+ * pointer.  Works with aj_set_sampling; not with aj_set_top_k or AJ_FLAG_NO_EXTRA_ROW
+ * (AJ_ERR_UNSUPPORTED).
+ */
+aj_status aj_verify_tree(aj_handle h, const void *h_target, const void *h_draft, const void *W_lm,
+                         const int32_t *draft_tok, const int32_t *parent, const float *judge_w, float judge_b,
+                         float tau, int B, int N, int d, int V,
+                         int32_t *accept_len, int32_t *next_tok, int32_t *best_node, int32_t *target_tok,
+                         float *top1_val, float *judge_p, void *cuda_stream);
+
+/*
  * The same cycle for a caller whose per-cycle tensors live in host memory: h_target, h_draft and
  * draft_tok are HOST pointers and are copied to the handle's staging buffers; accept_len and
  * next_tok (and target_tok, if not NULL) are HOST pointers and are copied back.  W_lm and judge_w

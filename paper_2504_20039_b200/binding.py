@@ -19,7 +19,7 @@ AJ_FLAG_FORCE_SIMT, AJ_FLAG_TIME_KERNELS, AJ_FLAG_ROW_TILES, AJ_FLAG_ONE_SM, AJ_
 
 EXPORTS = (
     "aj_create", "aj_verify", "aj_verify_host", "aj_last_status", "aj_last_gemm_ms", "aj_gemm_ms_stats", "aj_last_launch_count",
-    "aj_last_gemm_path", "aj_pair_schedule", "aj_destroy", "aj_set_top_k", "aj_set_sampling", "aj_shard_exchange_bytes", "aj_shard_exchange_alloc", "aj_shard_exchange_free", "aj_shard_range", "aj_create_sharded",
+    "aj_last_gemm_path", "aj_pair_schedule", "aj_destroy", "aj_set_top_k", "aj_set_sampling", "aj_verify_tree", "aj_shard_exchange_bytes", "aj_shard_exchange_alloc", "aj_shard_exchange_free", "aj_shard_range", "aj_create_sharded",
     "aj_shard_project", "aj_shard_finish", "aj_ipc_export", "aj_ipc_import", "aj_ipc_close", "aj_status_string", "aj_version", "aj_verify_static",
 )
 
@@ -47,6 +47,8 @@ def lib() -> ctypes.CDLL:
         L.aj_create.restype = ci
         L.aj_verify.argtypes = [vp, vp, vp, vp, vp, vp, cf, cf, ci, ci, ci, ci, vp, vp, vp, vp, vp, vp]
         L.aj_verify.restype = ci
+        L.aj_verify_tree.argtypes = [vp, vp, vp, vp, vp, vp, vp, cf, cf, ci, ci, ci, ci, vp, vp, vp, vp, vp, vp, vp]
+        L.aj_verify_tree.restype = ci
         L.aj_verify_host.argtypes = [vp, vp, vp, vp, vp, vp, cf, cf, ci, ci, ci, ci, vp, vp, vp, vp]
         L.aj_verify_host.restype = ci
         L.aj_last_status.argtypes = [vp]
@@ -246,6 +248,17 @@ class Handle:
                              _ptr(target_tok), _ptr(top1_val), _ptr(judge_p), stream or None)
         if check and st != AJ_OK:
             raise AjError(st, "aj_verify")
+        return st
+
+    def verify_tree(self, h_target, h_draft, W_lm, draft_tok, parent, judge_w, judge_b: float, tau: float, B: int, N: int,
+                    accept_len, next_tok, best_node=None, target_tok=None, top1_val=None, judge_p=None, stream: int = 0,
+                    check: bool = True) -> int:
+        """aj_verify_tree: the cycle for tree drafts (parent [B, N], -1 = child of the root; row n + 1 encodes node n)."""
+        st = lib().aj_verify_tree(self._h, _ptr(h_target), _ptr(h_draft), _ptr(W_lm), _ptr(draft_tok), _ptr(parent), _ptr(judge_w),
+                                  float(judge_b), float(tau), B, N, self.d, self.V, _ptr(accept_len), _ptr(next_tok),
+                                  _ptr(best_node), _ptr(target_tok), _ptr(top1_val), _ptr(judge_p), stream or None)
+        if check and st != AJ_OK:
+            raise AjError(st, "aj_verify_tree")
         return st
 
     def verify_host(self, h_target, h_draft, W_lm, draft_tok, judge_w, judge_b: float, tau: float, B: int, K: int,

@@ -408,8 +408,10 @@ static aj_status enqueue_project(aj_handle h, const void *h_target, const void *
 static aj_status enqueue_finish(aj_handle h, const void *h_target, const void *h_draft, const int32_t *draft_tok,
                                 const float *judge_w, float judge_b, float tau, int B, int K, int32_t *accept_len,
                                 int32_t *next_tok, int32_t *target_tok, float *top1_val, float *judge_p,
-                                cudaStream_t stream) {
+                                cudaStream_t stream, const int32_t *parent = nullptr, int32_t *best_node = nullptr) {
     JudgeArgs j;
+    j.parent = parent;
+    j.best_node = best_node;
     j.keys = h->keys;
     j.status = h->status;
     if (h->world) {
@@ -462,6 +464,27 @@ aj_status aj_verify(aj_handle h, const void *h_target, const void *h_draft, cons
     if (st != AJ_OK) return st;
     return enqueue_finish(h, h_target, h_draft, draft_tok, judge_w, judge_b, tau, B, K, accept_len, next_tok, target_tok,
                           top1_val, judge_p, stream);
+}
+
+aj_status aj_verify_tree(aj_handle h, const void *h_target, const void *h_draft, const void *W_lm, const int32_t *draft_tok,
+                         const int32_t *parent, const float *judge_w, float judge_b, float tau, int B, int N, int d, int V,
+                         int32_t *accept_len, int32_t *next_tok, int32_t *best_node, int32_t *target_tok, float *top1_val,
+                         float *judge_p, void *cuda_stream) {
+    aj_status st = check_call(h, h_target, h_draft, W_lm, draft_tok, judge_w, B, N, d, V, accept_len, next_tok);
+    if (st != AJ_OK) return st;
+    if (!parent) return AJ_ERR_INVALID_ARG;
+    // every node needs its own row, and the top-K rule's thresholds are taken per window position
+    if ((h->flags & AJ_FLAG_NO_EXTRA_ROW) || h->top_k > 0) return AJ_ERR_UNSUPPORTED;
+    if (h->dtype == AJ_BF16 && (!aligned16(h_target) || !aligned16(W_lm) || (h_draft && !aligned16(h_draft))))
+        return AJ_ERR_UNSUPPORTED;
+    if (h->projected) return AJ_ERR_INVALID_ARG;
+    DeviceGuard guard(h->device);
+    if (!guard.ok()) return AJ_ERR_CUDA;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    st = enqueue_project(h, h_target, W_lm, draft_tok, B, N, stream);
+    if (st != AJ_OK) return st;
+    return enqueue_finish(h, h_target, h_draft, draft_tok, judge_w, judge_b, tau, B, N, accept_len, next_tok, target_tok,
+                          top1_val, judge_p, stream, parent, best_node);
 }
 
 aj_status aj_verify_host(aj_handle h, const void *h_target_host, const void *h_draft_host, const void *W_lm,

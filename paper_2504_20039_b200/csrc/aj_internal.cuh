@@ -311,6 +311,8 @@ struct JudgeArgs {
     int top_k = 0;                   // > 0: the top-K rule replaces the classifier
     int V = 0;                       // vocabulary size (top-K rule: ids outside it are never accepted)
     unsigned *rank_cnt = nullptr;    // [B*R] counts from the projection kernel (top-K rule)
+    const int32_t *parent = nullptr; // [B, K] tree drafts: parent node of every node (-1 = the root), else nullptr
+    int32_t *best_node = nullptr;    // [B] tree drafts: the deepest accepted node (-1 = the root), optional
     int32_t *accept_len, *next_tok, *target_tok;
     float *top1_val, *judge_p;
 };

@@ -11,6 +11,12 @@
 // takes one item at a time and issues all of its 128-bit loads before it uses any of them.
 // Segment sums are added in a fixed order, so p does not depend on scheduling.
 //
+// Tree drafts (a.parent given): the K draft tokens are the nodes of a tree in topological order, row
+// i + 1 encodes node i, and node i is compared with the target's token of its PARENT's row.  The
+// classifier is evaluated at every mismatching node as above; a node is accepted iff its parent is
+// (the root always is) and it matches or is forgiven; the result is the deepest accepted node, the
+// lowest index among equally deep ones.  A chain (parent[i] = i - 1) is the window case.
+//
 // The kernel is launched as a programmatic dependent of the projection kernel: its blocks may
 // become resident while that kernel still runs and wait at the grid dependency before they
 // read the keys.  Each key is cleared right after it is read, so the next cycle finds zeros.
@@ -105,6 +111,7 @@ __global__ void __maxnreg__(96) judge_scan_kernel(JudgeArgs a) {
     int *rej_s = smem + R;                                    // [K]: 1 = mismatch not forgiven
     int *mis_s = rej_s + K;                                   // [K]
     float *part_s = reinterpret_cast<float *>(mis_s + K);     // [K][SEGS]
+    int *par_s = reinterpret_cast<int *>(part_s + K * SEGS);  // [K] tree drafts: parent, or below -1 if not valid
     const int b = blockIdx.x;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     const size_t esz = a.dtype == 0 ? 2 : 4;
@@ -117,6 +124,12 @@ __global__ void __maxnreg__(96) judge_scan_kernel(JudgeArgs a) {
     // the judge weights (and, for small batches, the candidate feature rows) into L2.
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     for (int i = threadIdx.x; i < K; i += blockDim.x) mis_s[i] = a.draft_tok[(size_t)b * K + i];
+    if (a.parent) {
+        for (int i = threadIdx.x; i < K; i += blockDim.x) {
+            const int q = a.parent[(size_t)b * K + i];
+            par_s[i] = (q >= -1 && q < i) ? q : -2;  // a parent must come earlier; anything else is never accepted
+        }
+    }
     if (a.top_k == 0) {  // the classifier's operands; the top-K rule needs none of them
         const char *wbytes = reinterpret_cast<const char *>(a.judge_w);
         const size_t wlines = ((size_t)(a.d + a.d_draft) * 4 + 127) / 128;
@@ -179,7 +192,11 @@ __global__ void __maxnreg__(96) judge_scan_kernel(JudgeArgs a) {
         if (a.top1_val) a.top1_val[(size_t)b * R + j] = key_value(key);
     }
     __syncthreads();
-    for (int i = threadIdx.x; i < K; i += blockDim.x) mis_s[i] = mis_s[i] != y_s[i];  // staged token vs greedy token
+    if (a.parent) {
+        for (int i = threadIdx.x; i < K; i += blockDim.x) mis_s[i] = par_s[i] < -1 || mis_s[i] != y_s[par_s[i] + 1];
+    } else {
+        for (int i = threadIdx.x; i < K; i += blockDim.x) mis_s[i] = mis_s[i] != y_s[i];  // staged token vs greedy token
+    }
     __syncthreads();
 
     const bool vec = (a.d % epc == 0) && (a.d_draft % epc == 0) && (row_bytes_t % 16 == 0) && (row_bytes_d % 16 == 0) &&
@@ -191,6 +208,7 @@ __global__ void __maxnreg__(96) judge_scan_kernel(JudgeArgs a) {
     for (int it = warp; it < K * SEGS; it += nwarps) {
         const int i = it / SEGS, seg = it % SEGS;
         if (!mis_s[i] || i + 1 >= R || a.top_k > 0) continue;  // at mismatches only, where the features exist; not under the top-K rule
+        if (a.parent && par_s[i] < -1) continue;                // a node without a valid parent is not judged
         const size_t row = (size_t)b * R + (i + 1);     // the hidden states that encode draft token i
         const char *xd = a.h_draft ? reinterpret_cast<const char *>(a.h_draft) + row * row_bytes_d : nullptr;
         const char *xt = reinterpret_cast<const char *>(a.h_target) + row * row_bytes_t;
@@ -213,7 +231,9 @@ __global__ void __maxnreg__(96) judge_scan_kernel(JudgeArgs a) {
     for (int i = threadIdx.x; i < K; i += blockDim.x) {
         float p = __int_as_float(0x7fc00000);  // NaN where the judge is not consulted
         int rej = 0;
-        if (mis_s[i] && a.top_k > 0) {
+        if (a.parent && par_s[i] < -1) {
+            rej = 1;
+        } else if (mis_s[i] && a.top_k > 0) {
             // top-K rule: accepted iff fewer than top_k entries outrank the draft token; p reports the rank
             const int tk = a.draft_tok[(size_t)b * K + i];
             const bool in_vocab = tk >= 0 && tk < a.V;
@@ -235,7 +255,30 @@ __global__ void __maxnreg__(96) judge_scan_kernel(JudgeArgs a) {
     }
     __syncthreads();
 
-    if (warp == 0) {
+    if (a.parent) {
+        // Walk the nodes in their (topological) order: rej_s becomes "not accepted", mis_s the depth.
+        if (threadIdx.x == 0) {
+            int best = -1, best_depth = 0;
+            for (int n = 0; n < K; n++) {
+                const int q = par_s[n];
+                if (q < -1) {
+                    rej_s[n] = 1;
+                    continue;
+                }
+                const int depth = (q < 0 ? 0 : mis_s[q]) + 1;
+                const int ok = (q < 0 || !rej_s[q]) && !rej_s[n];
+                mis_s[n] = depth;
+                rej_s[n] = !ok;
+                if (ok && depth > best_depth) {  // strict: the lowest index among equally deep nodes
+                    best = n;
+                    best_depth = depth;
+                }
+            }
+            a.accept_len[b] = best_depth;
+            a.next_tok[b] = y_s[best + 1];
+            if (a.best_node) a.best_node[b] = best;
+        }
+    } else if (warp == 0) {
         int first = K;
         for (int base = 0; base < K; base += 32) {
             const int i = base + lane;
@@ -258,7 +301,7 @@ cudaError_t launch_judge_scan(const JudgeArgs &a, cudaStream_t stream) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)a.B);
     cfg.blockDim = dim3(THREADS);
-    cfg.dynamicSmemBytes = (size_t)(3 * a.K + 1) * sizeof(int) + (size_t)a.K * SEGS * sizeof(float);
+    cfg.dynamicSmemBytes = (size_t)(4 * a.K + 1) * sizeof(int) + (size_t)a.K * SEGS * sizeof(float);
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;

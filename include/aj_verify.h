@@ -138,7 +138,8 @@ aj_status aj_set_top_k(aj_handle h, int top_k);
  * cycle enqueued on the handle and advances by one with every cycle, so that consecutive cycles
  * draw independent noise; set it again to replay a cycle.  The draw does not depend on the kernel
  * chosen, on tiling or on vocabulary sharding (the ranks of a vocabulary-parallel group must be
- * given the same temperature, seed and step).  temperature = 0 switches back to greedy
+ * given the same temperature, seed and step; replicas that verify different sequences should be given
+ * different seeds, since every handle numbers its rows from zero).  temperature = 0 switches back to greedy
  * verification.  Errors: AJ_ERR_INVALID_ARG (NULL handle, negative or non-finite temperature),
  * AJ_ERR_UNSUPPORTED (together with the top-K rule, or with AJ_FLAG_ROW_TILES).
  */

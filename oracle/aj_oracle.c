@@ -212,7 +212,7 @@ static int forgiven(double p, float tau)
 int ajo_verify_sampled(const void *h_target, const void *h_draft, const void *W,
                        const int32_t *draft_tok, const float *judge_w, float judge_b, float tau,
                        int dtype, int w_layout, int B, int K, int d, int d_draft, int V, int extra_row,
-                       double temperature, uint64_t seed, uint64_t step,
+                       double temperature, uint64_t seed, uint64_t step, int row0,
                        int32_t *accept_len, int32_t *next_tok, int32_t *target_tok,
                        double *top1, double *gap, double *judge_p);
 
@@ -223,17 +223,19 @@ int ajo_verify(const void *h_target, const void *h_draft, const void *W,
                double *top1, double *gap, double *judge_p)
 {
     return ajo_verify_sampled(h_target, h_draft, W, draft_tok, judge_w, judge_b, tau, dtype, w_layout, B, K, d, d_draft,
-                              V, extra_row, 0.0, 0, 0, accept_len, next_tok, target_tok, top1, gap, judge_p);
+                              V, extra_row, 0.0, 0, 0, 0, accept_len, next_tok, target_tok, top1, gap, judge_p);
 }
 
 /*
  * The whole step with the target's tokens drawn by the Gumbel-max trick at the given temperature
- * (0 = greedy); top1 and gap then refer to the noisy scores logit + temperature * g.
+ * (0 = greedy); top1 and gap then refer to the noisy scores logit + temperature * g.  The noise of row j
+ * of sequence b is that of row index row0 + b * (rows per sequence) + j: row0 = 0 for a whole batch, or
+ * the index of the first row when the sequences given are a slice of a larger batch.
  */
 int ajo_verify_sampled(const void *h_target, const void *h_draft, const void *W,
                        const int32_t *draft_tok, const float *judge_w, float judge_b, float tau,
                        int dtype, int w_layout, int B, int K, int d, int d_draft, int V, int extra_row,
-                       double temperature, uint64_t seed, uint64_t step,
+                       double temperature, uint64_t seed, uint64_t step, int row0,
                        int32_t *accept_len, int32_t *next_tok, int32_t *target_tok,
                        double *top1, double *gap, double *judge_p)
 {
@@ -254,7 +256,7 @@ int ajo_verify_sampled(const void *h_target, const void *h_draft, const void *W,
 #pragma omp parallel for schedule(static)
             for (int v = 0; v < V; v++)
                 for (int j = 0; j < R; j++)
-                    logits[(size_t)j * V + v] += temperature * ajo_gumbel(seed, step, b * R + j, v);
+                    logits[(size_t)j * V + v] += temperature * ajo_gumbel(seed, step, row0 + b * R + j, v);
         }
 
         int32_t *y = target_tok + (size_t)b * R;
@@ -334,7 +336,7 @@ void ajo_tree_accept(int N, const int32_t *tok, const int32_t *parent, const int
  */
 int ajo_verify_tree(const void *h_target, const void *h_draft, const void *W, const int32_t *draft_tok,
                     const int32_t *parent, const float *judge_w, float judge_b, float tau, int dtype, int w_layout,
-                    int B, int N, int d, int d_draft, int V, double temperature, uint64_t seed, uint64_t step,
+                    int B, int N, int d, int d_draft, int V, double temperature, uint64_t seed, uint64_t step, int row0,
                     int32_t *accept_len, int32_t *next_tok, int32_t *best_node, int32_t *target_tok,
                     double *top1, double *gap, double *judge_p)
 {
@@ -354,7 +356,7 @@ int ajo_verify_tree(const void *h_target, const void *h_draft, const void *W, co
 #pragma omp parallel for schedule(static)
             for (int v = 0; v < V; v++)
                 for (int j = 0; j < R; j++)
-                    logits[(size_t)j * V + v] += temperature * ajo_gumbel(seed, step, b * R + j, v);
+                    logits[(size_t)j * V + v] += temperature * ajo_gumbel(seed, step, row0 + b * R + j, v);
         }
         int32_t *y = target_tok + (size_t)b * R;
         for (int j = 0; j < R; j++)

@@ -67,7 +67,7 @@ def _lib():
         L.ajo_verify.argtypes = [vp, vp, vp, ip, fp, cf, cf, ci, ci, ci, ci, ci, ci, ci, ci, ip, ip, ip, dp, dp, dp]
         L.ajo_verify.restype = ci
         u64 = ctypes.c_uint64
-        L.ajo_verify_sampled.argtypes = [vp, vp, vp, ip, fp, cf, cf, ci, ci, ci, ci, ci, ci, ci, ci, ctypes.c_double, u64, u64,
+        L.ajo_verify_sampled.argtypes = [vp, vp, vp, ip, fp, cf, cf, ci, ci, ci, ci, ci, ci, ci, ci, ctypes.c_double, u64, u64, ci,
                                          ip, ip, ip, dp, dp, dp]
         L.ajo_verify_sampled.restype = ci
         L.ajo_philox4x32_10.argtypes = [vp, vp, vp]
@@ -162,7 +162,7 @@ def tree_accept(tok, parent, y, p, tau):
 
 
 def verify_tree(h_target, h_draft, W, draft_tok, parent, judge_w, judge_b, tau, dtype: int, w_layout: int = 0,
-                temperature: float = 0.0, seed: int = 0, step: int = 0) -> OracleResult:
+                temperature: float = 0.0, seed: int = 0, step: int = 0, row0: int = 0) -> OracleResult:
     """The whole step for tree drafts: h_target [B, N+1, d], draft_tok and parent [B, N]; the result also has best_node [B]."""
     ht = np.ascontiguousarray(h_target)
     B, R, d = ht.shape
@@ -182,10 +182,10 @@ def verify_tree(h_target, h_draft, W, draft_tok, parent, judge_w, judge_b, tau, 
     L = _lib()
     vp, ci, u64 = ctypes.c_void_p, ctypes.c_int, ctypes.c_uint64
     L.ajo_verify_tree.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_float, ctypes.c_float, ci, ci, ci, ci, ci, ci, ci,
-                                  ctypes.c_double, u64, u64, vp, vp, vp, vp, vp, vp, vp]
+                                  ctypes.c_double, u64, u64, ci, vp, vp, vp, vp, vp, vp, vp]
     L.ajo_verify_tree.restype = ci
     rc = L.ajo_verify_tree(_ptr(ht), _ptr(hd), _ptr(W), _ptr(tok), _ptr(par), _ptr(w), float(judge_b), float(tau), dtype, w_layout,
-                           B, N, d, dd, V, float(temperature), int(seed), int(step), _ptr(res.accept_len), _ptr(res.next_tok),
+                           B, N, d, dd, V, float(temperature), int(seed), int(step), int(row0), _ptr(res.accept_len), _ptr(res.next_tok),
                            _ptr(best), _ptr(res.target_tok), _ptr(res.top1), _ptr(res.gap), _ptr(res.judge_p))
     if rc:
         raise RuntimeError(f"ajo_verify_tree failed ({rc})")
@@ -211,7 +211,7 @@ def gumbel(seed: int, step: int, j: int, v: int) -> float:
 
 
 def verify(h_target, h_draft, W, draft_tok, judge_w, judge_b, tau, dtype: int, w_layout: int = 0,
-           extra_row: bool = True, temperature: float = 0.0, seed: int = 0, step: int = 0) -> OracleResult:
+           extra_row: bool = True, temperature: float = 0.0, seed: int = 0, step: int = 0, row0: int = 0) -> OracleResult:
     """The whole verify-and-judge step for B sequences (see aj_oracle.c for the definition).
 
     extra_row=False: the hidden states have K rows, not K + 1 (the last draft token is not encoded)."""
@@ -232,7 +232,7 @@ def verify(h_target, h_draft, W, draft_tok, judge_w, judge_b, tau, dtype: int, w
     )
     rc = _lib().ajo_verify_sampled(
         _ptr(ht), _ptr(hd), _ptr(W), _ptr(tok), _ptr(w), float(judge_b), float(tau), dtype, w_layout,
-        B, K, d, dd, V, 1 if extra_row else 0, float(temperature), int(seed), int(step), _ptr(res.accept_len), _ptr(res.next_tok), _ptr(res.target_tok),
+        B, K, d, dd, V, 1 if extra_row else 0, float(temperature), int(seed), int(step), int(row0), _ptr(res.accept_len), _ptr(res.next_tok), _ptr(res.target_tok),
         _ptr(res.top1), _ptr(res.gap), _ptr(res.judge_p),
     )
     if rc:

@@ -143,3 +143,68 @@ def test_c2_under_the_top_k_rule():
                 assert g.accept_len[0] == n and g.next_tok[0] == o.next_tok[0]
     finally:
         case.close()
+
+
+def test_c2_and_c3_with_sampled_target_tokens():
+    """Sampled verification at the full vocabulary: every row of the batch-1 shape on the one-SM kernel, sampled
+    sequences of the batched shape on the CTA-pair kernel; draft tokens planted against the oracle's own draws."""
+    orc = _orc()
+    for cfg, n_sample, path, T, seed, step in ((gen.C2, 1, "umma_vm_128x32", 0.7, 11, 5), (gen.C3, 3, "umma_pair_256x256", 1.0, 12, 40)):
+        Wh, Wd = _W(cfg)
+        ht, hd = gen.make_hidden(cfg)
+        w = gen.make_judge(cfg)
+        seqs = _sample(cfg, n_sample)
+        R = cfg.K + 1
+
+        def oracle(b, tok_b):  # sequence b alone, with the noise its rows have in the full batch
+            return orc.verify(ht[b : b + 1], hd[b : b + 1], Wh, tok_b, w, cfg.judge_b, cfg.tau, cfg.dtype,
+                              temperature=T, seed=seed, step=step, row0=b * R)
+
+        case = DeviceCase(cfg, Wd, ht, hd, w)
+        try:
+            case.handle.set_sampling(T, seed, step)
+            first = case.run(gen.random_draft_tokens(cfg), 0.5)       # the device's own draws, for the sequences the oracle does not see
+            tok = gen.plant_draft_tokens(cfg, first.target_tok)
+            for b in seqs:
+                drawn = oracle(b, np.zeros((1, cfg.K), np.int32)).target_tok
+                tok[b] = gen.plant_draft_tokens(cfg, drawn, rows=[b])[0]
+            case.handle.set_sampling(T, seed, step)                   # the same cycle again
+            g = case.run(tok, cfg.tau)
+            assert g.path == path and g.launches == 2
+            np.testing.assert_array_equal(g.target_tok, first.target_tok)  # same state, same draws
+            for b in seqs:
+                rep = check_parity(oracle(b, tok[b : b + 1]), g, tok[b : b + 1], cfg.tau, seqs=[b])
+                assert rep.rows == R
+            check_self_consistency(g, tok, cfg.tau, cfg.V)
+            greedy = orc.verify(ht[:1], hd[:1], Wh, tok[:1], w, cfg.judge_b, cfg.tau, cfg.dtype).target_tok
+            assert (greedy != g.target_tok[:1]).any()
+        finally:
+            case.close()
+
+
+def test_c2_as_a_tree():
+    """The batch-1 8B shape with its 16 draft tokens arranged as a tree (two candidates per level)."""
+    orc = _orc()
+    cfg = gen.C2
+    Wh, Wd = _W(cfg)
+    ht, hd = gen.make_hidden(cfg)
+    w = gen.make_judge(cfg)
+    N = cfg.K
+    parent = np.array([[-1, -1] + [n - 2 - (n % 2) for n in range(2, N)]], dtype=np.int32)  # nodes 2l, 2l+1 hang under node 2(l-1)
+    y = np.array([[orc.argmax(r)[0] for r in orc.logits(ht[0], Wh, cfg.dtype)]])
+    rng = np.random.default_rng(4)
+    want = y[0][parent[0] + 1]
+    tok = np.where(rng.random(N) < 0.8, want, (want + 1 + rng.integers(0, cfg.V - 1, N)) % cfg.V).astype(np.int32)[None, :]
+    from test_gpu_tree import check_tree, run_tree
+
+    case = DeviceCase(cfg, Wd, ht, hd, w)
+    try:
+        for tau in (0.0, 0.5, 1.0):
+            o = orc.verify_tree(ht, hd, Wh, tok, parent, w, cfg.judge_b, tau, cfg.dtype)
+            g = run_tree(case, tok, parent, tau)
+            assert case.handle.last_gemm_path() == "umma_vm_128x32"
+            assert check_tree(orc, o, g, tok, parent, tau) == 0
+            np.testing.assert_array_equal(g["tt"], y)
+        assert g["acc"][0] == N // 2  # tau = 1: the deepest level
+    finally:
+        case.close()

@@ -595,3 +595,19 @@ def test_tree_step_reduces_to_the_window_step_on_a_chain_and_composes_from_its_p
     # sampled target tokens: the same rows and noise as the window step
     s = orc.verify_tree(ht, hd, W, tok, chain, w, cfg.judge_b, 0.5, dtype, temperature=0.8, seed=3, step=2)
     np.testing.assert_array_equal(s.target_tok, orc.verify(ht, hd, W, tok, w, cfg.judge_b, 0.5, dtype, temperature=0.8, seed=3, step=2).target_tok)
+
+
+def test_a_slice_of_a_batch_draws_the_noise_of_its_own_rows():
+    cfg = gen.Config("slice", B=4, K=3, d=16, d_draft=8, V=40, dtype=F32, sigma_W=0.5, sigma_w=0.3, seed=83)
+    W = gen.make_W(cfg)
+    ht, hd = gen.make_hidden(cfg)
+    w = gen.make_judge(cfg)
+    tok = gen.random_draft_tokens(cfg)
+    full = orc.verify(ht, hd, W, tok, w, cfg.judge_b, 0.5, F32, temperature=1.1, seed=6, step=7)
+    for b in range(cfg.B):
+        one = orc.verify(ht[b : b + 1], hd[b : b + 1], W, tok[b : b + 1], w, cfg.judge_b, 0.5, F32, temperature=1.1, seed=6, step=7, row0=b * 4)
+        np.testing.assert_array_equal(one.target_tok[0], full.target_tok[b])
+        np.testing.assert_array_equal(one.top1[0], full.top1[b])
+        assert one.accept_len[0] == full.accept_len[b]
+    moved = orc.verify(ht[1:2], hd[1:2], W, tok[1:2], w, cfg.judge_b, 0.5, F32, temperature=1.1, seed=6, step=7, row0=0)
+    assert (moved.top1[0] != full.top1[1]).any()

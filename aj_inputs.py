@@ -22,7 +22,7 @@ GENERATOR_VERSION = "aj_inputs/1"
 BF16 = 0  # storage: uint16 holding the upper half of an IEEE fp32
 F32 = 1
 
-_T_W, _T_HT, _T_HD, _T_JW, _T_RATE, _T_TOK = range(6)
+_T_W, _T_HT, _T_HD, _T_JW, _T_RATE, _T_TOK, _T_LRX, _T_LRU, _T_LRN = range(9)
 
 
 @dataclass(frozen=True)
@@ -156,3 +156,17 @@ def plant_draft_tokens(cfg: Config, y: np.ndarray, rows=None) -> np.ndarray:
 def random_draft_tokens(cfg: Config) -> np.ndarray:
     """Draft tokens drawn without reference to any target token (almost all mismatch)."""
     return _rng(cfg.seed, _T_TOK).integers(0, cfg.V, size=(cfg.B, cfg.K)).astype(np.int32)
+
+
+def make_labelled_features(n: int, F: int, dtype: int = BF16, seed: int = 1234, important: float = 0.2, noise: float = 1.0):
+    """A synthetic training set for the classifier: n feature rows [n, F] (i.i.d. unit Gaussians in the given
+    storage, like the hidden states above) and labels [n] uint8, 1 = "important".  A row is labelled important
+    when its projection on a random unit direction plus Gaussian noise of the given size is among the largest
+    `important` share (the paper reports about 20 % important among the mismatches it mines, Section 4.1), so
+    the labels are learnable but not separable."""
+    X = _normal(seed, _T_LRX, (n, F), 1.0, dtype)
+    u = _rng(seed, _T_LRU).standard_normal(F)
+    u /= np.linalg.norm(u)
+    score = to_f64(X, dtype) @ u + noise * _rng(seed, _T_LRN).standard_normal(n)
+    cut = np.quantile(score, 1.0 - important)
+    return X, (score > cut).astype(np.uint8)

@@ -170,6 +170,28 @@ aj_status aj_verify_tree(aj_handle h, const void *h_target, const void *h_draft,
                          float *top1_val, float *judge_p, void *cuda_stream);
 
 /*
+ * Fit the classifier (the paper's Section 3.2 "Classifier model & training", Section 4.1 and its appendix
+ * on classifier ablations: a logistic regression with L2 regularisation, fitted as scikit-learn does with
+ * coefficient C, e.g. 1e-4 for the 8B / 70B pair).  The result is the minimiser of
+ *     f(w, b) = 1/2 w.w + C * sum_i log(1 + exp(-s_i (x_i.w + b))),   s_i = +1 if labels[i] != 0 else -1
+ * (intercept not regularised), found by L-BFGS with every evaluation of f and its gradient done in one
+ * pass of a kernel over X.
+ *   X       [n, F] DEVICE, row-major, dtype as given; row i is the concatenation [h_draft ; h_target] of a
+ *           mined mismatch, the layout judge_w expects.  16-byte aligned, F * element size a multiple of 16.
+ *   labels  [n] DEVICE bytes, non-zero = important.
+ *   w_out   [F] DEVICE fp32, b_out HOST: the fitted judge_w and judge_b.
+ *   iters_out (HOST, optional) receives {iterations, evaluations}; grad_out (HOST, optional) the largest
+ *           absolute component of the gradient of f at the result.
+ * Stops when that component is <= tol, after max_iter iterations, or when no step lowers f any more
+ * (evaluations are fp32 per row, fp64 across rows).  Synchronous; allocates and frees its own workspace
+ * ((SMs + 2) * F floats).  Errors: AJ_ERR_INVALID_ARG, AJ_ERR_UNSUPPORTED (alignment, or F too wide for
+ * four rows to fit in shared memory: about 13 000 features in bf16), AJ_ERR_NOT_SM100, AJ_ERR_CUDA.
+ */
+aj_status aj_lr_fit(int device, const void *X, const uint8_t *labels, long long n, int F, aj_dtype dtype, float C,
+                    int max_iter, float tol, float *w_out, float *b_out, int *iters_out, float *grad_out,
+                    void *cuda_stream);
+
+/*
  * The same cycle for a caller whose per-cycle tensors live in host memory: h_target, h_draft and
  * draft_tok are HOST pointers and are copied to the handle's staging buffers; accept_len and
  * next_tok (and target_tok, if not NULL) are HOST pointers and are copied back.  W_lm and judge_w

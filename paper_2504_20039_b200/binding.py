@@ -19,7 +19,7 @@ AJ_FLAG_FORCE_SIMT, AJ_FLAG_TIME_KERNELS, AJ_FLAG_ROW_TILES, AJ_FLAG_ONE_SM, AJ_
 
 EXPORTS = (
     "aj_create", "aj_verify", "aj_verify_host", "aj_last_status", "aj_last_gemm_ms", "aj_gemm_ms_stats", "aj_last_launch_count",
-    "aj_last_gemm_path", "aj_pair_schedule", "aj_destroy", "aj_set_top_k", "aj_set_sampling", "aj_verify_tree", "aj_shard_exchange_bytes", "aj_shard_exchange_alloc", "aj_shard_exchange_free", "aj_shard_range", "aj_create_sharded",
+    "aj_last_gemm_path", "aj_pair_schedule", "aj_destroy", "aj_set_top_k", "aj_set_sampling", "aj_verify_tree", "aj_lr_fit", "aj_shard_exchange_bytes", "aj_shard_exchange_alloc", "aj_shard_exchange_free", "aj_shard_range", "aj_create_sharded",
     "aj_shard_project", "aj_shard_finish", "aj_ipc_export", "aj_ipc_import", "aj_ipc_close", "aj_status_string", "aj_version", "aj_verify_static",
 )
 
@@ -49,6 +49,9 @@ def lib() -> ctypes.CDLL:
         L.aj_verify.restype = ci
         L.aj_verify_tree.argtypes = [vp, vp, vp, vp, vp, vp, vp, cf, cf, ci, ci, ci, ci, vp, vp, vp, vp, vp, vp, vp]
         L.aj_verify_tree.restype = ci
+        L.aj_lr_fit.argtypes = [ci, vp, vp, ctypes.c_longlong, ci, ci, cf, ci, cf, vp, ctypes.POINTER(ctypes.c_float),
+                                ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_float), vp]
+        L.aj_lr_fit.restype = ci
         L.aj_verify_host.argtypes = [vp, vp, vp, vp, vp, vp, cf, cf, ci, ci, ci, ci, vp, vp, vp, vp]
         L.aj_verify_host.restype = ci
         L.aj_last_status.argtypes = [vp]
@@ -97,6 +100,19 @@ def lib() -> ctypes.CDLL:
         L.aj_version.restype = ctypes.c_char_p
         _lib = L
     return _lib
+
+
+def lr_fit(device: int, X, labels, n: int, F: int, dtype: int, C: float, w_out, max_iter: int = 500, tol: float = 1e-4,
+           stream: int = 0, check: bool = True):
+    """aj_lr_fit: fit the classifier on device-resident features; returns (status, b, iterations, evaluations, max |grad|)."""
+    b = ctypes.c_float()
+    it = (ctypes.c_int * 2)()
+    gn = ctypes.c_float()
+    st = lib().aj_lr_fit(device, _ptr(X), _ptr(labels), n, F, dtype, float(C), max_iter, float(tol), _ptr(w_out),
+                         ctypes.byref(b), it, ctypes.byref(gn), stream or None)
+    if check and st != AJ_OK:
+        raise AjError(st, "aj_lr_fit")
+    return st, b.value, it[0], it[1], gn.value
 
 
 def status_string(status: int) -> str:

@@ -324,7 +324,7 @@ def reference_arm(args):
         return
     from oracle import aj_oracle as orc
 
-    cfg = workload(args.workload if args.workload != "sweep" else "c2")
+    cfg = workload(args.workload if args.workload not in ("sweep", "lr_fit") else "c2")
     steps = args.steps if args.steps is not None else 3
     warmup = args.warmup if args.warmup is not None else 1
     W = gen.make_W(cfg)
@@ -347,12 +347,90 @@ def reference_arm(args):
     print(json.dumps(line))
 
 
+def lr_fit_line(args):
+    """The classifier fit at the paper's training-set size (Section 4.1: about 130 K mined mismatches, 20 %
+    important; features [h_draft ; h_target] of the 1B / 8B pair; C = 1e-4): whole fits timed with CUDA events,
+    HBM roofline of the loss + gradient kernel from its share of the fit (one pass over X per evaluation)."""
+    import torch
+
+    import paper_2504_20039_b200 as aj
+
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    n, F, C = 131072, 6144, 1e-4
+    dev = torch.device("cuda:0")
+    torch.cuda.set_device(dev)
+    g = torch.Generator(device=dev).manual_seed(20250420)
+    X = torch.empty((n, F), dtype=torch.bfloat16, device=dev)
+    u = torch.randn(F, generator=g, device=dev)
+    u /= u.norm()
+    score = torch.empty(n, device=dev)
+    for i in range(0, n, 8192):  # unit Gaussians, labelled by a noisy projection: the top 20 % are "important"
+        blk = torch.randn((min(8192, n - i), F), generator=g, device=dev)
+        X[i : i + blk.shape[0]] = blk.to(torch.bfloat16)
+        score[i : i + blk.shape[0]] = X[i : i + blk.shape[0]].float() @ u
+    score += torch.randn(n, generator=g, device=dev)
+    y = (score > torch.quantile(score[:: max(1, n // 65536)], 0.8)).to(torch.uint8)
+    w = torch.zeros(F, dtype=torch.float32, device=dev)
+    steps = args.steps if args.steps is not None else 3
+    warmup = args.warmup if args.warmup is not None else 1
+    stream = torch.cuda.current_stream().cuda_stream
+    for _ in range(warmup):
+        aj.lr_fit(0, X, y, n, F, aj.AJ_BF16, C, w, stream=stream)
+    pk = peaks()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(0) as cs:
+        torch.cuda.synchronize()
+        t0 = time.time()
+        e0.record()
+        evals, kernel_ms = 0, 0.0
+        for _ in range(steps):
+            st, b, iters, ev, gnorm = aj.lr_fit(0, X, y, n, F, aj.AJ_BF16, C, w, stream=stream)
+            evals += ev
+            kernel_ms += aj.lr_fit.kernel_ms
+        e1.record()
+        torch.cuda.synchronize()
+        t1 = time.time()
+    ms = e0.elapsed_time(e1)
+    byts = float(n) * F * 2
+    per_eval_s = kernel_ms * 1e-3 / evals  # the loss + gradient kernel alone (CUDA events inside the library)
+    line = {
+        "metric": "lr_fit_rows_per_s", "value": n * evals / (ms * 1e-3), "unit": "rows/s", "n_gpus": 1, "steps": steps, "warmup": warmup,
+        "ms_per_step": ms / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16 features, fp32 accumulate, fp64 optimiser",
+        "data": "synthetic", "config": {"workload": "lr_fit_131072x6144", "n": n, "F": F, "C": C, "iterations": iters, "evaluations_per_fit": evals // steps,
+                                          "max_abs_gradient": gnorm, "intercept": b, "positives": float(y.float().mean().item()),
+                                          "l2": "X is 1.61 GB, larger than the 126 MB L2"},
+        "clocks": cs.summary(t0, t1),
+        "roofline": {"bound": "hbm", "achieved": byts / per_eval_s / 1e9, "peak": pk["hbm_gbs"], "unit": "GB/s",
+                     "frac": byts / per_eval_s / 1e9 / pk["hbm_gbs"], "traffic": None, "peak_source": f"of {pk['source']}",
+                     "kernel_ms": kernel_ms / evals, "note": "the loss + gradient kernel, one pass over X per evaluation; a whole fit also allocates its workspace, copies w down and the gradient up per evaluation and runs L-BFGS on the host",
+                     "algorithmic_bytes": byts},
+        "gpu_launches": 2 * evals, "e2e": None,
+    }
+    if not args.no_cpu:
+        from oracle import aj_lr_oracle as lro
+
+        rows = 4096
+        Xs = X[:rows].float().cpu().numpy().astype(np.float64)
+        ys = y[:rows].cpu().numpy()
+        wz = np.zeros(F)
+        t = time.time()
+        passes = 0
+        while time.time() - t < 10.0:
+            lro.objective(Xs, ys, C, wz, 0.0)
+            passes += 1
+        dt = time.time() - t
+        line["cpu_baseline"] = {"value": rows * passes / dt, "unit": "rows/s", "cores": os.cpu_count(), "kind": "oracle",
+                                "sample": f"{passes} evaluations of the objective and its gradient on the first {rows} rows (fp64 numpy)"}
+    print(json.dumps(line))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
-    ap.add_argument("--workload", default="c2", choices=["c2", "c3", "c4", "sweep"])
+    ap.add_argument("--workload", default="c2", choices=["c2", "c3", "c4", "sweep", "lr_fit"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extra", action="store_true", help="skip the batched configurations reported under 'extra'")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline")
@@ -366,6 +444,8 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         return reference_arm(args)
+    if args.workload == "lr_fit":
+        return lr_fit_line(args)
 
     import torch
 

@@ -180,15 +180,16 @@ aj_status aj_verify_tree(aj_handle h, const void *h_target, const void *h_draft,
  *           mined mismatch, the layout judge_w expects.  16-byte aligned, F * element size a multiple of 16.
  *   labels  [n] DEVICE bytes, non-zero = important.
  *   w_out   [F] DEVICE fp32, b_out HOST: the fitted judge_w and judge_b.
- *   iters_out (HOST, optional) receives {iterations, evaluations}; grad_out (HOST, optional) the largest
- *           absolute component of the gradient of f at the result.
+ *   iters_out (HOST, optional, 2 ints) receives {iterations, evaluations}; stats_out (HOST, optional, 2 floats)
+ *           {the largest absolute component of the gradient of f at the result, the milliseconds the
+ *           evaluations' loss + gradient kernel took in total (CUDA events)}.
  * Stops when that component is <= tol, after max_iter iterations, or when no step lowers f any more
  * (evaluations are fp32 per row, fp64 across rows).  Synchronous; allocates and frees its own workspace
- * ((SMs + 2) * F floats).  Errors: AJ_ERR_INVALID_ARG, AJ_ERR_UNSUPPORTED (alignment, or F too wide for
- * four rows to fit in shared memory: about 13 000 features in bf16), AJ_ERR_NOT_SM100, AJ_ERR_CUDA.
+ * ((SMs + 2) * F floats).  Errors: AJ_ERR_INVALID_ARG, AJ_ERR_UNSUPPORTED (alignment, or rows wider than
+ * 32 KB: 16 384 features in bf16, 8 192 in fp32), AJ_ERR_NOT_SM100, AJ_ERR_CUDA.
  */
 aj_status aj_lr_fit(int device, const void *X, const uint8_t *labels, long long n, int F, aj_dtype dtype, float C,
-                    int max_iter, float tol, float *w_out, float *b_out, int *iters_out, float *grad_out,
+                    int max_iter, float tol, float *w_out, float *b_out, int *iters_out, float *stats_out,
                     void *cuda_stream);
 
 /*

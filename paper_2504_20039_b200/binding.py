@@ -104,15 +104,17 @@ def lib() -> ctypes.CDLL:
 
 def lr_fit(device: int, X, labels, n: int, F: int, dtype: int, C: float, w_out, max_iter: int = 500, tol: float = 1e-4,
            stream: int = 0, check: bool = True):
-    """aj_lr_fit: fit the classifier on device-resident features; returns (status, b, iterations, evaluations, max |grad|)."""
+    """aj_lr_fit: fit the classifier on device-resident features; returns (status, b, iterations, evaluations, max |grad|);
+    the kernel milliseconds of the fit are left in lr_fit.kernel_ms."""
     b = ctypes.c_float()
     it = (ctypes.c_int * 2)()
-    gn = ctypes.c_float()
+    stats = (ctypes.c_float * 2)()
     st = lib().aj_lr_fit(device, _ptr(X), _ptr(labels), n, F, dtype, float(C), max_iter, float(tol), _ptr(w_out),
-                         ctypes.byref(b), it, ctypes.byref(gn), stream or None)
+                         ctypes.byref(b), it, stats, stream or None)
     if check and st != AJ_OK:
         raise AjError(st, "aj_lr_fit")
-    return st, b.value, it[0], it[1], gn.value
+    lr_fit.kernel_ms = stats[1]
+    return st, b.value, it[0], it[1], stats[0]
 
 
 def status_string(status: int) -> str:

@@ -4,10 +4,10 @@
 //
 // (the intercept is not regularised; this is scikit-learn's convention, which the paper uses).
 // One evaluation of f and its gradient is ONE pass over X: a CTA stages a block of rows in shared
-// memory (cp.async, four buffers, three in flight), computes the rows' scores z = x.w + b from the
+// memory (cp.async, four buffers, two or three in flight), computes the rows' scores z = x.w + b from the
 // staged copy, turns them into residuals r_i = -C s_i sigma(-s_i z_i), and adds r_i x_i to its
 // own gradient accumulator from the same staged copy.  Every thread owns a fixed set of 16-byte
-// feature chunks in both phases.  CTAs write their partial gradients and partial losses to
+// feature chunks in both phases and keeps their weights and gradient sums in registers.  CTAs write their partial gradients and partial losses to
 // separate slots, which a second kernel (gradient) and the host (loss, intercept) add in a fixed
 // order, so an evaluation does not depend on scheduling.  The minimiser is found by L-BFGS on the
 // host in fp64 (two-loop recursion, Armijo backtracking); only w travels down and the gradient up.
@@ -18,16 +18,18 @@
 #include <math.h>
 #include <stdint.h>
 
+#include <type_traits>
 #include <vector>
 
 namespace aj {
 
 namespace {
 
-constexpr int LR_THREADS = 256;
+constexpr int LR_THREADS = 512;
 constexpr int LR_WARPS = LR_THREADS / 32;
 constexpr int LR_NBUF = 4;     // shared-memory buffers of one row block each
 constexpr int LR_RB_MAX = 8;   // rows per block at most (score accumulators per thread)
+constexpr int LR_MAXC = 4;     // 16-byte feature chunks a thread owns at most: rows of up to 32 KB
 constexpr int LR_SMEM_BUDGET = 220 * 1024;
 
 __device__ inline void cp_async_16(void *smem_dst, const void *gmem_src) {
@@ -37,7 +39,7 @@ __device__ inline void cp_async_16(void *smem_dst, const void *gmem_src) {
 __device__ inline void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N> __device__ inline void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-// eight consecutive features of a staged row as floats
+// the features of one 16-byte chunk of a staged row as floats
 template <bool BF16> struct Chunk;
 template <> struct Chunk<true> {
     static constexpr int ELEMS = 8;
@@ -74,31 +76,39 @@ struct LrArgs {
     double *partial_gb;      // [grid]
 };
 
-template <bool BF16>
+// Thread t owns the chunks t, t + LR_THREADS, ... of every row: their weights and its share of the
+// CTA's gradient stay in registers for the whole launch; shared memory holds only the staged rows.
+// MAXC: chunks a thread owns at most; RB: rows per block (a shorter last block takes the guarded path).
+template <bool BF16, int MAXC, int RB>
 __global__ void __launch_bounds__(LR_THREADS, 1) lr_loss_grad_kernel(const LrArgs a) {
     extern __shared__ __align__(16) char lr_smem[];
     constexpr int EPC = Chunk<BF16>::ELEMS;
-    const int F = a.F, rb = a.rb, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    constexpr int rb = RB;
+    const int F = a.F, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int chunks = F / EPC;
-    const size_t stage_bytes = (size_t)rb * a.row_bytes;
-    float *w_s = reinterpret_cast<float *>(lr_smem);           // [F]
-    float *acc_s = w_s + F;                                     // [F] this CTA's gradient
-    float *z_part = acc_s + F;                                  // [LR_WARPS][LR_RB_MAX]
-    float *r_s = z_part + LR_WARPS * LR_RB_MAX;                 // [LR_RB_MAX]
-    char *x_s = reinterpret_cast<char *>(r_s + LR_RB_MAX);      // [LR_NBUF][rb rows]
+    const int row_bytes = (int)a.row_bytes;           // at most 32 KB
+    const int stage_bytes = rb * row_bytes;
+    float *z_part = reinterpret_cast<float *>(lr_smem);         // [2][LR_WARPS][LR_RB_MAX], alternating between blocks
+    char *x_s = reinterpret_cast<char *>(z_part + 2 * LR_WARPS * LR_RB_MAX);  // [LR_NBUF][rb rows]
 
-    for (int f = tid; f < F; f += LR_THREADS) {
-        w_s[f] = a.w[f];
-        acc_s[f] = 0.0f;
+    float wv[MAXC][8], g[MAXC][8];
+#pragma unroll
+    for (int k = 0; k < MAXC; k++) {
+        const int c = tid + k * LR_THREADS;
+#pragma unroll
+        for (int i = 0; i < 8; i++) {
+            wv[k][i] = (c < chunks && i < EPC) ? a.w[(size_t)c * EPC + i] : 0.0f;
+            g[k][i] = 0.0f;
+        }
     }
     const long long nblk = (a.n + rb - 1) / rb;
     auto issue = [&](long long blk, int buf) {
         if (blk < nblk) {
             const long long row0 = blk * rb;
-            const size_t bytes = (size_t)(a.n - row0 < rb ? a.n - row0 : rb) * a.row_bytes;
+            const int bytes = (int)(a.n - row0 < rb ? a.n - row0 : rb) * row_bytes;
             const char *src = a.X + (size_t)row0 * a.row_bytes;
-            char *dst = x_s + (size_t)buf * stage_bytes;
-            for (size_t off = (size_t)tid * 16; off < bytes; off += (size_t)LR_THREADS * 16) cp_async_16(dst + off, src + off);
+            char *dst = x_s + buf * stage_bytes;
+            for (int off = tid * 16; off < bytes; off += LR_THREADS * 16) cp_async_16(dst + off, src + off);
         }
         cp_async_commit();  // an empty group keeps the count of pending groups uniform
     };
@@ -107,87 +117,97 @@ __global__ void __launch_bounds__(LR_THREADS, 1) lr_loss_grad_kernel(const LrArg
     double loss = 0.0, gb = 0.0;  // lane 0 of warp 0 only
     long long it = 0;
     for (long long blk = blockIdx.x; blk < nblk; blk += gridDim.x, ++it) {
-        issue(blk + (long long)(LR_NBUF - 1) * gridDim.x, (int)((it + LR_NBUF - 1) % LR_NBUF));
-        cp_async_wait<LR_NBUF - 1>();
-        __syncthreads();  // the block's rows (and, the first time, w_s) are visible to every thread
-        const char *xb = x_s + (size_t)(it % LR_NBUF) * stage_bytes;
+        cp_async_wait<LR_NBUF - 2>();
+        __syncthreads();  // the block's rows are visible to every thread, and every thread is done with the block before
+        issue(blk + (long long)(LR_NBUF - 1) * gridDim.x, (int)((it + LR_NBUF - 1) % LR_NBUF));  // refills that block's buffer
+        const char *xb = x_s + (int)(it % LR_NBUF) * stage_bytes;
         const long long row0 = blk * rb;
         const int rows = (int)(a.n - row0 < rb ? a.n - row0 : rb);
+        const bool full = rows == rb;  // all blocks but possibly the last
 
         // scores: every thread adds its chunks' share of every row's dot product
-        float zp[LR_RB_MAX];
+        float zp[RB];
 #pragma unroll
-        for (int r = 0; r < LR_RB_MAX; r++) zp[r] = 0.0f;
-        for (int c = tid; c < chunks; c += LR_THREADS) {
-            float wv[8];
+        for (int r = 0; r < RB; r++) zp[r] = 0.0f;
 #pragma unroll
-            for (int i = 0; i < 8; i++) wv[i] = i < EPC ? w_s[c * EPC + i] : 0.0f;
+        for (int k = 0; k < MAXC; k++) {
+            const int c = tid + k * LR_THREADS;
+            if (c < chunks) {
+                const char *xc = xb + c * 16;
 #pragma unroll
-            for (int r = 0; r < LR_RB_MAX; r++) {
-                if (r < rows) {
-                    float x[8];
-                    Chunk<BF16>::load(xb + (size_t)r * a.row_bytes + (size_t)c * 16, x);
+                for (int r = 0; r < RB; r++) {
+                    if (full || r < rows) {
+                        float x[8];
+                        Chunk<BF16>::load(xc + r * row_bytes, x);
 #pragma unroll
-                    for (int i = 0; i < EPC; i++) zp[r] = fmaf(x[i], wv[i], zp[r]);
+                        for (int i = 0; i < EPC; i++) zp[r] = fmaf(x[i], wv[k][i], zp[r]);
+                    }
                 }
             }
         }
 #pragma unroll
-        for (int r = 0; r < LR_RB_MAX; r++) {
+        for (int r = 0; r < RB; r++) {
 #pragma unroll
             for (int off = 16; off > 0; off >>= 1) zp[r] += __shfl_xor_sync(0xffffffffu, zp[r], off);
-            if (lane == 0) z_part[warp * LR_RB_MAX + r] = zp[r];
+            if (lane == 0) z_part[((int)(it & 1) * LR_WARPS + warp) * LR_RB_MAX + r] = zp[r];
         }
         __syncthreads();
-        if (warp == 0) {  // lane r finishes row r; the other lanes contribute zeros to the sums
-            float softplus = 0.0f, r = 0.0f;
-            if (lane < rows) {
-                float z = a.b;
+        // every warp finishes the rows itself (lane r: row r), so that none waits for another
+        float softplus = 0.0f, res = 0.0f;
+        if (lane < rows) {
+            float z = a.b;
 #pragma unroll
-                for (int k = 0; k < LR_WARPS; k++) z += z_part[k * LR_RB_MAX + lane];  // fixed order
-                const float s = a.labels[row0 + lane] ? 1.0f : -1.0f;
-                const float t = s * z;
-                const float e = expf(-fabsf(t));
-                softplus = log1pf(e) + fmaxf(-t, 0.0f);                            // log(1 + exp(-t))
-                const float sig = t >= 0.0f ? e / (1.0f + e) : 1.0f / (1.0f + e);  // sigma(-t)
-                r = -a.C * s * sig;
-                r_s[lane] = r;
-            }
-            double l = softplus, g = r;
+            for (int k = 0; k < LR_WARPS; k++) z += z_part[((int)(it & 1) * LR_WARPS + k) * LR_RB_MAX + lane];  // fixed order
+            const float s = a.labels[row0 + lane] ? 1.0f : -1.0f;
+            const float t = s * z;
+            const float e = expf(-fabsf(t));
+            softplus = log1pf(e) + fmaxf(-t, 0.0f);                            // log(1 + exp(-t))
+            const float sig = t >= 0.0f ? e / (1.0f + e) : 1.0f / (1.0f + e);  // sigma(-t)
+            res = -a.C * s * sig;
+        }
+        if (warp == 0) {  // the sums are kept by one warp; lanes without a row contribute zeros
+            double l = softplus, gg = res;
             for (int off = 16; off > 0; off >>= 1) {
                 l += __shfl_xor_sync(0xffffffffu, l, off);
-                g += __shfl_xor_sync(0xffffffffu, g, off);
+                gg += __shfl_xor_sync(0xffffffffu, gg, off);
             }
             if (lane == 0) {
                 loss += l;
-                gb += g;
+                gb += gg;
             }
         }
-        __syncthreads();
+        float rr_row[RB];
+#pragma unroll
+        for (int r = 0; r < RB; r++) rr_row[r] = __shfl_sync(0xffffffffu, res, r);
 
         // gradient: the same chunks, the same staged rows
-        for (int c = tid; c < chunks; c += LR_THREADS) {
-            float g[8];
 #pragma unroll
-            for (int i = 0; i < 8; i++) g[i] = i < EPC ? acc_s[c * EPC + i] : 0.0f;
+        for (int k = 0; k < MAXC; k++) {
+            const int c = tid + k * LR_THREADS;
+            if (c < chunks) {
+                const char *xc = xb + c * 16;
 #pragma unroll
-            for (int r = 0; r < LR_RB_MAX; r++) {
-                if (r < rows) {
-                    float x[8];
-                    Chunk<BF16>::load(xb + (size_t)r * a.row_bytes + (size_t)c * 16, x);
-                    const float rr = r_s[r];
+                for (int r = 0; r < RB; r++) {
+                    if (full || r < rows) {
+                        float x[8];
+                        Chunk<BF16>::load(xc + r * row_bytes, x);
+                        const float rr = rr_row[r];
 #pragma unroll
-                    for (int i = 0; i < EPC; i++) g[i] = fmaf(rr, x[i], g[i]);
+                        for (int i = 0; i < EPC; i++) g[k][i] = fmaf(rr, x[i], g[k][i]);
+                    }
                 }
             }
-#pragma unroll
-            for (int i = 0; i < EPC; i++) acc_s[c * EPC + i] = g[i];
         }
-        __syncthreads();  // the buffer may be refilled, r_s and z_part rewritten
     }
     cp_async_wait<0>();
-    __syncthreads();
-    for (int f = tid; f < F; f += LR_THREADS) a.partial_g[(size_t)blockIdx.x * F + f] = acc_s[f];
+#pragma unroll
+    for (int k = 0; k < MAXC; k++) {
+        const int c = tid + k * LR_THREADS;
+        if (c < chunks) {
+#pragma unroll
+            for (int i = 0; i < EPC; i++) a.partial_g[(size_t)blockIdx.x * F + (size_t)c * EPC + i] = g[k][i];
+        }
+    }
     if (tid == 0) {
         a.partial_loss[blockIdx.x] = loss;
         a.partial_gb[blockIdx.x] = gb;
@@ -223,7 +243,7 @@ struct Workspace {
 }  // namespace aj
 
 extern "C" aj_status aj_lr_fit(int device, const void *X, const uint8_t *labels, long long n, int F, aj_dtype dtype, float C,
-                               int max_iter, float tol, float *w_out, float *b_out, int *iters_out, float *grad_out,
+                               int max_iter, float tol, float *w_out, float *b_out, int *iters_out, float *stats_out,
                                void *cuda_stream) {
     using namespace aj;
     if (!X || !labels || !w_out || !b_out || n < 1 || F < 1 || !(C > 0.0f) || max_iter < 1 || !(tol >= 0.0f)) return AJ_ERR_INVALID_ARG;
@@ -231,8 +251,9 @@ extern "C" aj_status aj_lr_fit(int device, const void *X, const uint8_t *labels,
     const size_t esz = dtype == AJ_BF16 ? 2 : 4;
     const size_t row_bytes = (size_t)F * esz;
     if (row_bytes % 16 != 0 || (reinterpret_cast<uintptr_t>(X) & 15) != 0) return AJ_ERR_UNSUPPORTED;
-    const size_t fixed = (size_t)F * 8 + (LR_WARPS * LR_RB_MAX + LR_RB_MAX) * sizeof(float);
-    if (fixed + LR_NBUF * row_bytes > (size_t)LR_SMEM_BUDGET) return AJ_ERR_UNSUPPORTED;  // a row block must fit four times
+    const size_t fixed = 2 * LR_WARPS * LR_RB_MAX * sizeof(float);
+    if (row_bytes > (size_t)LR_MAXC * LR_THREADS * 16) return AJ_ERR_UNSUPPORTED;  // a thread owns at most LR_MAXC chunks of a row
+    if (fixed + LR_NBUF * row_bytes > (size_t)LR_SMEM_BUDGET) return AJ_ERR_UNSUPPORTED;  // a row must fit four times
     int rb = (int)((LR_SMEM_BUDGET - fixed) / (LR_NBUF * row_bytes));
     if (rb > LR_RB_MAX) rb = LR_RB_MAX;
     const size_t smem = fixed + (size_t)LR_NBUF * rb * row_bytes;
@@ -243,14 +264,39 @@ extern "C" aj_status aj_lr_fit(int device, const void *X, const uint8_t *labels,
         int d;
         ~Restore() { cudaSetDevice(d); }
     } restore{prev};
-    cudaDeviceProp prop;
-    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return AJ_ERR_CUDA;
-    if (prop.major != 10) return AJ_ERR_NOT_SM100;
+    int cc_major = 0, num_sms = 0;
+    if (cudaDeviceGetAttribute(&cc_major, cudaDevAttrComputeCapabilityMajor, device) != cudaSuccess ||
+        cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess)
+        return AJ_ERR_CUDA;
+    if (cc_major != 10) return AJ_ERR_NOT_SM100;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    auto kernel = dtype == AJ_BF16 ? lr_loss_grad_kernel<true> : lr_loss_grad_kernel<false>;
+    const int maxc = (int)((row_bytes / 16 + LR_THREADS - 1) / LR_THREADS);  // 1 .. LR_MAXC
+    using Kernel = void (*)(const LrArgs);
+    auto pick_rb = [&](auto bf, auto mc) -> Kernel {
+        constexpr bool B = decltype(bf)::value;
+        constexpr int M = decltype(mc)::value;
+        switch (rb) {
+            case 1: return lr_loss_grad_kernel<B, M, 1>;
+            case 2: return lr_loss_grad_kernel<B, M, 2>;
+            case 3: return lr_loss_grad_kernel<B, M, 3>;
+            case 4: return lr_loss_grad_kernel<B, M, 4>;
+            case 5: return lr_loss_grad_kernel<B, M, 5>;
+            case 6: return lr_loss_grad_kernel<B, M, 6>;
+            case 7: return lr_loss_grad_kernel<B, M, 7>;
+            default: return lr_loss_grad_kernel<B, M, 8>;
+        }
+    };
+    auto pick_mc = [&](auto bf) -> Kernel {
+        switch (maxc) {
+            case 1: return pick_rb(bf, std::integral_constant<int, 1>{});
+            case 2: return pick_rb(bf, std::integral_constant<int, 2>{});
+            default: return pick_rb(bf, std::integral_constant<int, LR_MAXC>{});
+        }
+    };
+    Kernel kernel = dtype == AJ_BF16 ? pick_mc(std::true_type{}) : pick_mc(std::false_type{});
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return AJ_ERR_CUDA;
     const long long nblk = (n + rb - 1) / rb;
-    const int grid = (int)(nblk < prop.multiProcessorCount ? nblk : prop.multiProcessorCount);
+    const int grid = (int)(nblk < num_sms ? nblk : num_sms);
 
     Workspace ws;
     if (cudaMalloc(&ws.w_dev, F * sizeof(float)) != cudaSuccess || cudaMalloc(&ws.g_dev, F * sizeof(float)) != cudaSuccess ||
@@ -264,6 +310,16 @@ extern "C" aj_status aj_lr_fit(int device, const void *X, const uint8_t *labels,
 
     const int D = F + 1;  // the intercept is the last coordinate
     bool cuda_ok = true;
+    cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+    if (cudaEventCreate(&ev0) != cudaSuccess || cudaEventCreate(&ev1) != cudaSuccess) return AJ_ERR_CUDA;
+    struct Events {
+        cudaEvent_t a, b;
+        ~Events() {
+            cudaEventDestroy(a);
+            cudaEventDestroy(b);
+        }
+    } events{ev0, ev1};
+    double kernel_ms = 0.0;
     // f and its gradient at v (fp64 on the host, w rounded to fp32 for the device)
     auto eval = [&](const std::vector<double> &v, std::vector<double> &grad) -> double {
         for (int f = 0; f < F; f++) ws.w_host[f] = (float)v[f];
@@ -281,13 +337,17 @@ extern "C" aj_status aj_lr_fit(int device, const void *X, const uint8_t *labels,
         a.partial_loss = ws.partial_ld;
         a.partial_gb = ws.partial_ld + grid;
         cuda_ok = cuda_ok && cudaMemcpyAsync(ws.w_dev, ws.w_host, F * sizeof(float), cudaMemcpyHostToDevice, stream) == cudaSuccess;
+        cudaEventRecord(ev0, stream);
         kernel<<<grid, LR_THREADS, smem, stream>>>(a);
+        cudaEventRecord(ev1, stream);
         lr_reduce_kernel<<<(F + 255) / 256, 256, 0, stream>>>(ws.partial_g, grid, F, ws.g_dev);
         cuda_ok = cuda_ok && cudaGetLastError() == cudaSuccess;
         cuda_ok = cuda_ok && cudaMemcpyAsync(ws.g_host, ws.g_dev, F * sizeof(float), cudaMemcpyDeviceToHost, stream) == cudaSuccess;
         cuda_ok = cuda_ok && cudaMemcpyAsync(ws.ld_host, ws.partial_ld, 2 * (size_t)grid * sizeof(double), cudaMemcpyDeviceToHost, stream) == cudaSuccess;
         cuda_ok = cuda_ok && cudaStreamSynchronize(stream) == cudaSuccess;
         if (!cuda_ok) return 0.0;
+        float ms = 0.0f;
+        if (cudaEventElapsedTime(&ms, ev0, ev1) == cudaSuccess) kernel_ms += ms;
         double loss = 0.0, gb = 0.0, ww = 0.0;
         for (int k = 0; k < grid; k++) {
             loss += ws.ld_host[k];
@@ -388,6 +448,9 @@ extern "C" aj_status aj_lr_fit(int device, const void *X, const uint8_t *labels,
         iters_out[0] = iters;
         iters_out[1] = evals;
     }
-    if (grad_out) *grad_out = (float)max_abs(g);
+    if (stats_out) {
+        stats_out[0] = (float)max_abs(g);
+        stats_out[1] = (float)kernel_ms;
+    }
     return AJ_OK;
 }

@@ -186,7 +186,7 @@ aj_status aj_verify_tree(aj_handle h, const void *h_target, const void *h_draft,
  * Stops when that component is <= tol, after max_iter iterations, or when no step lowers f any more
  * (evaluations are fp32 per row, fp64 across rows).  Synchronous; allocates and frees its own workspace
  * ((SMs + 2) * F floats).  Errors: AJ_ERR_INVALID_ARG, AJ_ERR_UNSUPPORTED (alignment, or rows wider than
- * 32 KB: 16 384 features in bf16, 8 192 in fp32), AJ_ERR_NOT_SM100, AJ_ERR_CUDA.
+ * 48 KB: 24 576 features in bf16, 12 288 in fp32), AJ_ERR_NOT_SM100, AJ_ERR_CUDA.
  */
 aj_status aj_lr_fit(int device, const void *X, const uint8_t *labels, long long n, int F, aj_dtype dtype, float C,
                     int max_iter, float tol, float *w_out, float *b_out, int *iters_out, float *stats_out,

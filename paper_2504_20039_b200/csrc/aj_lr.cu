@@ -3,12 +3,11 @@
 //   f(w, b) = 1/2 w.w + C * sum_i log(1 + exp(-s_i (x_i.w + b))),   s_i = +1 if labels[i] != 0 else -1
 //
 // (the intercept is not regularised; this is scikit-learn's convention, which the paper uses).
-// One evaluation of f and its gradient is ONE pass over X: a CTA stages a block of rows in shared
-// memory (cp.async, four buffers, two or three in flight), computes the rows' scores z = x.w + b from the
-// staged copy, turns them into residuals r_i = -C s_i sigma(-s_i z_i), and adds r_i x_i to its
-// own gradient accumulator from the same staged copy.  Every thread owns a fixed set of 16-byte
-// feature chunks in both phases and keeps their weights and gradient sums in registers.  CTAs write their partial gradients and partial losses to
-// separate slots, which a second kernel (gradient) and the host (loss, intercept) add in a fixed
+// One evaluation of f and its gradient is ONE pass over X: a group of warps loads a row into
+// registers (the next one is in flight meanwhile), computes its score z = x.w + b, turns it into the
+// residual r = -C s sigma(-s z), and adds r x to its gradient sums from the same registers.  CTAs
+// write their partial gradients and partial losses to separate slots, which a second kernel
+// (gradient) and the host (loss, intercept) add in a fixed
 // order, so an evaluation does not depend on scheduling.  The minimiser is found by L-BFGS on the
 // host in fp64 (two-loop recursion, Armijo backtracking); only w travels down and the gradient up.
 #include "../../include/aj_verify.h"
@@ -27,38 +26,25 @@ namespace {
 
 constexpr int LR_THREADS = 512;
 constexpr int LR_WARPS = LR_THREADS / 32;
-constexpr int LR_NBUF = 4;     // shared-memory buffers of one row block each
-constexpr int LR_RB_MAX = 8;   // rows per block at most (score accumulators per thread)
-constexpr int LR_MAXC = 4;     // 16-byte feature chunks a thread owns at most: rows of up to 32 KB
-constexpr int LR_SMEM_BUDGET = 220 * 1024;
+constexpr int LR_CPL_MAX = 6;  // 16-byte chunks of a row a lane owns at most
 
-__device__ inline void cp_async_16(void *smem_dst, const void *gmem_src) {
-    const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gmem_src) : "memory");
-}
-__device__ inline void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N> __device__ inline void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
-
-// the features of one 16-byte chunk of a staged row as floats
+// the features of one 16-byte chunk of a row as floats
 template <bool BF16> struct Chunk;
 template <> struct Chunk<true> {
     static constexpr int ELEMS = 8;
-    static __device__ inline void load(const char *p, float (&x)[8]) {
-        const uint4 v = *reinterpret_cast<const uint4 *>(p);
-        const __nv_bfloat162 *h = reinterpret_cast<const __nv_bfloat162 *>(&v);
+    static __device__ inline void unpack(const uint4 &v, float (&x)[8]) {
+        const uint32_t u[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-        for (int i = 0; i < 4; i++) {
-            const float2 f = __bfloat1622float2(h[i]);
-            x[2 * i] = f.x;
-            x[2 * i + 1] = f.y;
+        for (int i = 0; i < 4; i++) {  // a bf16 is the upper half of an fp32
+            x[2 * i] = __uint_as_float(u[i] << 16);
+            x[2 * i + 1] = __uint_as_float(u[i] & 0xffff0000u);
         }
     }
 };
 template <> struct Chunk<false> {
     static constexpr int ELEMS = 4;
-    static __device__ inline void load(const char *p, float (&x)[8]) {
-        const float4 v = *reinterpret_cast<const float4 *>(p);
-        x[0] = v.x, x[1] = v.y, x[2] = v.z, x[3] = v.w;
+    static __device__ inline void unpack(const uint4 &v, float (&x)[8]) {
+        x[0] = __uint_as_float(v.x), x[1] = __uint_as_float(v.y), x[2] = __uint_as_float(v.z), x[3] = __uint_as_float(v.w);
         x[4] = x[5] = x[6] = x[7] = 0.0f;
     }
 };
@@ -67,7 +53,7 @@ struct LrArgs {
     const char *X;           // [n, F], rows of row_bytes bytes
     const uint8_t *labels;   // [n]
     long long n;
-    int F, rb;               // features; rows per block
+    int F;
     size_t row_bytes;
     const float *w;          // [F]
     float b, C;
@@ -76,141 +62,134 @@ struct LrArgs {
     double *partial_gb;      // [grid]
 };
 
-// Thread t owns the chunks t, t + LR_THREADS, ... of every row: their weights and its share of the
-// CTA's gradient stay in registers for the whole launch; shared memory holds only the staged rows.
-// MAXC: chunks a thread owns at most; RB: rows per block (a shorter last block takes the guarded path).
-template <bool BF16, int MAXC, int RB>
+// A group of G warps takes one row at a time: lane l of the group owns the 16-byte chunks l, l + 32 G, ...
+// (CPL of them at most) of every row the group takes, loads them straight from global memory into
+// registers one row ahead, and keeps its share of the gradient in registers for the whole launch.
+// The groups of a CTA run independently of one another; the warps of a group meet once per row at a
+// named barrier to add their partial scores.  The weights are read from shared memory.
+template <bool BF16, int CPL, int G>
 __global__ void __launch_bounds__(LR_THREADS, 1) lr_loss_grad_kernel(const LrArgs a) {
     extern __shared__ __align__(16) char lr_smem[];
     constexpr int EPC = Chunk<BF16>::ELEMS;
-    constexpr int rb = RB;
+    constexpr int GROUPS = LR_WARPS / G;
+    constexpr int GL = 32 * G;  // lanes of a group
     const int F = a.F, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int chunks = F / EPC;
-    const int row_bytes = (int)a.row_bytes;           // at most 32 KB
-    const int stage_bytes = rb * row_bytes;
-    float *z_part = reinterpret_cast<float *>(lr_smem);         // [2][LR_WARPS][LR_RB_MAX], alternating between blocks
-    char *x_s = reinterpret_cast<char *>(z_part + 2 * LR_WARPS * LR_RB_MAX);  // [LR_NBUF][rb rows]
-
-    float wv[MAXC][8], g[MAXC][8];
-#pragma unroll
-    for (int k = 0; k < MAXC; k++) {
-        const int c = tid + k * LR_THREADS;
-#pragma unroll
-        for (int i = 0; i < 8; i++) {
-            wv[k][i] = (c < chunks && i < EPC) ? a.w[(size_t)c * EPC + i] : 0.0f;
-            g[k][i] = 0.0f;
-        }
+    // weights as two arrays of float4 (first and second half of every chunk): conflict-free 16-byte reads
+    float4 *w_lo = reinterpret_cast<float4 *>(lr_smem);
+    float4 *w_hi = w_lo + chunks;                                              // bf16 only
+    float *zbuf = reinterpret_cast<float *>(lr_smem + (size_t)F * 4);          // [GROUPS][2][G] partial scores
+    double *red = reinterpret_cast<double *>(zbuf + 2 * LR_WARPS);             // [2][GROUPS] losses, intercept gradients
+    for (int c = tid; c < chunks; c += LR_THREADS) {
+        const float4 *src = reinterpret_cast<const float4 *>(a.w + (size_t)c * EPC);
+        w_lo[c] = src[0];
+        if (BF16) w_hi[c] = src[1];
     }
-    const long long nblk = (a.n + rb - 1) / rb;
-    auto issue = [&](long long blk, int buf) {
-        if (blk < nblk) {
-            const long long row0 = blk * rb;
-            const int bytes = (int)(a.n - row0 < rb ? a.n - row0 : rb) * row_bytes;
-            const char *src = a.X + (size_t)row0 * a.row_bytes;
-            char *dst = x_s + buf * stage_bytes;
-            for (int off = tid * 16; off < bytes; off += LR_THREADS * 16) cp_async_16(dst + off, src + off);
+    __syncthreads();
+
+    const int group = warp / G, wg = warp % G, gl = wg * 32 + lane;
+    const long long ngroups = (long long)gridDim.x * GROUPS;
+    float g[CPL][8];
+#pragma unroll
+    for (int j = 0; j < CPL; j++)
+#pragma unroll
+        for (int i = 0; i < 8; i++) g[j][i] = 0.0f;
+    uint4 xc[CPL], xn[CPL];
+    auto load_row = [&](long long row, uint4 (&x)[CPL]) {
+        const uint4 *src = reinterpret_cast<const uint4 *>(a.X + (size_t)row * a.row_bytes);
+#pragma unroll
+        for (int j = 0; j < CPL; j++) {
+            const int c = j * GL + gl;
+            x[j] = (row < a.n && c < chunks) ? __ldcs(src + c) : make_uint4(0u, 0u, 0u, 0u);
         }
-        cp_async_commit();  // an empty group keeps the count of pending groups uniform
     };
-    for (int i = 0; i < LR_NBUF - 1; i++) issue((long long)blockIdx.x + (long long)i * gridDim.x, i);
+    long long row = (long long)blockIdx.x * GROUPS + group;
+    load_row(row, xc);
+    double loss = 0.0, gb = 0.0;  // lane 0 of the group's first warp
+    for (int it = 0; row < a.n; row += ngroups, ++it) {
+        load_row(row + ngroups, xn);  // in flight while this row is worked on
 
-    double loss = 0.0, gb = 0.0;  // lane 0 of warp 0 only
-    long long it = 0;
-    for (long long blk = blockIdx.x; blk < nblk; blk += gridDim.x, ++it) {
-        cp_async_wait<LR_NBUF - 2>();
-        __syncthreads();  // the block's rows are visible to every thread, and every thread is done with the block before
-        issue(blk + (long long)(LR_NBUF - 1) * gridDim.x, (int)((it + LR_NBUF - 1) % LR_NBUF));  // refills that block's buffer
-        const char *xb = x_s + (int)(it % LR_NBUF) * stage_bytes;
-        const long long row0 = blk * rb;
-        const int rows = (int)(a.n - row0 < rb ? a.n - row0 : rb);
-        const bool full = rows == rb;  // all blocks but possibly the last
-
-        // scores: every thread adds its chunks' share of every row's dot product
-        float zp[RB];
+        float zp = 0.0f;
 #pragma unroll
-        for (int r = 0; r < RB; r++) zp[r] = 0.0f;
-#pragma unroll
-        for (int k = 0; k < MAXC; k++) {
-            const int c = tid + k * LR_THREADS;
+        for (int j = 0; j < CPL; j++) {
+            const int c = j * GL + gl;
             if (c < chunks) {
-                const char *xc = xb + c * 16;
-#pragma unroll
-                for (int r = 0; r < RB; r++) {
-                    if (full || r < rows) {
-                        float x[8];
-                        Chunk<BF16>::load(xc + r * row_bytes, x);
-#pragma unroll
-                        for (int i = 0; i < EPC; i++) zp[r] = fmaf(x[i], wv[k][i], zp[r]);
-                    }
+                float x[8];
+                Chunk<BF16>::unpack(xc[j], x);
+                const float4 lo = w_lo[c];
+                zp = fmaf(x[0], lo.x, zp), zp = fmaf(x[1], lo.y, zp), zp = fmaf(x[2], lo.z, zp), zp = fmaf(x[3], lo.w, zp);
+                if (BF16) {
+                    const float4 hi = w_hi[c];
+                    zp = fmaf(x[4], hi.x, zp), zp = fmaf(x[5], hi.y, zp), zp = fmaf(x[6], hi.z, zp), zp = fmaf(x[7], hi.w, zp);
                 }
             }
         }
 #pragma unroll
-        for (int r = 0; r < RB; r++) {
+        for (int off = 16; off > 0; off >>= 1) zp += __shfl_xor_sync(0xffffffffu, zp, off);
+        float z = zp;
+        if (G > 1) {  // add the G warps' partial scores: a fixed tree, the same in every warp
+            float *slot = zbuf + (group * 2 + (it & 1)) * G;
+            if (lane == 0) slot[wg] = zp;
+            asm volatile("bar.sync %0, %1;" ::"r"(1 + group), "r"(GL) : "memory");
+            float v = lane < G ? slot[lane] : 0.0f;
 #pragma unroll
-            for (int off = 16; off > 0; off >>= 1) zp[r] += __shfl_xor_sync(0xffffffffu, zp[r], off);
-            if (lane == 0) z_part[((int)(it & 1) * LR_WARPS + warp) * LR_RB_MAX + r] = zp[r];
+            for (int off = G / 2; off > 0; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+            z = __shfl_sync(0xffffffffu, v, 0);
+        }
+        z += a.b;
+        const float s = a.labels[row] ? 1.0f : -1.0f;
+        const float t = s * z;
+        const float e = expf(-fabsf(t));
+        const float softplus = log1pf(e) + fmaxf(-t, 0.0f);                  // log(1 + exp(-t))
+        const float sig = t >= 0.0f ? e / (1.0f + e) : 1.0f / (1.0f + e);    // sigma(-t)
+        const float res = -a.C * s * sig;
+        if (gl == 0) {
+            loss += softplus;
+            gb += res;
+        }
+#pragma unroll
+        for (int j = 0; j < CPL; j++) {
+            const int c = j * GL + gl;
+            if (c < chunks) {
+                float x[8];
+                Chunk<BF16>::unpack(xc[j], x);
+#pragma unroll
+                for (int i = 0; i < EPC; i++) g[j][i] = fmaf(res, x[i], g[j][i]);
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < CPL; j++) xc[j] = xn[j];
+    }
+
+    // the groups' gradients are added in shared memory, one group after the other (the weights are done with)
+    __syncthreads();
+    float *acc = reinterpret_cast<float *>(lr_smem);
+    for (int sel = 0; sel < GROUPS; sel++) {
+        if (group == sel) {
+#pragma unroll
+            for (int j = 0; j < CPL; j++) {
+                const int c = j * GL + gl;
+                if (c < chunks) {
+#pragma unroll
+                    for (int i = 0; i < EPC; i++) acc[c * EPC + i] = (sel == 0 ? 0.0f : acc[c * EPC + i]) + g[j][i];
+                }
+            }
+            if (gl == 0) {
+                red[sel] = loss;
+                red[GROUPS + sel] = gb;
+            }
         }
         __syncthreads();
-        // every warp finishes the rows itself (lane r: row r), so that none waits for another
-        float softplus = 0.0f, res = 0.0f;
-        if (lane < rows) {
-            float z = a.b;
-#pragma unroll
-            for (int k = 0; k < LR_WARPS; k++) z += z_part[((int)(it & 1) * LR_WARPS + k) * LR_RB_MAX + lane];  // fixed order
-            const float s = a.labels[row0 + lane] ? 1.0f : -1.0f;
-            const float t = s * z;
-            const float e = expf(-fabsf(t));
-            softplus = log1pf(e) + fmaxf(-t, 0.0f);                            // log(1 + exp(-t))
-            const float sig = t >= 0.0f ? e / (1.0f + e) : 1.0f / (1.0f + e);  // sigma(-t)
-            res = -a.C * s * sig;
-        }
-        if (warp == 0) {  // the sums are kept by one warp; lanes without a row contribute zeros
-            double l = softplus, gg = res;
-            for (int off = 16; off > 0; off >>= 1) {
-                l += __shfl_xor_sync(0xffffffffu, l, off);
-                gg += __shfl_xor_sync(0xffffffffu, gg, off);
-            }
-            if (lane == 0) {
-                loss += l;
-                gb += gg;
-            }
-        }
-        float rr_row[RB];
-#pragma unroll
-        for (int r = 0; r < RB; r++) rr_row[r] = __shfl_sync(0xffffffffu, res, r);
-
-        // gradient: the same chunks, the same staged rows
-#pragma unroll
-        for (int k = 0; k < MAXC; k++) {
-            const int c = tid + k * LR_THREADS;
-            if (c < chunks) {
-                const char *xc = xb + c * 16;
-#pragma unroll
-                for (int r = 0; r < RB; r++) {
-                    if (full || r < rows) {
-                        float x[8];
-                        Chunk<BF16>::load(xc + r * row_bytes, x);
-                        const float rr = rr_row[r];
-#pragma unroll
-                        for (int i = 0; i < EPC; i++) g[k][i] = fmaf(rr, x[i], g[k][i]);
-                    }
-                }
-            }
-        }
     }
-    cp_async_wait<0>();
-#pragma unroll
-    for (int k = 0; k < MAXC; k++) {
-        const int c = tid + k * LR_THREADS;
-        if (c < chunks) {
-#pragma unroll
-            for (int i = 0; i < EPC; i++) a.partial_g[(size_t)blockIdx.x * F + (size_t)c * EPC + i] = g[k][i];
-        }
-    }
+    for (int f = tid; f < F; f += LR_THREADS) a.partial_g[(size_t)blockIdx.x * F + f] = acc[f];
     if (tid == 0) {
-        a.partial_loss[blockIdx.x] = loss;
-        a.partial_gb[blockIdx.x] = gb;
+        double l = 0.0, gg = 0.0;
+        for (int k = 0; k < GROUPS; k++) {
+            l += red[k];
+            gg += red[GROUPS + k];
+        }
+        a.partial_loss[blockIdx.x] = l;
+        a.partial_gb[blockIdx.x] = gg;
     }
 }
 
@@ -251,12 +230,14 @@ extern "C" aj_status aj_lr_fit(int device, const void *X, const uint8_t *labels,
     const size_t esz = dtype == AJ_BF16 ? 2 : 4;
     const size_t row_bytes = (size_t)F * esz;
     if (row_bytes % 16 != 0 || (reinterpret_cast<uintptr_t>(X) & 15) != 0) return AJ_ERR_UNSUPPORTED;
-    const size_t fixed = 2 * LR_WARPS * LR_RB_MAX * sizeof(float);
-    if (row_bytes > (size_t)LR_MAXC * LR_THREADS * 16) return AJ_ERR_UNSUPPORTED;  // a thread owns at most LR_MAXC chunks of a row
-    if (fixed + LR_NBUF * row_bytes > (size_t)LR_SMEM_BUDGET) return AJ_ERR_UNSUPPORTED;  // a row must fit four times
-    int rb = (int)((LR_SMEM_BUDGET - fixed) / (LR_NBUF * row_bytes));
-    if (rb > LR_RB_MAX) rb = LR_RB_MAX;
-    const size_t smem = fixed + (size_t)LR_NBUF * rb * row_bytes;
+    // warps per row: the fewest (1, 2, 4, 8 or 16) with at most LR_CPL_MAX chunks per lane
+    const int chunks = (int)(row_bytes / 16);
+    int G = 1;
+    while (G < LR_WARPS && (chunks + 32 * G - 1) / (32 * G) > LR_CPL_MAX) G *= 2;
+    const int cpl = (chunks + 32 * G - 1) / (32 * G);
+    if (cpl > LR_CPL_MAX) return AJ_ERR_UNSUPPORTED;  // rows wider than 48 KB
+    const int groups = LR_WARPS / G;
+    const size_t smem = (size_t)F * 4 + 2 * LR_WARPS * sizeof(float) + 2 * LR_WARPS * sizeof(double);
 
     int prev = 0;
     if (cudaGetDevice(&prev) != cudaSuccess || cudaSetDevice(device) != cudaSuccess) return AJ_ERR_CUDA;
@@ -270,33 +251,32 @@ extern "C" aj_status aj_lr_fit(int device, const void *X, const uint8_t *labels,
         return AJ_ERR_CUDA;
     if (cc_major != 10) return AJ_ERR_NOT_SM100;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    const int maxc = (int)((row_bytes / 16 + LR_THREADS - 1) / LR_THREADS);  // 1 .. LR_MAXC
     using Kernel = void (*)(const LrArgs);
-    auto pick_rb = [&](auto bf, auto mc) -> Kernel {
+    auto pick_g = [&](auto bf, auto cp) -> Kernel {
         constexpr bool B = decltype(bf)::value;
-        constexpr int M = decltype(mc)::value;
-        switch (rb) {
-            case 1: return lr_loss_grad_kernel<B, M, 1>;
-            case 2: return lr_loss_grad_kernel<B, M, 2>;
-            case 3: return lr_loss_grad_kernel<B, M, 3>;
-            case 4: return lr_loss_grad_kernel<B, M, 4>;
-            case 5: return lr_loss_grad_kernel<B, M, 5>;
-            case 6: return lr_loss_grad_kernel<B, M, 6>;
-            case 7: return lr_loss_grad_kernel<B, M, 7>;
-            default: return lr_loss_grad_kernel<B, M, 8>;
+        constexpr int P = decltype(cp)::value;
+        switch (G) {
+            case 1: return lr_loss_grad_kernel<B, P, 1>;
+            case 2: return lr_loss_grad_kernel<B, P, 2>;
+            case 4: return lr_loss_grad_kernel<B, P, 4>;
+            case 8: return lr_loss_grad_kernel<B, P, 8>;
+            default: return lr_loss_grad_kernel<B, P, 16>;
         }
     };
-    auto pick_mc = [&](auto bf) -> Kernel {
-        switch (maxc) {
-            case 1: return pick_rb(bf, std::integral_constant<int, 1>{});
-            case 2: return pick_rb(bf, std::integral_constant<int, 2>{});
-            default: return pick_rb(bf, std::integral_constant<int, LR_MAXC>{});
+    auto pick_cpl = [&](auto bf) -> Kernel {
+        switch (cpl) {
+            case 1: return pick_g(bf, std::integral_constant<int, 1>{});
+            case 2: return pick_g(bf, std::integral_constant<int, 2>{});
+            case 3: return pick_g(bf, std::integral_constant<int, 3>{});
+            case 4: return pick_g(bf, std::integral_constant<int, 4>{});
+            case 5: return pick_g(bf, std::integral_constant<int, 5>{});
+            default: return pick_g(bf, std::integral_constant<int, 6>{});
         }
     };
-    Kernel kernel = dtype == AJ_BF16 ? pick_mc(std::true_type{}) : pick_mc(std::false_type{});
+    Kernel kernel = dtype == AJ_BF16 ? pick_cpl(std::true_type{}) : pick_cpl(std::false_type{});
     if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return AJ_ERR_CUDA;
-    const long long nblk = (n + rb - 1) / rb;
-    const int grid = (int)(nblk < num_sms ? nblk : num_sms);
+    const long long want = (n + groups - 1) / groups;  // CTAs that would have a row for every group
+    const int grid = (int)(want < num_sms ? want : num_sms);
 
     Workspace ws;
     if (cudaMalloc(&ws.w_dev, F * sizeof(float)) != cudaSuccess || cudaMalloc(&ws.g_dev, F * sizeof(float)) != cudaSuccess ||
@@ -328,7 +308,6 @@ extern "C" aj_status aj_lr_fit(int device, const void *X, const uint8_t *labels,
         a.labels = labels;
         a.n = n;
         a.F = F;
-        a.rb = rb;
         a.row_bytes = row_bytes;
         a.w = ws.w_dev;
         a.b = (float)v[F];

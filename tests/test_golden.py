@@ -25,3 +25,21 @@ def test_oracle_reproduces_golden(name):
     gp = np.array([[np.nan if x is None else x for x in row] for row in got["judge_p"]])
     wp = np.array([[np.nan if x is None else x for x in row] for row in want["judge_p"]])
     np.testing.assert_allclose(gp, wp, rtol=0, atol=1e-10, equal_nan=True)
+
+
+@pytest.mark.parametrize("name", sorted(make_golden.VARIANTS))
+def test_oracle_reproduces_golden_variants(name):
+    """Sampled target tokens (Appendix A) and a draft tree (Section 3.3, "Generality")."""
+    with open(os.path.join(HERE, "golden", f"{name}.json")) as f:
+        want = json.load(f)
+    got = make_golden.compute_variant(**make_golden.VARIANTS[name])
+    assert set(got) == set(want)
+    for key in got:
+        if key in ("top1", "noise"):
+            np.testing.assert_allclose(np.array(got[key]), np.array(want[key]), rtol=0, atol=1e-10)
+        elif key == "judge_p":
+            gp = np.array([[np.nan if x is None else x for x in row] for row in got[key]])
+            wp = np.array([[np.nan if x is None else x for x in row] for row in want[key]])
+            np.testing.assert_allclose(gp, wp, rtol=0, atol=1e-10, equal_nan=True)
+        else:
+            assert got[key] == want[key], key

@@ -201,19 +201,32 @@ __global__ void lr_reduce_kernel(const float *__restrict__ partial_g, int parts,
     g[f] = s;
 }
 
+// One device allocation and one pinned host allocation per fit, carved into the pieces below.
 struct Workspace {
+    char *dev = nullptr, *host = nullptr;
+    size_t head_bytes = 0;         // partial losses, w and the gradient: the part mirrored on the host
+    double *partial_ld = nullptr;  // device [2 * grid]: losses, then intercept gradients
     float *w_dev = nullptr, *g_dev = nullptr, *partial_g = nullptr;
-    double *partial_ld = nullptr;  // [2 * grid]: losses, then intercept gradients
-    float *w_host = nullptr, *g_host = nullptr;
     double *ld_host = nullptr;
+    float *w_host = nullptr, *g_host = nullptr;
+    bool alloc(int F, int grid) {
+        const size_t ld = (2 * (size_t)grid * sizeof(double) + 255) & ~(size_t)255;  // every piece starts on a 256-byte boundary
+        const size_t vec = ((size_t)F * sizeof(float) + 255) & ~(size_t)255;
+        if (cudaMalloc(&dev, ld + 2 * vec + (size_t)grid * F * sizeof(float)) != cudaSuccess) return false;
+        if (cudaMallocHost(&host, ld + 2 * vec) != cudaSuccess) return false;
+        head_bytes = ld + 2 * vec;
+        partial_ld = reinterpret_cast<double *>(dev);
+        w_dev = reinterpret_cast<float *>(dev + ld);
+        g_dev = reinterpret_cast<float *>(reinterpret_cast<char *>(w_dev) + vec);
+        partial_g = reinterpret_cast<float *>(reinterpret_cast<char *>(g_dev) + vec);
+        ld_host = reinterpret_cast<double *>(host);
+        w_host = reinterpret_cast<float *>(host + ld);
+        g_host = reinterpret_cast<float *>(reinterpret_cast<char *>(w_host) + vec);
+        return true;
+    }
     ~Workspace() {
-        cudaFree(w_dev);
-        cudaFree(g_dev);
-        cudaFree(partial_g);
-        cudaFree(partial_ld);
-        cudaFreeHost(w_host);
-        cudaFreeHost(g_host);
-        cudaFreeHost(ld_host);
+        cudaFree(dev);
+        cudaFreeHost(host);
     }
 };
 
@@ -279,11 +292,7 @@ extern "C" aj_status aj_lr_fit(int device, const void *X, const uint8_t *labels,
     const int grid = (int)(want < num_sms ? want : num_sms);
 
     Workspace ws;
-    if (cudaMalloc(&ws.w_dev, F * sizeof(float)) != cudaSuccess || cudaMalloc(&ws.g_dev, F * sizeof(float)) != cudaSuccess ||
-        cudaMalloc(&ws.partial_g, (size_t)grid * F * sizeof(float)) != cudaSuccess ||
-        cudaMalloc(&ws.partial_ld, 2 * (size_t)grid * sizeof(double)) != cudaSuccess ||
-        cudaMallocHost(&ws.w_host, F * sizeof(float)) != cudaSuccess || cudaMallocHost(&ws.g_host, F * sizeof(float)) != cudaSuccess ||
-        cudaMallocHost(&ws.ld_host, 2 * (size_t)grid * sizeof(double)) != cudaSuccess) {
+    if (!ws.alloc(F, grid)) {
         cudaGetLastError();
         return AJ_ERR_CUDA;
     }
@@ -321,8 +330,8 @@ extern "C" aj_status aj_lr_fit(int device, const void *X, const uint8_t *labels,
         cudaEventRecord(ev1, stream);
         lr_reduce_kernel<<<(F + 255) / 256, 256, 0, stream>>>(ws.partial_g, grid, F, ws.g_dev);
         cuda_ok = cuda_ok && cudaGetLastError() == cudaSuccess;
-        cuda_ok = cuda_ok && cudaMemcpyAsync(ws.g_host, ws.g_dev, F * sizeof(float), cudaMemcpyDeviceToHost, stream) == cudaSuccess;
-        cuda_ok = cuda_ok && cudaMemcpyAsync(ws.ld_host, ws.partial_ld, 2 * (size_t)grid * sizeof(double), cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+        // one copy brings back the partial losses and the gradient (and, between them, w as it was sent)
+        cuda_ok = cuda_ok && cudaMemcpyAsync(ws.host, ws.dev, ws.head_bytes, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
         cuda_ok = cuda_ok && cudaStreamSynchronize(stream) == cudaSuccess;
         if (!cuda_ok) return 0.0;
         float ms = 0.0f;

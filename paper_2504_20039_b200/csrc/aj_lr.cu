@@ -105,9 +105,11 @@ __global__ void __launch_bounds__(LR_THREADS, 1) lr_loss_grad_kernel(const LrArg
     };
     long long row = (long long)blockIdx.x * GROUPS + group;
     load_row(row, xc);
+    unsigned label = row < a.n ? a.labels[row] : 0u, label_next = 0u;  // fetched a row ahead, like the features
     double loss = 0.0, gb = 0.0;  // lane 0 of the group's first warp
     for (int it = 0; row < a.n; row += ngroups, ++it) {
         load_row(row + ngroups, xn);  // in flight while this row is worked on
+        label_next = row + ngroups < a.n ? a.labels[row + ngroups] : 0u;
 
         float zp = 0.0f;
 #pragma unroll
@@ -137,15 +139,19 @@ __global__ void __launch_bounds__(LR_THREADS, 1) lr_loss_grad_kernel(const LrArg
             z = __shfl_sync(0xffffffffu, v, 0);
         }
         z += a.b;
-        const float s = a.labels[row] ? 1.0f : -1.0f;
+        const float s = label ? 1.0f : -1.0f;
         const float t = s * z;
-        const float e = expf(-fabsf(t));
-        const float softplus = log1pf(e) + fmaxf(-t, 0.0f);                  // log(1 + exp(-t))
-        const float sig = t >= 0.0f ? e / (1.0f + e) : 1.0f / (1.0f + e);    // sigma(-t)
+        // sigma(-t) = 1 / (1 + exp(t)) from the hardware exponential and reciprocal (about 1e-6 relative; the
+        // same bits in every warp of the group); exp(t) = inf gives 0, exp(t) = 0 gives 1
+        const float sig = __fdividef(1.0f, 1.0f + __expf(t));
         const float res = -a.C * s * sig;
-        if (gl == 0) {
-            loss += softplus;
-            gb += res;
+        if (wg == 0) {  // the loss is kept by the group's first warp only: log(1 + exp(-t)), accurately
+            const float e = expf(-fabsf(t));
+            const float softplus = log1pf(e) + fmaxf(-t, 0.0f);
+            if (lane == 0) {
+                loss += softplus;
+                gb += res;
+            }
         }
 #pragma unroll
         for (int j = 0; j < CPL; j++) {
@@ -159,6 +165,7 @@ __global__ void __launch_bounds__(LR_THREADS, 1) lr_loss_grad_kernel(const LrArg
         }
 #pragma unroll
         for (int j = 0; j < CPL; j++) xc[j] = xn[j];
+        label = label_next;
     }
 
     // the groups' gradients are added in shared memory, one group after the other (the weights are done with)

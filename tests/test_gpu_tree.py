@@ -196,3 +196,38 @@ def test_tree_entry_point_refuses_what_it_does_not_define():
         assert call(h) == aj.AJ_ERR_UNSUPPORTED
     finally:
         h.destroy()
+
+
+def test_tree_cycle_on_a_vocabulary_parallel_handle():
+    """A group of one rank: the tree entry point publishes to and gathers from its own exchange buffer and
+    returns what the unsharded handle returns."""
+    import torch
+
+    import paper_2504_20039_b200 as aj
+
+    orc = _orc()
+    B, N, V = 3, 12, 2048
+    cfg = gen.Config("tree_sharded", B=B, K=N, d=128, d_draft=64, V=V, sigma_W=0.2, sigma_w=0.05, seed=95)
+    W = gen.make_W(cfg)
+    ht, hd = gen.make_hidden(cfg)
+    w = gen.make_judge(cfg)
+    rng = np.random.default_rng(8)
+    y = np.stack([[orc.argmax(r)[0] for r in orc.logits(ht[b], W, gen.BF16)] for b in range(B)])
+    parent = np.stack([make_tree(rng, N, "random") for _ in range(B)])
+    tok = plant(rng, y, parent, V, 0.7)
+    dev = DeviceCase(cfg, W, ht, hd, w)
+    buf = torch.zeros(aj.shard_exchange_bytes(B, N, 1) // 8, dtype=torch.int64, device="cuda")
+    sharded = aj.Handle(0, B, N, cfg.d, cfg.d_draft, V, gen.BF16, aj.AJ_W_VD, 0, shard=(0, 1, 0, V, [buf]))
+    try:
+        want = run_tree(dev, tok, parent, 0.5)
+        check_tree(orc, orc.verify_tree(ht, hd, W, tok, parent, w, cfg.judge_b, 0.5, gen.BF16), want, tok, parent, 0.5)
+        plain = dev.handle
+        dev.handle = sharded
+        for _ in range(2):  # two cycles: both slot parities
+            got = run_tree(dev, tok, parent, 0.5)
+            for k in want:
+                np.testing.assert_array_equal(got[k], want[k])
+        dev.handle = plain
+    finally:
+        sharded.destroy()
+        dev.close()

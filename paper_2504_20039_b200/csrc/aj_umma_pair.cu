@@ -45,11 +45,12 @@ constexpr int BN = 256;       // rows of h per accumulator (half of them staged 
 constexpr int BK = 64;        // bf16 elements per k-block = 128 bytes = one swizzle span
 constexpr int UMMA_K = 16;
 // Warp 0 loads, warp 1 issues the MMAs, the rest drain the accumulators: one warp per TMEM lane quadrant,
-// or two (which take alternate chunks of columns) where the epilogue also generates the noise and, with
-// two accumulators per tile, is not hidden under the next tile's MMAs.  (Measured on one GPU against four
-// warps, sampled mode: 3 % and 4 % faster with two accumulators at 2080 x 8192 and 264 x 4096, 3 % slower
-// with one at 2112 and 528 rows x 4096.)
-__host__ __device__ constexpr int epilogue_warps(int epi, bool dual) { return epi == EPI_SAMPLE && dual ? 8 : 4; }
+// or two (which take alternate groups of column chunks) where the epilogue does more than the argmax (the
+// noise, or the count of the top-K rule) and, with two accumulators per tile, is not hidden under the next
+// tile's MMAs.  Measured on one GPU against four warps: sampled mode 3 % and 4 % faster with two
+// accumulators at 2080 x 8192 and 264 x 4096, but 3 % slower with one at 2112 and 528 rows x 4096; top-K
+// rule 8 % and 4 % faster at the same two shapes; the plain argmax unchanged at both (3 % faster at 392 rows).
+__host__ __device__ constexpr int epilogue_warps(int epi, bool dual) { return epi != EPI_PLAIN && dual ? 8 : 4; }
 __host__ __device__ constexpr int num_threads(int epi, bool dual) { return 64 + 32 * epilogue_warps(epi, dual); }
 constexpr int A_BYTES = BV_CTA * BK * 2;   // 16 KB: this CTA's 128 rows of W, one k-block
 constexpr int RING_BYTES = 224 * 1024;     // shared memory given to the stage ring (the SM has 227 KB per CTA)
@@ -432,7 +433,8 @@ cudaError_t launch_umma_pair(const GemmArgs &a, const UmmaPlan &p, cudaStream_t 
     const int stream_w = (sc.n_n == 1) ? 1 : 0;  // W is read by one pair only: do not keep it in L2
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)p.grid);  // 2 CTAs per pair
-    cfg.blockDim = dim3(num_threads(a.noise.temperature > 0.0f ? EPI_SAMPLE : EPI_PLAIN, sc.dual != 0));
+    const int epi = a.noise.temperature > 0.0f ? EPI_SAMPLE : a.rank.thr ? EPI_COUNT : EPI_PLAIN;
+    cfg.blockDim = dim3(num_threads(epi, sc.dual != 0));
     cfg.dynamicSmemBytes = SMEM_BYTES;
     cfg.stream = stream;
     cudaLaunchAttribute attr[2];

@@ -218,8 +218,8 @@ CSRC = os.path.join(ROOT, "paper_2504_20039_b200", "csrc")
 NCU_TRAFFIC = {
     # (workload, kernel configuration): (bytes per launch, kernel source files, sha1 of those files)
     ("c2_8b_b1_k16", "umma_vm_128x32"): (1.0547e9, ["aj_umma_vm.cu"], "e8fb306d3308"),        # profiles/umma_vm_128x32_c2_8b_b1_k16.md
-    ("c3_8b_b64_k32", "umma_pair_256x256"): (1.0909e9, ["aj_umma_pair.cu"], "0bcefaf197da"),  # profiles/umma_pair_256x256_c3_8b_b64_k32.md
-    ("c4_70b_b32_k64", "umma_pair_256x256"): (3.1709e9, ["aj_umma_pair.cu"], "0bcefaf197da"),  # profiles/umma_pair_256x256_c4_70b_b32_k64.md
+    ("c3_8b_b64_k32", "umma_pair_256x256"): (1.0809e9, ["aj_umma_pair.cu"], "82740e3d26df"),  # profiles/umma_pair_256x256_c3_8b_b64_k32.md
+    ("c4_70b_b32_k64", "umma_pair_256x256"): (3.1834e9, ["aj_umma_pair.cu"], "82740e3d26df"),  # profiles/umma_pair_256x256_c4_70b_b32_k64.md
 }
 
 

@@ -147,7 +147,10 @@ class GpuWorkload:
             if rule and rule.get("top_k"):
                 h.set_top_k(rule["top_k"])
             if rule and rule.get("temperature"):
-                h.set_sampling(rule["temperature"], seed=20250420, step=0)
+                from paper_2504_20039_b200 import dist as ajd_
+
+                rk = int(os.environ.get("RANK", "0"))
+                h.set_sampling(rule["temperature"], seed=ajd_.sampling_seed(20250420, rk, "vocab" if group is not None else "batch"), step=0)
         for ex in self.exchanges:
             ex.ready()
         # draft tokens planted against the device's own greedy tokens (a benchmark input, never an oracle input)

@@ -31,6 +31,15 @@ def rank_config(cfg, rank: int):
     return cfg if rank == 0 else replace(cfg, seed=cfg.seed + 7919 * rank)
 
 
+def sampling_seed(seed: int, rank: int, sharding: str = "batch") -> int:
+    """The seed rank `rank` gives aj_set_sampling.  Ranks that verify different sequences (batch sharding) must
+    draw different noise, and every handle numbers its rows from zero, so each gets its own seed; the ranks of
+    a vocabulary-parallel group verify the same rows and must all use the same one."""
+    if sharding == "vocab":
+        return seed & (2**64 - 1)
+    return (seed + 0x9E3779B97F4A7C15 * rank) & (2**64 - 1)
+
+
 def job_positions(cfg, world: int) -> int:
     """Draft positions the whole job verifies per step: every rank's B*K."""
     return cfg.B * cfg.K * world

@@ -26,6 +26,8 @@ def _worker(rank, world, port, out):
         slowest = g.max_over_ranks(10.0 + rank)          # rank r "took" 10 + r ms
         total = g.sum_over_ranks(float(cfg.B * cfg.K))    # positions verified by the whole job
         handles = g.all_gather_bytes(bytes([rank]) * 64)  # stand-ins for 64-byte IPC handles
+        seeds = g.all_gather_bytes(ajd.sampling_seed(77, rank).to_bytes(8, "little"))
+        assert len({bytes(s) for s in seeds}) == world and ajd.sampling_seed(77, rank, "vocab") == 77
         out.put((rank, cfg.seed, float(ht.astype("float64").sum()), slowest, total, [h[0] for h in handles], len(handles[0])))
     finally:
         g.close()

@@ -29,7 +29,8 @@ CASES = [
     ("ragged_rows_bf16", 1003, 64, gen.BF16, 1e-2),       # n is not a multiple of the row block
     ("many_rows_bf16", 20011, 256, gen.BF16, 1e-3),
     ("judge_width_bf16", 3000, 6144, gen.BF16, 1e-4),     # d_draft + d of the 1B / 8B pair, the paper's C
-    ("few_rows", 5, 8, gen.BF16, 1.0),                    # fewer rows than one block
+    ("few_rows", 5, 8, gen.BF16, 1.0),                    # fewer rows than there are warp groups
+    ("f32_two_warps_per_row", 600, 1024, gen.F32, 1e-2),
 ]
 
 
@@ -104,3 +105,19 @@ def test_fit_refuses_bad_arguments():
     wide = torch.zeros((4, 32768), dtype=torch.bfloat16, device="cuda")
     assert aj.lr_fit(0, wide, y, 4, 32768, aj.AJ_BF16, 1.0, torch.zeros(32768, device="cuda"), check=False)[0] == aj.AJ_ERR_UNSUPPORTED
     assert aj.lr_fit(0, X, y, 8, 16, aj.AJ_BF16, 1.0, w, check=False)[0] == aj.AJ_OK
+
+
+def test_widest_rows_reach_a_stationary_point():
+    """Rows of 48 KB (all 16 warps of a CTA on one row): too wide for the oracle's Newton steps, so the result is
+    certified instead: the objective is strongly convex (modulus 1 in w), hence |w - w*| <= |gradient| at w,
+    and the oracle evaluates that gradient in fp64."""
+    from oracle import aj_lr_oracle as lro
+
+    n, F, C = 300, 24576, 1e-3
+    X, y = gen.make_labelled_features(n, F, gen.BF16, seed=37)
+    w, b, iters, evals, gnorm = _fit(X, y, gen.BF16, C)
+    Xf = gen.to_f64(X, gen.BF16)
+    _, gw, gb = lro.objective(Xf, y, C, w, b)
+    assert np.linalg.norm(gw) <= 1e-4 and abs(gb) <= 1e-5, (np.linalg.norm(gw), gb, iters, evals, gnorm)
+    p = lro.predict_proba(Xf, w, b)
+    assert p[y == 1].mean() > p[y == 0].mean()

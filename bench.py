@@ -2,7 +2,7 @@
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2|c3|c4|sweep] [--impl reference]
 
-A step is one whole cycle (clear keys, LM-head projection + argmax, judge + prefix scan) over one
+A step is one whole cycle (LM-head projection + argmax, then judge + prefix scan: two launches) over one
 batch of seeded synthetic inputs shaped like the paper's Llama-3.x pairs.  The headline workload is
 the batch-1 8B-shaped configuration (B=1, K=16, d=4096, V=128256, bf16), the setting the paper's own
 measurements use (batch size 1); the batched 8B- and 70B-shaped configurations are reported under

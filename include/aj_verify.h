@@ -54,17 +54,20 @@ typedef enum {
 } aj_w_layout;
 
 enum {
-    AJ_FLAG_FORCE_SIMT = 1u,  /* use the plain fp32-accumulate CUDA-core kernel for the projection */
     AJ_FLAG_TIME_KERNELS = 2u, /* record CUDA events around the projection kernel (see aj_last_gemm_ms) */
-    AJ_FLAG_ROW_TILES = 4u,    /* tensor-core path with 128-row tiles of h on the UMMA M axis (the earlier
-                                  tiling, kept for comparison) instead of vocabulary-major tiles */
-    AJ_FLAG_ONE_SM = 8u,       /* keep batches of more than 128 rows on the one-SM vocabulary-major kernel
-                                  instead of the two-SM (CTA pair) kernel; for comparison */
     AJ_FLAG_NO_EXTRA_ROW = 16u /* the caller does not encode the last draft token (Section 3.2, design choice 1,
                                   second way): h_target and h_draft are [B, K, ...], target_tok and top1_val are
                                   [B, K]; a mismatch at the last position is rejected without the classifier
                                   (judge_p there is NaN); when all K tokens pass, next_tok is -1 (there is no
                                   row to predict a further token from) */
+};
+
+/* Comparison switches: they select a slower kernel for the same result and exist for tests and
+ * measurements.  Not part of the interface a caller should build on. */
+enum {
+    AJ_FLAG_FORCE_SIMT = 1u, /* the plain fp32-accumulate CUDA-core kernel for the projection */
+    AJ_FLAG_ONE_SM = 8u      /* keep batches of more than 128 rows on the one-SM kernel instead of the
+                                two-SM (CTA pair) kernel */
 };
 
 /*
@@ -118,8 +121,8 @@ aj_status aj_verify(aj_handle h, const void *h_target, const void *h_draft, cons
  * are ignored; judge_p, if given, receives the draft token's rank (as a float, 0 = the target's own
  * token) at every mismatching position and NaN elsewhere.  A cycle then launches three kernels (the
  * draft tokens' own logits, the projection with the count fused into its epilogue, the scan).
- * top_k = 0 switches back to the classifier.  Not available on vocabulary-parallel handles, with
- * AJ_FLAG_ROW_TILES or with AJ_FLAG_NO_EXTRA_ROW (AJ_ERR_UNSUPPORTED).  Errors: AJ_ERR_INVALID_ARG.
+ * top_k = 0 switches back to the classifier.  Not available on vocabulary-parallel handles or with
+ * AJ_FLAG_NO_EXTRA_ROW (AJ_ERR_UNSUPPORTED).  Errors: AJ_ERR_INVALID_ARG.
  */
 aj_status aj_set_top_k(aj_handle h, int top_k);
 
@@ -141,7 +144,7 @@ aj_status aj_set_top_k(aj_handle h, int top_k);
  * given the same temperature, seed and step; replicas that verify different sequences should be given
  * different seeds, since every handle numbers its rows from zero).  temperature = 0 switches back to greedy
  * verification.  Errors: AJ_ERR_INVALID_ARG (NULL handle, negative or non-finite temperature),
- * AJ_ERR_UNSUPPORTED (together with the top-K rule, or with AJ_FLAG_ROW_TILES).
+ * AJ_ERR_UNSUPPORTED (together with the top-K rule).
  */
 aj_status aj_set_sampling(aj_handle h, float temperature, uint64_t seed, uint64_t step);
 
@@ -228,7 +231,7 @@ aj_status aj_last_gemm_ms(aj_handle h, float *ms);
 aj_status aj_gemm_ms_stats(aj_handle h, float *mean_ms, float *min_ms, int *count);
 
 /* Number of kernels of this library that the most recent aj_verify / aj_verify_host call launched
- * (the projection kernel and the judge kernel; the memset that clears the keys is not counted). */
+ * (the projection kernel and the judge kernel; one more under the top-K rule). */
 int aj_last_launch_count(aj_handle h);
 
 /*
@@ -239,14 +242,16 @@ int aj_last_launch_count(aj_handle h);
  *   [4] rows of h_target each SM of a pair stages per 64-column block and accumulator
  *   [5] groups the row tiles are walked in (each group against the whole vocabulary, so that a
  *       group's rows of h_target stay in L2)    [6],[7] group g holds out[6] + (g < out[7]) row tiles
- *   [8] 1 if each tile uses two accumulators that share the staged block of W_lm (a tile then holds up
- *       to 512 rows; chosen for 257..448 rows, and from 1024 rows on when d >= 8192), else 0 (tiles of
- *       at most 256 rows on one accumulator, double-buffered)      [9] depth of the shared-memory ring
+ *   [8] 1 if each tile uses two accumulators, each with its own issuing warp, that share the staged
+ *       block of W_lm (a tile then holds up to 512 rows; chosen for every batch of more than 256 rows),
+ *       else 0 (one tile of at most 256 rows on one accumulator, double-buffered)
+ *   [9] depth of the shared-memory ring
  * Errors: AJ_ERR_INVALID_ARG.
  */
 aj_status aj_pair_schedule(int M, int d, int V, int32_t out[10]);
 
-/* Name of the projection kernel configuration the most recent call used, e.g. "umma_128x256". */
+/* Name of the projection kernel configuration the most recent call used: "umma_vm_128x32" ... "umma_vm_128x256"
+ * (one SM per tile: 128 vocabulary entries x up to that many rows), "umma_pair_256x256" (CTA pairs) or "simt". */
 const char *aj_last_gemm_path(aj_handle h);
 
 /*
@@ -316,7 +321,7 @@ aj_status aj_shard_range(int V, int world, int rank, int *v_begin, int *v_count)
 /*
  * aj_create for one GPU of a vocabulary-parallel group.  V is the WHOLE vocabulary (token ids in
  * the outputs are global); this GPU's W_lm argument in later calls is its shard, v_count rows
- * (layout AJ_W_VD: [v_count, d]; AJ_W_DV: [d, v_count]).  AJ_FLAG_ROW_TILES is not available here.
+ * (layout AJ_W_VD: [v_count, d]; AJ_W_DV: [d, v_count]).
  * Errors: as aj_create, and AJ_ERR_INVALID_ARG for a bad rank, range or buffer.
  */
 aj_status aj_create_sharded(aj_handle *out, int device, int max_B, int max_K, int d, int d_draft, int V,

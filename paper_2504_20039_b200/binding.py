@@ -15,7 +15,7 @@ LIB_PATH = os.path.join(_HERE, "libaj_verify.so")
 AJ_OK, AJ_ERR_INVALID_ARG, AJ_ERR_UNSUPPORTED, AJ_ERR_WORKSPACE, AJ_ERR_CUDA, AJ_ERR_TIMEOUT, AJ_ERR_NOT_SM100 = range(7)
 AJ_BF16, AJ_F32 = 0, 1
 AJ_W_VD, AJ_W_DV = 0, 1
-AJ_FLAG_FORCE_SIMT, AJ_FLAG_TIME_KERNELS, AJ_FLAG_ROW_TILES, AJ_FLAG_ONE_SM, AJ_FLAG_NO_EXTRA_ROW = 1, 2, 4, 8, 16
+AJ_FLAG_FORCE_SIMT, AJ_FLAG_TIME_KERNELS, AJ_FLAG_ONE_SM, AJ_FLAG_NO_EXTRA_ROW = 1, 2, 8, 16
 
 EXPORTS = (
     "aj_create", "aj_verify", "aj_verify_host", "aj_last_status", "aj_last_gemm_ms", "aj_gemm_ms_stats", "aj_last_launch_count",

@@ -7,7 +7,7 @@ import subprocess
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libaj_verify.so")
-SOURCES = ["aj_api.cu", "aj_umma_vm.cu", "aj_umma_pair.cu", "aj_umma.cu", "aj_simt.cu", "aj_judge.cu", "aj_rank.cu", "aj_static.cu", "aj_lr.cu"]
+SOURCES = ["aj_api.cu", "aj_umma_vm.cu", "aj_umma_pair.cu", "aj_simt.cu", "aj_judge.cu", "aj_rank.cu", "aj_static.cu", "aj_lr.cu"]
 HEADERS = ["aj_internal.cuh", "aj_ptx.cuh", os.path.join("..", "..", "include", "aj_verify.h")]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

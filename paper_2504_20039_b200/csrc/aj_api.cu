@@ -126,8 +126,6 @@ const CUtensorMap *get_tmap(aj_handle h, const void *ptr, long long rows, int bo
     return &victim->map;
 }
 
-int choose_bn(int M) { return M <= 128 ? 128 : 256; }
-
 // Batches with more rows than this run on the two-SM kernel; smaller ones are bound by the W_lm
 // stream from HBM and keep the one-SM kernel, which has more loads in flight per SM.
 constexpr int PAIR_MIN_ROWS = 128;
@@ -188,7 +186,7 @@ aj_status aj_create(aj_handle *out, int device, int max_B, int max_K, int d, int
     if (device < 0 || max_B < 1 || max_K < 1 || max_K > 1024 || d < 1 || d_draft < 0 || V < 1) return AJ_ERR_INVALID_ARG;
     if (dtype != AJ_BF16 && dtype != AJ_F32) return AJ_ERR_INVALID_ARG;
     if (layout != AJ_W_VD && layout != AJ_W_DV) return AJ_ERR_INVALID_ARG;
-    if (flags & ~(AJ_FLAG_FORCE_SIMT | AJ_FLAG_TIME_KERNELS | AJ_FLAG_ROW_TILES | AJ_FLAG_ONE_SM | AJ_FLAG_NO_EXTRA_ROW))
+    if (flags & ~(AJ_FLAG_FORCE_SIMT | AJ_FLAG_TIME_KERNELS | AJ_FLAG_ONE_SM | AJ_FLAG_NO_EXTRA_ROW))
         return AJ_ERR_INVALID_ARG;
     if ((long long)max_B * (max_K + 1) > (1ll << 24)) return AJ_ERR_INVALID_ARG;
     if (dtype == AJ_BF16 && (d % 8 != 0 || d_draft % 8 != 0)) return AJ_ERR_UNSUPPORTED;
@@ -219,7 +217,7 @@ aj_status aj_create(aj_handle *out, int device, int max_B, int max_K, int d, int
     // tensor-core path: bf16, d a multiple of 64; W_lm as [V, d], or as [d, V] with a row pitch that
     // TMA accepts (a multiple of 16 bytes) on the vocabulary-major kernels
     h->umma_ok = dtype == AJ_BF16 && d % 64 == 0 && !(flags & AJ_FLAG_FORCE_SIMT) &&
-                 (layout == AJ_W_VD || (V % 8 == 0 && !(flags & AJ_FLAG_ROW_TILES)));
+                 (layout == AJ_W_VD || V % 8 == 0);
 
     const size_t max_M = (size_t)max_B * (max_K + 1);
     const size_t esz = elem_size(dtype);
@@ -242,7 +240,7 @@ aj_status aj_create(aj_handle *out, int device, int max_B, int max_K, int d, int
         ok = cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &fn, 12000, cudaEnableDefault, &qres) == cudaSuccess &&
              qres == cudaDriverEntryPointSuccess && fn != nullptr;
         h->encode = reinterpret_cast<EncodeTiledFn>(fn);
-        if (ok) ok = umma_prepare() == cudaSuccess && umma_vm_prepare() == cudaSuccess;
+        if (ok) ok = umma_vm_prepare() == cudaSuccess;
         if (ok) h->pair_ok = umma_pair_prepare(h->num_sms) == cudaSuccess && umma_pair_max_pairs() > 0;
         if (!h->pair_ok) cudaGetLastError();  // no room for CTA pairs: the one-SM kernel serves every batch
     }
@@ -350,7 +348,7 @@ static aj_status enqueue_project(aj_handle h, const void *h_target, const void *
     const int slot = (int)(h->n_timed % EVENT_RING);
     if (time_it && cudaEventRecord(h->ev0[slot], stream) != cudaSuccess) return AJ_ERR_CUDA;
     cudaError_t e;
-    if (h->umma_ok && h->pair_ok && M > PAIR_MIN_ROWS && !(h->flags & (AJ_FLAG_ROW_TILES | AJ_FLAG_ONE_SM))) {
+    if (h->umma_ok && h->pair_ok && M > PAIR_MIN_ROWS && !(h->flags & AJ_FLAG_ONE_SM)) {
         // tensor-bound regime: two-SM tiles of 256 vocabulary entries x up to 256 rows
         UmmaPlan p;
         p.bn = 256;
@@ -365,7 +363,7 @@ static aj_status enqueue_project(aj_handle h, const void *h_target, const void *
         p.grid = 2 * (int)(tiles < pairs ? tiles : pairs);
         e = launch_umma_pair(g, p, stream);
         h->last_path = "umma_pair_256x256";
-    } else if (h->umma_ok && !(h->flags & AJ_FLAG_ROW_TILES)) {
+    } else if (h->umma_ok) {
         UmmaPlan p;
         p.bn = vm_choose_bn(M);
         const CUtensorMap *tw = get_tmap(h, W_lm, V, h->layout == AJ_W_DV ? -1 : 128);
@@ -377,19 +375,6 @@ static aj_status enqueue_project(aj_handle h, const void *h_target, const void *
         p.grid = (int)(tiles < h->num_sms ? tiles : h->num_sms);
         e = launch_umma_vm(g, p, stream);
         h->last_path = umma_vm_path_name(p.bn);
-    } else if (h->umma_ok) {
-        UmmaPlan p;
-        p.bn = choose_bn(M);
-        const CUtensorMap *th = get_tmap(h, h_target, M, 128);
-        const CUtensorMap *tw = get_tmap(h, W_lm, V, p.bn);
-        if (!th || !tw) return AJ_ERR_CUDA;
-        p.tmap_h = *th;
-        p.tmap_w = *tw;
-        const int n_m = (M + 127) / 128, n_v = (V + p.bn - 1) / p.bn;
-        const long long tiles = (long long)n_m * n_v;
-        p.grid = (int)(tiles < h->num_sms ? tiles : h->num_sms);
-        e = launch_umma_gemm_argmax(g, p, stream);
-        h->last_path = umma_path_name(p.bn);
     } else {
         e = launch_simt_gemm_argmax(g, h->num_sms, stream);
         h->last_path = "simt";
@@ -597,7 +582,6 @@ aj_status aj_create_sharded(aj_handle *out, int device, int max_B, int max_K, in
     if (v_begin < 0 || v_count < 1 || (long long)v_begin + v_count > V) return AJ_ERR_INVALID_ARG;
     for (int r = 0; r < world; r++)
         if (!exchange[r] || (reinterpret_cast<uintptr_t>(exchange[r]) & 255)) return AJ_ERR_INVALID_ARG;
-    if (flags & AJ_FLAG_ROW_TILES) return AJ_ERR_UNSUPPORTED;
     aj_handle h = nullptr;
     if (layout == AJ_W_DV && v_count % 8 != 0) flags |= AJ_FLAG_FORCE_SIMT;  // the shard's row pitch is not TMA-loadable
     aj_status st = aj_create(&h, device, max_B, max_K, d, d_draft, V, dtype, layout, flags);
@@ -707,8 +691,8 @@ aj_status aj_ipc_close(void *device_ptr) {
 
 aj_status aj_set_top_k(aj_handle h, int top_k) {
     if (!h || top_k < 0) return AJ_ERR_INVALID_ARG;
-    // the count is kept per GPU and the row-tile kernel does not produce it
-    if (top_k > 0 && (h->world || (h->flags & (AJ_FLAG_ROW_TILES | AJ_FLAG_NO_EXTRA_ROW)))) return AJ_ERR_UNSUPPORTED;
+    // the count is kept per GPU
+    if (top_k > 0 && (h->world || (h->flags & AJ_FLAG_NO_EXTRA_ROW))) return AJ_ERR_UNSUPPORTED;
     if (top_k > 0 && h->temperature > 0.0f) return AJ_ERR_UNSUPPORTED;  // the rule ranks the plain logits
     h->top_k = top_k;
     return AJ_OK;
@@ -716,8 +700,7 @@ aj_status aj_set_top_k(aj_handle h, int top_k) {
 
 aj_status aj_set_sampling(aj_handle h, float temperature, uint64_t seed, uint64_t step) {
     if (!h || !(temperature >= 0.0f) || !(temperature <= 3.0e38f)) return AJ_ERR_INVALID_ARG;
-    // the row-tile kernel's epilogue does not add the noise
-    if (temperature > 0.0f && (h->top_k > 0 || (h->flags & AJ_FLAG_ROW_TILES))) return AJ_ERR_UNSUPPORTED;
+    if (temperature > 0.0f && h->top_k > 0) return AJ_ERR_UNSUPPORTED;
     h->temperature = temperature;
     h->seed = seed;
     h->step = step;

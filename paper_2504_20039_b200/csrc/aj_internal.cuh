@@ -52,6 +52,13 @@ __device__ inline uint32_t warp_max_u32(uint32_t x) {
     asm volatile("redux.sync.max.u32 %0, %1, 0xffffffff;" : "=r"(r) : "r"(x));
     return r;
 }
+
+// Minimum of x over the 32 lanes of the warp.
+__device__ inline uint32_t warp_min_u32(uint32_t x) {
+    uint32_t r;
+    asm volatile("redux.sync.min.u32 %0, %1, 0xffffffff;" : "=r"(r) : "r"(x));
+    return r;
+}
 #endif
 
 // Device status word values (mirrors aj_status where they overlap).
@@ -261,19 +268,14 @@ enum : int { EPI_PLAIN = 0, EPI_COUNT = 1, EPI_SAMPLE = 2 };
 // CUDA-core projection + argmax (any dtype / layout).
 cudaError_t launch_simt_gemm_argmax(const GemmArgs &a, int num_sms, cudaStream_t stream);
 
-// tcgen05 projection + argmax (bf16, [V,d]).  `bn` is the vocabulary tile width (64, 128 or 256).
+// tcgen05 projection + argmax (bf16), vocabulary on the UMMA M axis, one SM per tile.
 struct UmmaPlan {
-    CUtensorMap tmap_h;  // rows of h, box 64 x 128, 128-byte swizzle
-    CUtensorMap tmap_w;  // rows of W, box 64 x bn
-    int bn;
+    CUtensorMap tmap_h;  // rows of h, 128-byte swizzle
+    CUtensorMap tmap_w;  // rows of W (or, for [d, V], 64 entries x 64 k-rows)
+    int bn;              // rows of h per tile
     int grid;
 };
-cudaError_t umma_prepare();  // opt-in shared memory attributes; call once per device
-cudaError_t launch_umma_gemm_argmax(const GemmArgs &a, const UmmaPlan &p, cudaStream_t stream);
-const char *umma_path_name(int bn);
-
-// tcgen05 projection + argmax with the vocabulary on the UMMA M axis (the default path).
-// Here tmap_w has a 64 x 128 box and tmap_h a 64 x bn box, bn = vm_choose_bn(M) rows of h per tile.
+// tmap_w has a 64 x 128 box and tmap_h a 64 x bn box, bn = vm_choose_bn(M) rows of h per tile.
 int vm_choose_bn(int M);
 cudaError_t umma_vm_prepare();
 cudaError_t launch_umma_vm(const GemmArgs &a, const UmmaPlan &p, cudaStream_t stream);

@@ -302,6 +302,12 @@ cudaError_t launch_judge_scan(const JudgeArgs &a, cudaStream_t stream) {
     cfg.gridDim = dim3((unsigned)a.B);
     cfg.blockDim = dim3(THREADS);
     cfg.dynamicSmemBytes = (size_t)(4 * a.K + 1) * sizeof(int) + (size_t)a.K * SEGS * sizeof(float);
+    if (cfg.dynamicSmemBytes > 48 * 1024) {
+        // only the largest window (K = 1024) needs more than the default limit, by four bytes
+        const cudaError_t e = cudaFuncSetAttribute(judge_scan_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                   (int)cfg.dynamicSmemBytes);
+        if (e != cudaSuccess) return e;
+    }
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;

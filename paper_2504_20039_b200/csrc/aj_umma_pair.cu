@@ -1,33 +1,50 @@
-// Tensor-core projection + running argmax for sm_100a on CTA pairs (two SMs per tile), the
-// tensor-bound regime (more than 128 rows of hidden states):
+// Tensor-core projection + running argmax for sm_100a on CTA pairs (two SMs per tile), for batches
+// of more than 128 rows of hidden states:
 //
 //   logit[v, m] = sum_k W[v, k] * h[m, k]        bf16 x bf16 -> fp32 in tensor memory, never stored
 //   keys[m]     = max over v of pack(logit[v, m], v)
 //
-// A tile is 256 vocabulary entries (UMMA M = 256, 128 per SM = the 128 TMEM lanes of each SM) by
-// up to 256 rows of hidden states (UMMA N, any multiple of 16).  The rows are cut into the fewest
-// tiles of at most 256 rows and spread over them evenly in units of 16 rows (2112 rows = 6 tiles of
-// 240 + 3 of 224), so no tensor work is spent on padding and all tiles take nearly the same time,
-// which keeps the pairs that share a block of W in step and that block in L2.  When h_target
-// outgrows L2 the row tiles are walked in groups, each group against the whole vocabulary.
+// A tile is 256 vocabulary entries (UMMA M = 256, 128 per SM = the 128 TMEM lanes of each SM) by a
+// block of rows of hidden states (UMMA N, any multiple of 16).  The rows are cut into the fewest
+// tiles and spread over them evenly in units of 16 rows, so no tensor work is spent on padding and
+// all tiles take nearly the same time, which keeps the pairs that share a block of W in step and
+// that block in L2.  When h_target outgrows L2 the row tiles are walked in groups, each group
+// against the whole vocabulary.
+//
+// Two forms (512 columns of tensor memory either way):
+//   narrow tiles (DUAL = false, batches of at most 256 rows): one accumulator of up to 256 columns in
+//     one of two buffers that alternate from tile to tile, so the epilogue of one tile runs under the
+//     MMAs of the next; one issuing thread;
+//   wide tiles (DUAL = true): up to 512 rows on TWO accumulators of up to 256 columns that share each
+//     staged block of W, each with its own issuing warp and its own pair of barriers.
+// Why two issuing warps: a tcgen05.mma holds the thread that issues it for about 100 cycles whatever
+// its N (measured: one thread issuing 128 x N x 16 MMAs back to back gets one through per 104 cycles
+// for every N <= 208; two warps issuing on two accumulators get one through per max(52, N/2) cycles,
+// the tensor pipe's own rate).  With one issuing thread a k-block of two accumulators costs 8 x 104
+// cycles plus the waits whatever the tensor work; with two, each accumulator's 4 MMAs per k-block are
+// issued in parallel and the tensor pipe is the limit from about 140 rows per accumulator on.  The
+// price of the wide form is that an accumulator has to be drained before its next tile can start
+// (about 7,000 cycles per tile between the last MMA of one tile and the first of the next, against
+// 55,000 cycles of MMAs at d = 4096); measured on one GPU it is the faster form for every batch of
+// more than 256 rows (520 rows: 466 vs 562 us, 2112 rows: 1.57 vs 1.75 ms, 2080 x 8192: 3.13 vs 3.52 ms).
 //
 // The two CTAs of a cluster sit on one SM pair; the even CTA (the leader) issues
-// tcgen05.mma.cta_group::2 for both.  Each CTA stages its own 128 rows of W and HALF of the tile's
-// rows of h, so a k-block costs at most 32 KB of L2 -> SM traffic per SM where the one-SM kernel
-// needs 48 KB for the same tensor work.  Nothing is multicast: every CTA fetches its own half-tiles
-// with ordinary tiled TMA loads, and the follower's loads report their bytes to the leader's barrier.
+// tcgen05.mma.cta_group::2 for both.  Each CTA stages its own 128 rows of W and HALF of each
+// accumulator's rows of h.  Nothing is multicast: every CTA fetches its own half-tiles with ordinary
+// tiled TMA loads, and the follower's loads report their bytes to the leader's barrier.
 //
-// Roles in each CTA (192 threads):
+// Roles in each CTA:
 //   warp 0      TMA producer (one thread): waits for its own stage to be free, then loads
-//               W[v0 + 128*rank .. +128, kb] and h[n0 + (N/2)*rank .. , kb] with 128-byte swizzle;
-//   warp 1      allocates tensor memory (both CTAs); in the leader one thread issues the MMAs and
-//               commits stage-release and accumulator-ready barriers to both CTAs at once;
-//   warps 2..5  epilogue: thread = one TMEM lane = one vocabulary entry.  32 columns (rows of h) at a
-//               time are compared with the best value each row has so far (read from its key); only
-//               a chunk in which some logit reaches that value is reduced (per column the warp
-//               maximum by redux.sync on the order-preserving image of the logit, the lowest lane
-//               attaining it by ballot) and merged into the row's packed key by a 64-bit atomic max.
-// Two accumulator buffers of 256 columns: the epilogue of one tile runs under the MMAs of the next.
+//               W[v0 + 128*rank .. +128, kb] and, per accumulator a, h[row0[a] + (N[a]/2)*rank .. , kb];
+//   warp 1, 2   warp 1 allocates tensor memory (both CTAs); in the leader one thread of each issues
+//               the MMAs of accumulator 0 / 1 (warp 2 only for wide tiles) and commits stage-release
+//               and accumulator-ready barriers to both CTAs at once;
+//   warps 3..   epilogue, one warp per TMEM lane quadrant and accumulator:
+//               thread = one TMEM lane = one vocabulary entry.  32 columns (rows of h) at a time are
+//               compared with the best value each row has so far (read from its key); only a chunk
+//               in which some logit reaches that value is reduced (per column the warp maximum by
+//               redux.sync on the order-preserving image of the logit, the lowest lane attaining it
+//               by ballot) and merged into the row's packed key by a 64-bit atomic max.
 // No split over k.  Every wait is bounded; a wait that runs out sets the status word, and both CTAs
 // still meet at the cluster barrier before tensor memory is freed.
 #include "aj_internal.cuh"
@@ -41,28 +58,28 @@ namespace {
 
 constexpr int BV = 256;       // vocabulary entries per tile (128 per CTA)
 constexpr int BV_CTA = 128;
-constexpr int BN = 256;       // rows of h per accumulator (half of them staged by each CTA)
+constexpr int BN = 256;       // columns of one tensor-memory buffer
 constexpr int BK = 64;        // bf16 elements per k-block = 128 bytes = one swizzle span
 constexpr int UMMA_K = 16;
-// Warp 0 loads, warp 1 issues the MMAs, the rest drain the accumulators: one warp per TMEM lane quadrant,
-// or two (which take alternate groups of column chunks) where the epilogue does more than the argmax (the
-// noise, or the count of the top-K rule) and, with two accumulators per tile, is not hidden under the next
-// tile's MMAs.  Measured on one GPU against four warps: sampled mode 3 % and 4 % faster with two
-// accumulators at 2080 x 8192 and 264 x 4096, but 3 % slower with one at 2112 and 528 rows x 4096; top-K
-// rule 8 % and 4 % faster at the same two shapes; the plain argmax unchanged at both (3 % faster at 392 rows).
-__host__ __device__ constexpr int epilogue_warps(int epi, bool dual) { return epi != EPI_PLAIN && dual ? 8 : 4; }
-__host__ __device__ constexpr int num_threads(int epi, bool dual) { return 64 + 32 * epilogue_warps(epi, dual); }
+// Warp 0 loads, warps 1 and 2 issue the MMAs of accumulator 0 and 1, the rest drain the accumulators:
+// one warp per TMEM lane quadrant and accumulator.
+__host__ __device__ constexpr int epilogue_warps(bool dual) { return dual ? 8 : 4; }  // four per accumulator
+__host__ __device__ constexpr int num_threads(bool dual) { return 96 + 32 * epilogue_warps(dual); }
+constexpr int FIRST_EPI_WARP = 3;
 constexpr int A_BYTES = BV_CTA * BK * 2;   // 16 KB: this CTA's 128 rows of W, one k-block
 constexpr int RING_BYTES = 224 * 1024;     // shared memory given to the stage ring (the SM has 227 KB per CTA)
 constexpr int MAX_STAGES = 8;
 constexpr int TMEM_COLS = 2 * BN;
-constexpr int BAR_BYTES = 8 * (2 * MAX_STAGES + 4) + 16;
+constexpr int BAR_BYTES = 8 * (2 * MAX_STAGES + 8) + 16;
 constexpr int SMEM_BYTES = RING_BYTES + BAR_BYTES + 1024;
 
 struct Tile {
     int v_tile;     // block of 256 vocabulary entries
     int row0[2];    // first row of h of each accumulator
-    int n_inst[2];  // rows of each accumulator = UMMA N, a multiple of 16 (the second is 0 in single mode)
+    int n_inst[2];  // rows of each accumulator = UMMA N, a multiple of 16 (the second is 0 for narrow tiles)
+    // (selected, not indexed: the struct stays in registers)
+    __device__ int first_row(int a) const { return a ? row0[1] : row0[0]; }
+    __device__ int rows(int a) const { return a ? n_inst[1] : n_inst[0]; }
 };
 
 // Tile t of the schedule.  Row tiles come in groups; a group is walked against every vocabulary
@@ -70,7 +87,7 @@ struct Tile {
 // neighbouring pairs at the same time, share a block of W.  Which row tile of the group a pair gets
 // rotates with the vocabulary block, so that pairs whose number is a multiple of the group size
 // apart do not always get the larger (or the smaller) row tiles and drift away from the pairs they
-// share W with.  In dual mode a row tile is split over the two accumulators.
+// share W with.  A wide tile's units of 16 rows are split over the two accumulators, the larger half first.
 __device__ inline Tile decode_tile(const PairSched &sc, int t) {
     int g = 0, start = 0, sz = sc.g_base + (0 < sc.g_rem ? 1 : 0);
     while (g + 1 < sc.n_groups && t >= start + sz * sc.n_v) {
@@ -93,11 +110,11 @@ __device__ inline Tile decode_tile(const PairSched &sc, int t) {
     return r;
 }
 
-// DUAL: every tile uses two accumulators that share the staged block of W.  WDV: W is stored [d, V].
-// EPI: EPI_COUNT also counts, per row, the entries that outrank the draft token (top-K rule);
-// EPI_SAMPLE adds Gumbel noise to the logits before the argmax.
+// DUAL: wide tiles (two accumulators, two issuing warps) instead of narrow ones.  WDV: W is stored
+// [d, V].  EPI: EPI_COUNT also counts, per row, the entries that outrank the draft token (top-K
+// rule); EPI_SAMPLE adds Gumbel noise to the logits before the argmax.
 template <bool DUAL, bool WDV, int EPI>
-__global__ void __launch_bounds__(num_threads(EPI, DUAL), 1)
+__global__ void __launch_bounds__(num_threads(DUAL), 1)
 umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_h,
                  int M, int V, int d, PairSched sc, int stream_w, int v_offset,
                  unsigned long long *__restrict__ keys, int *__restrict__ status, const Publish pub, const RankArgs rk,
@@ -110,9 +127,9 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
     const uint32_t bar_base = base + RING_BYTES;
     auto full_bar = [&](int s) { return bar_base + 8u * s; };                                  // used in the leader only
     auto empty_bar = [&](int s) { return bar_base + 8u * (MAX_STAGES + s); };
-    auto acc_full_bar = [&](int a) { return bar_base + 8u * (2 * MAX_STAGES + a); };
-    auto acc_empty_bar = [&](int a) { return bar_base + 8u * (2 * MAX_STAGES + 2 + a); };      // used in the leader only
-    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + RING_BYTES + 8 * (2 * MAX_STAGES + 4));
+    auto acc_full_bar = [&](int a) { return bar_base + 8u * (2 * MAX_STAGES + a); };           // a = 2 * buffer + accumulator
+    auto acc_empty_bar = [&](int a) { return bar_base + 8u * (2 * MAX_STAGES + 4 + a); };      // used in the leader only
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + RING_BYTES + 8 * (2 * MAX_STAGES + 8));
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5;  // warp-uniform
@@ -122,20 +139,20 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
     const int num_pairs = gridDim.x >> 1;
     const int num_kb = d / BK;
     const int num_tiles = sc.n_n * sc.n_v;
-    constexpr int n_acc = DUAL ? 2 : 1;
     const int stages = sc.stages;
     const uint32_t b_bytes = (uint32_t)sc.box_rows * BK * 2;       // one accumulator's rows of h staged by this CTA
+    constexpr int n_acc = DUAL ? 2 : 1;
     const uint32_t stage_bytes = A_BYTES + n_acc * b_bytes;         // a multiple of 1024
     const uint32_t stage_tx = 2u * stage_bytes;                     // bytes both CTAs load per stage
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < MAX_STAGES; s++) {
             mbar_init(full_bar(s), 1);   // the leader's producer; bytes arrive from both CTAs
-            mbar_init(empty_bar(s), 1);  // one commit from the leader's MMA thread
+            mbar_init(empty_bar(s), n_acc);  // one commit from each of the leader's issuing threads
         }
-        for (int a = 0; a < 2; a++) {
-            mbar_init(acc_full_bar(a), 1);
-            mbar_init(acc_empty_bar(a), 2 * epilogue_warps(EPI, DUAL));  // the epilogue warps of the two CTAs
+        for (int a = 0; a < 4; a++) {
+            mbar_init(acc_full_bar(a), 1);   // the accumulator's issuing thread
+            mbar_init(acc_empty_bar(a), 8);  // the four warps that drain it, in both CTAs
         }
         *abort_flag = 0;
         fence_barrier_init();
@@ -154,10 +171,10 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
         *abort_flag = 1;
         atomicCAS(status, DEV_OK, DEV_TIMEOUT);
     };
-    // Accumulator hand-over.  Single mode: the two 256-column buffers alternate from tile to tile
-    // (buffer it & 1, each with its own pair of barriers).  Dual mode: every tile uses both buffers
-    // as two accumulators that share the staged block of W, and one pair of barriers.
-    auto acc_slot = [&](int it) { return DUAL ? 0 : (it & 1); };
+    // Accumulator hand-over.  Narrow tiles: the two 256-column buffers alternate from tile to tile.
+    // Wide tiles: accumulator a in buffer a.  Every buffer has its own full / empty barriers.
+    auto acc_id = [&](int it, int a) { return DUAL ? a : (it & 1); };
+    auto acc_col = [&](int it, int a) { return (uint32_t)(acc_id(it, a) * BN); };
     auto acc_phase = [&](int it) { return (uint32_t)(DUAL ? it : (it >> 1)) & 1u; };
 
     if (warp == 0) {
@@ -197,30 +214,29 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
                 }
             }
         }
-    } else if (warp == 1) {
-        if (lane == 0 && rank == 0) {
-            // ------------------------------------------- MMA issuer (leader CTA only)
+    } else if (warp <= 2) {
+        if (lane == 0 && rank == 0 && warp <= n_acc) {
+            // --------------------- MMA issuer of accumulator a = warp - 1 (leader CTA only)
             // (rebuilding the descriptors per k-block measured slightly faster than stepping them
             // from stage to stage, which chains every k-block's issue to the previous one)
-            const unsigned long long acc_step = b_bytes >> 4;
+            const int a = warp - 1;
             constexpr unsigned long long a_step = WDV ? MN_KSTEP : 2ull;
+            constexpr uint32_t a_major = WDV ? IDESC_A_MN_MAJOR : 0u;
+            const uint32_t b_off = A_BYTES + (uint32_t)a * b_bytes;
             int s = 0;
             uint32_t ph = 0;
             bool ok = true;
             int it = 0;
             for (int t = pair; ok && t < num_tiles; t += num_pairs, ++it) {
                 const Tile tl = decode_tile(sc, t);
-                constexpr uint32_t a_major = WDV ? IDESC_A_MN_MAJOR : 0u;
-                const uint32_t idesc0 = instr_desc(BV, tl.n_inst[0]) | a_major;
-                const uint32_t idesc1 = instr_desc(BV, tl.n_inst[1]) | a_major;
-                const int slot = acc_slot(it);
-                if (!mbar_wait(acc_empty_bar(slot), acc_phase(it) ^ 1u, abort_flag)) {
+                const int n_inst = tl.rows(a);  // 0: this accumulator has no rows in this tile (one unit of 16); the barriers still turn
+                const uint32_t idesc = instr_desc(BV, n_inst) | a_major;
+                if (!mbar_wait(acc_empty_bar(acc_id(it, a)), acc_phase(it) ^ 1u, abort_flag)) {
                     give_up();
                     break;
                 }
                 tc_fence_after();
-                const uint32_t d_tmem0 = tmem_base + (uint32_t)(slot * BN);
-                const uint32_t d_tmem1 = tmem_base + (uint32_t)BN;  // dual mode only
+                const uint32_t d_tmem = tmem_base + acc_col(it, a);
                 for (int kb = 0; kb < num_kb; kb++) {
                     if (!mbar_wait(full_bar(s), ph, abort_flag)) {
                         give_up();
@@ -230,100 +246,103 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
                     tc_fence_after();
                     const uint32_t a_addr = base + s * stage_bytes;
                     const unsigned long long adesc = WDV ? smem_desc_sw128_mn(a_addr) : smem_desc_sw128(a_addr);
-                    const unsigned long long bdesc0 = smem_desc_sw128(a_addr + A_BYTES);
-#pragma unroll
-                    for (int k = 0; k < BK / UMMA_K; k++)
-                        umma_bf16_pair(d_tmem0, adesc + a_step * k, bdesc0 + 2ull * k, idesc0, (uint32_t)((kb | k) != 0));
-                    if (n_acc == 2) {
-                        const unsigned long long bdesc1 = bdesc0 + acc_step;
+                    const unsigned long long bdesc = smem_desc_sw128(a_addr + b_off);
+                    if (n_inst) {
 #pragma unroll
                         for (int k = 0; k < BK / UMMA_K; k++)
-                            umma_bf16_pair(d_tmem1, adesc + a_step * k, bdesc1 + 2ull * k, idesc1, (uint32_t)((kb | k) != 0));
+                            umma_bf16_pair(d_tmem, adesc + a_step * k, bdesc + 2ull * k, idesc, (uint32_t)((kb | k) != 0));
                     }
-                    umma_commit_pair(empty_bar(s));  // frees the stage in both CTAs
+                    umma_commit_pair(empty_bar(s));  // this accumulator is done with the stage, in both CTAs
                     if (++s == stages) {
                         s = 0;
                         ph ^= 1u;
                     }
                 }
-                if (ok) umma_commit_pair(acc_full_bar(slot));  // the accumulators in both CTAs are complete
+                if (ok) umma_commit_pair(acc_full_bar(acc_id(it, a)));  // the accumulator is complete in both CTAs
             }
         }
     } else {
         // -------------------------------------------------------------------- epilogue
         // A logit can only matter if it reaches the best value its row has so far.  Lane j reads
-        // that value for column 32c + j from the row's key before the tile's accumulators are
-        // ready (a stale value is only lower, never wrong).  A chunk of 32 columns is then checked
-        // with one comparison per element against the shuffled-in thresholds and one vote; only
-        // if some element qualifies does the chunk take the reduction path (warp maximum per
-        // column by redux.sync, lowest lane by ballot, 64-bit atomic max into the key).  After the
-        // first few vocabulary blocks nearly every chunk is skipped.
+        // the key of the row of column 32c + j before the accumulator is ready (a stale key is only
+        // lower, never wrong); its high half is that value as an ordered integer.  A chunk of 32
+        // columns is first tested against the LOWEST of its 32 thresholds (one redux.sync.min, and
+        // per lane the maximum of its 32 logits): nearly every chunk ends there.  Otherwise the
+        // elements are compared one by one with the shuffled-in thresholds, and only if some
+        // element qualifies does the chunk take the reduction path (warp maximum per column by
+        // redux.sync, lowest lane by ballot, 64-bit atomic max into the key).
         const int q = warp & 3;  // TMEM lane quadrant this warp may read
-        constexpr int SPLIT = epilogue_warps(EPI, DUAL) / 4;           // warps per quadrant
-        const int part = SPLIT == 1 ? 0 : (warp - 2) >> 2;        // which of them this one is
-        const float never = __int_as_float(0x7fc00000);  // NaN: no comparison with it is ever true
-        // Chunk g of a tile is columns 32 (g & 7) .. + 32 of accumulator g >> 3.  Its threshold for
-        // lane j is the best value the row of column 32 (g & 7) + j has so far, read from the key.
-        auto load_thr = [&](const Tile &tl, int g) {
-            const int a = g >> 3, col = (g & 7) * 32 + lane;
-            const int row = (a ? tl.row0[1] : tl.row0[0]) + col;
-            if (a >= n_acc || col >= (a ? tl.n_inst[1] : tl.n_inst[0]) || row >= M) return never;
-            const unsigned long long k = __ldcg(keys + row);
-            return k == 0ull ? -INFINITY : key_value(k);
+        const int a = DUAL ? (warp - FIRST_EPI_WARP) >> 2 : 0;              // the accumulator this warp drains
+        constexpr int CH = BN / 32;                                         // 32-column chunks per accumulator
+        constexpr uint32_t NO_ROW = 0xFFFFFFFFu;  // above every value: nothing qualifies
+        // Chunk c is columns 32 c .. + 32 of the accumulator.  Only the high half of the key is read,
+        // the best value as an ordered integer; 0 = the row has no key yet.
+        auto load_key = [&](const Tile &tl, int c) {
+            const int col = c * 32 + lane;
+            const int row = tl.first_row(a) + col;
+            if (col >= tl.rows(a) || row >= M) return NO_ROW;
+            return __ldcg(reinterpret_cast<const uint32_t *>(keys + row) + 1);
         };
-        // thresholds are fetched GRP chunks ahead of their use, an L2 round trip: four chunks, or one
-        // where the noise makes a chunk take that long by itself (and one copy of its code, not four,
-        // then stays within the instruction cache)
-        constexpr int GRP = EPI == EPI_SAMPLE ? 1 : 4;
+        // All of the accumulator's keys are fetched before it is ready, so no chunk waits for an L2
+        // round trip.  The chunk loop is kept rolled, one copy of its code stays in the instruction
+        // cache: the keys rotate through kk[0].
         int it = 0;
         for (int t = pair; t < num_tiles; t += num_pairs, ++it) {
             const Tile tl = decode_tile(sc, t);
-            const int slot = acc_slot(it);
-            float cur[GRP], nxt[GRP];
+            uint32_t kk[CH];
 #pragma unroll
-            for (int u = 0; u < GRP; u++) cur[u] = load_thr(tl, part * GRP + u);  // in flight while the accumulators are being computed
+            for (int i = 0; i < CH; i++) kk[i] = load_key(tl, i);
+            const int v_first = tl.v_tile * BV + (int)rank * BV_CTA + q * 32;  // vocabulary entry of lane 0
+            const bool v_ok = v_first + lane < V;                            // entries past V hold zero-filled junk
+            const uint32_t tbase = tmem_base + ((uint32_t)(q * 32) << 16);
             // the whole warp takes one decision, so the aligned TMEM loads below stay converged
-            if (!__all_sync(0xffffffffu, mbar_wait(acc_full_bar(slot), acc_phase(it), abort_flag))) {
+            if (!__all_sync(0xffffffffu, mbar_wait(acc_full_bar(acc_id(it, a)), acc_phase(it), abort_flag))) {
                 give_up();
                 break;
             }
             tc_fence_after();
-            const int v_first = tl.v_tile * BV + (int)rank * BV_CTA + q * 32;  // vocabulary entry of lane 0
-            const bool v_ok = v_first + lane < V;                            // entries past V hold zero-filled junk
-            const uint32_t tbase = tmem_base + ((uint32_t)(q * 32) << 16);
-            // the group loop is kept rolled: one copy of the code stays in the instruction cache
+            const int n_inst = tl.rows(a), row_a = tl.first_row(a);
 #pragma unroll 1
-            for (int g0 = part * GRP; g0 < 8 * n_acc; g0 += GRP * SPLIT) {
+            for (int c = 0; c * 32 < n_inst; c++) {
+                const uint32_t kthr = kk[0];
 #pragma unroll
-                for (int u = 0; u < GRP; u++) nxt[u] = (g0 + GRP * SPLIT < 8 * n_acc) ? load_thr(tl, g0 + GRP * SPLIT + u) : never;
+                for (int i = 0; i + 1 < CH; i++) kk[i] = kk[i + 1];
+                {
+                    float v[32];
+                    tmem_ld32(tbase + acc_col(it, a) + (uint32_t)(c * 32), v);
+                    if (EPI == EPI_COUNT) count_outranking(rk, v, v_first, v_ok, row_a + c * 32, n_inst - c * 32, M, lane);
+                    if (EPI == EPI_SAMPLE) add_gumbel_noise(nz, v, v_first + lane + v_offset, row_a + c * 32);
+                    // the lowest threshold of the chunk (a row without a key yet: everything qualifies)
+                    const uint32_t tmin = warp_min_u32(kthr);
+                    float vmax = v[0];
 #pragma unroll
-                for (int u = 0; u < GRP; u++) {
-                    const int g = g0 + u, a = g >> 3, c = g & 7;
-                    const int n_inst = a ? tl.n_inst[1] : tl.n_inst[0];
-                    if (c * 32 < n_inst) {  // warp-uniform
-                        const float thr = cur[u];
-                        float v[32];
-                        tmem_ld32(tbase + (uint32_t)((DUAL ? a : slot) * BN + c * 32), v);
-                        if (EPI == EPI_COUNT)
-                            count_outranking(rk, v, v_first, v_ok, (a ? tl.row0[1] : tl.row0[0]) + c * 32, n_inst - c * 32, M, lane);
-                        if (EPI == EPI_SAMPLE) add_gumbel_noise(nz, v, v_first + lane + v_offset, (a ? tl.row0[1] : tl.row0[0]) + c * 32);
+                    for (int j = 1; j < 32; j++) vmax = fmaxf(vmax, v[j]);
+                    if (__any_sync(0xffffffffu, v_ok && ordered_image(vmax) >= tmin)) {
+                        const float thr = kthr == NO_ROW ? __int_as_float(0x7fc00000)  // NaN: no comparison with it is ever true
+                                          : kthr == 0u  ? -INFINITY
+                                                        : key_value((unsigned long long)kthr << 32);
                         bool hit = false;
 #pragma unroll
                         for (int j = 0; j < 32; j++) hit |= v[j] >= __shfl_sync(0xffffffffu, thr, j);
                         if (__any_sync(0xffffffffu, hit && v_ok)) {
+                            // all 32 reductions are issued before any result is used, so that their
+                            // latencies overlap instead of adding up
+                            uint32_t x[32], m[32];
+#pragma unroll
+                            for (int j = 0; j < 32; j++) x[j] = v_ok ? ordered_image(v[j]) : 0u;
+#pragma unroll
+                            for (int j = 0; j < 32; j++) m[j] = warp_max_u32(x[j]);
                             uint32_t best_u = 0u;  // lane j: maximum of column 32c + j over this warp's 32 entries
                             int best_i = 0;
 #pragma unroll
                             for (int j = 0; j < 32; j++) {
-                                const uint32_t x = v_ok ? ordered_image(v[j]) : 0u;
-                                const uint32_t m = warp_max_u32(x);
-                                const uint32_t who = __ballot_sync(0xffffffffu, x == m);
+                                const uint32_t who = __ballot_sync(0xffffffffu, x[j] == m[j]);
                                 if (lane == j) {
-                                    best_u = m;
+                                    best_u = m[j];
                                     best_i = v_first + __ffs(who) - 1;  // the lowest entry that attains the maximum
                                 }
                             }
-                            const int row = (a ? tl.row0[1] : tl.row0[0]) + c * 32 + lane;
+                            const int row = row_a + c * 32 + lane;
                             if (c * 32 + lane < n_inst && row < M && best_u != 0u) {
                                 const unsigned long long key =
                                     ((unsigned long long)best_u << 32) | (uint32_t)(~(uint32_t)(best_i + v_offset));
@@ -332,13 +351,11 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
                         }
                     }
                 }
-#pragma unroll
-                for (int u = 0; u < GRP; u++) cur[u] = nxt[u];
             }
-            // the accumulators are drained: hand them back to the leader's MMA thread
+            // the accumulator is drained: hand it back to its issuing thread in the leader
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(map_to_cta(acc_empty_bar(slot), 0));
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(acc_empty_bar(acc_id(it, a)), 0));
         }
     }
 
@@ -378,7 +395,7 @@ cudaError_t umma_pair_prepare(int num_sms) {
     // how many CTA pairs can be resident at once (pairs need both SMs of a pair free)
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(num_sms & ~1));
-    cfg.blockDim = dim3(num_threads(EPI_SAMPLE, true));  // the largest block: residency is the same, one CTA per SM
+    cfg.blockDim = dim3(num_threads(true));  // the largest block: residency is the same, one CTA per SM
     cfg.dynamicSmemBytes = SMEM_BYTES;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -400,14 +417,9 @@ int umma_pair_max_pairs() { return g_max_pairs; }
 PairSched pair_schedule(int M, int V, int d) {
     PairSched sc;
     const int units = (M + 15) / 16;  // rows in units of 16 (the UMMA N granule)
-    // Two accumulators per tile (up to 512 rows share each staged block of W; 25 % less operand
-    // traffic, but the epilogue is no longer hidden under the next tile's MMAs) or one (at most 256
-    // rows, double-buffered)?  Measured on the same GPU: two win from 257 to about 450 rows, where
-    // they save a second pass over W (-10 % at 264 and 400 rows, +4 % at 512), and for deep
-    // contractions with many rows, where the exposed epilogue is a small share of a tile and the
-    // operand traffic weighs most (d = 8192: -1.5 % at 1056 rows, -6 % at 2080, -9 % at 4160; but
-    // +1.5 % at 528, and +3 ... +8 % for every batch at d = 4096).
-    sc.dual = (units > 16 && (units <= 28 || (d >= 8192 && units >= 64))) ? 1 : 0;
+    // Wide tiles (up to 512 rows on two accumulators with an issuing warp each) for every batch of more
+    // than 256 rows; up to 256 rows one narrow tile per vocabulary block, double-buffered.
+    sc.dual = units > 16 ? 1 : 0;
     const int cap = sc.dual ? 32 : 16;
     sc.n_n = (units + cap - 1) / cap;
     sc.u_base = units / sc.n_n;
@@ -419,7 +431,7 @@ PairSched pair_schedule(int M, int V, int d) {
     const int stage_bytes = A_BYTES + (sc.dual ? 2 : 1) * sc.box_rows * BK * 2;
     sc.stages = RING_BYTES / stage_bytes < MAX_STAGES ? RING_BYTES / stage_bytes : MAX_STAGES;
     // row tiles per group: keep a group's rows of h (tile rows x d x 2 bytes) within about 40 MB of L2
-    const long long tile_bytes = 256ll * d * 2;
+    const long long tile_bytes = (sc.dual ? 512ll : 256ll) * d * 2;
     int g_max = (int)((40ll << 20) / tile_bytes);
     if (g_max < 1) g_max = 1;
     sc.n_groups = (sc.n_n + g_max - 1) / g_max;
@@ -433,8 +445,7 @@ cudaError_t launch_umma_pair(const GemmArgs &a, const UmmaPlan &p, cudaStream_t 
     const int stream_w = (sc.n_n == 1) ? 1 : 0;  // W is read by one pair only: do not keep it in L2
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)p.grid);  // 2 CTAs per pair
-    const int epi = a.noise.temperature > 0.0f ? EPI_SAMPLE : a.rank.thr ? EPI_COUNT : EPI_PLAIN;
-    cfg.blockDim = dim3(num_threads(epi, sc.dual != 0));
+    cfg.blockDim = dim3(num_threads(sc.dual != 0));
     cfg.dynamicSmemBytes = SMEM_BYTES;
     cfg.stream = stream;
     cudaLaunchAttribute attr[2];

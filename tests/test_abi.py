@@ -80,7 +80,7 @@ def test_two_sm_schedule_covers_every_row_once(built):
         s = aj.pair_schedule(M, d, 128256)
         assert s["n_v"] == 501
         units = (M + 15) // 16
-        assert s["dual"] == (1 if (256 < M <= 448 or (d >= 8192 and M > 1008)) else 0)
+        assert s["dual"] == (1 if M > 256 else 0)              # wide tiles (two accumulators) above 256 rows
         cap = 32 if s["dual"] else 16                         # units per tile: two accumulators or one
         sizes = [s["u_base"] + (i < s["u_rem"]) for i in range(s["n_n"])]
         assert sum(sizes) == units and max(sizes) <= cap and min(sizes) >= (2 if s["dual"] else 1)
@@ -92,7 +92,7 @@ def test_two_sm_schedule_covers_every_row_once(built):
         assert 4 <= s["stages"] == min(8, (224 * 1024) // stage) and s["stages"] * stage <= 224 * 1024
         groups = [s["g_base"] + (g < s["g_rem"]) for g in range(s["n_groups"])]
         assert sum(groups) == s["n_n"] and min(groups) >= 1 and max(groups) - min(groups) <= 1
-        assert max(groups) * 256 * d * 2 <= 40 << 20 or max(groups) == 1
+        assert max(groups) * (512 if s["dual"] else 256) * d * 2 <= 40 << 20 or max(groups) == 1
     assert aj.pair_schedule(2112, 4096, 128256)["n_groups"] == 1
     assert aj.pair_schedule(2080, 8192, 128256)["n_groups"] == 1
     assert aj.pair_schedule(16640, 4096, 128256)["n_groups"] == 4

@@ -1,10 +1,10 @@
 """GPU parity at the full benchmark sizes, in the launch configuration the benchmark times.
 
-The CPU oracle verifies whole sequences sampled from the batch (all of them for the batch-1
-workload); their draft tokens are planted against the oracle's own greedy tokens.  The other
-sequences of the batch get draft tokens planted against the device's greedy tokens (never an
-oracle input) and are checked through properties that hold at any size.  Set AJ_FULL_ORACLE=1 to
-have the oracle verify every sequence.
+The CPU oracle verifies every sequence of the four named workloads; their draft tokens are planted
+against the oracle's own greedy tokens.  At the points of the throughput sweep it verifies whole
+sequences sampled from the batch; the other sequences there get draft tokens planted against the
+device's greedy tokens (never an oracle input) and are checked through properties that hold at any
+size.  Set AJ_FULL_ORACLE=1 to have the oracle verify every sequence of the sweep points too.
 """
 import os
 
@@ -79,21 +79,42 @@ def test_c2_8b_batch1_every_row():
     assert all(r.rows == 17 for r in reps)
 
 
-def test_c3_8b_batched_sampled_sequences():
-    reps = _run_workload(gen.C3, (gen.C3.tau,), 8, "umma_pair_256x256")
-    assert reps[0].seqs >= 8 and reps[0].seqs_exempt <= reps[0].seqs // 2
+def test_c3_8b_batched_every_sequence():
+    reps = _run_workload(gen.C3, (gen.C3.tau,), gen.C3.B, "umma_pair_256x256")
+    assert reps[0].seqs == gen.C3.B and reps[0].rows == gen.C3.M and reps[0].seqs_exempt <= reps[0].seqs // 2
 
 
-def test_c5_sweep_points_on_the_8b_shape():
-    # smallest, the HBM/tensor crossover, and the largest point of the sweep
-    for B, K, path in [(1, 8, "umma_vm_128x32"), (8, 32, "umma_pair_256x256"), (256, 8, "umma_pair_256x256"), (256, 64, "umma_pair_256x256")]:
-        reps = _run_workload(gen.sweep_config(B, K), (0.5,), 3, path)
-        assert reps[0].seqs >= min(B, 3)
+SWEEP_POINTS = [
+    # B, K, kernel, (wide tiles, row tiles) of the two-SM kernel: every kernel configuration the sweep reaches
+    (1, 8, "umma_vm_128x32", None),       # M = 9
+    (1, 32, "umma_vm_128x64", None),      # M = 33
+    (1, 64, "umma_vm_128x128", None),     # M = 65
+    (8, 8, "umma_vm_128x128", None),      # M = 72
+    (8, 16, "umma_pair_256x256", (0, 1)),   # M = 136: one narrow tile of 144 rows
+    (8, 32, "umma_pair_256x256", (1, 1)),   # M = 264: one wide tile (144 + 128 rows), the HBM / tensor crossover
+    (8, 64, "umma_pair_256x256", (1, 2)),   # M = 520: two wide tiles
+    (64, 8, "umma_pair_256x256", (1, 2)),   # M = 576
+    (256, 8, "umma_pair_256x256", (1, 5)),  # M = 2304
+    (256, 64, "umma_pair_256x256", (1, 33)),  # M = 16640: the largest point, row tiles walked in four groups
+]
 
 
-def test_c4_70b_sampled_sequences_tau_sweep():
-    reps = _run_workload(gen.C4, gen.C4_TAUS, 4, "umma_pair_256x256")
-    assert len(reps) == 9 and all(r.seqs >= 4 for r in reps)
+@pytest.mark.parametrize("point", SWEEP_POINTS, ids=[f"b{p[0]}_k{p[1]}" for p in SWEEP_POINTS])
+def test_c5_sweep_points_on_the_8b_shape(point):
+    import paper_2504_20039_b200 as aj
+
+    B, K, path, tiles = point
+    cfg = gen.sweep_config(B, K)
+    if tiles is not None:
+        s = aj.pair_schedule(cfg.M, cfg.d, cfg.V)
+        assert (s["dual"], s["n_n"]) == tiles
+    reps = _run_workload(cfg, (0.5,), 3, path)
+    assert reps[0].seqs >= min(B, 3)
+
+
+def test_c4_70b_every_sequence_tau_sweep():
+    reps = _run_workload(gen.C4, gen.C4_TAUS, gen.C4.B, "umma_pair_256x256")
+    assert len(reps) == 9 and all(r.seqs == gen.C4.B and r.rows == gen.C4.M for r in reps)
 
 
 def test_c2_with_the_lm_head_stored_d_by_v_gives_the_same_bits():

@@ -103,12 +103,41 @@ SHAPES = [
 
 
 @pytest.mark.parametrize("shape", SHAPES, ids=[s[0] for s in SHAPES])
-@pytest.mark.parametrize("flags", [0, 8, 4, 1], ids=["umma_default", "umma_one_sm", "umma_rows", "simt"])
+@pytest.mark.parametrize("flags", [0, 8, 1], ids=["umma_default", "umma_one_sm", "simt"])
 def test_cut_down_shapes_bf16(shape, flags):
     name, B, K, d, dd, V = shape
     cfg = gen.Config(name, B=B, K=K, d=d, d_draft=dd, V=V, sigma_W=0.2, sigma_w=0.05, match_lo=0.5, match_hi=0.95, seed=3)
     reps = _full_parity(cfg, (0.0, 0.3, 0.5, 1.0), flags=flags)
     assert all(r.seqs_exempt <= r.seqs // 2 + 1 for r in reps)
+
+
+MANY_TILES = [
+    # name, B, K, flags, kernel: a vocabulary of 60000 entries gives every CTA (or CTA pair) at least three
+    # tiles, so the alternation of the accumulator buffers, the wrap of the ring's phases from tile to
+    # tile and the write-back of the running maxima on a change of row tile are exercised for every
+    # tile width, not only the narrowest
+    ("vm64_many_tiles", 1, 39, 0, "umma_vm_128x64"),        # M = 40: 469 tiles of 128 entries on 148 CTAs
+    ("vm128_many_tiles", 4, 24, 0, "umma_vm_128x128"),      # M = 100
+    ("vm256_many_tiles", 5, 59, 8, "umma_vm_128x256"),      # M = 300 on the one-SM kernel: two row tiles (256 + 48 rows)
+    ("pair_narrow_many_tiles", 5, 39, 0, "umma_pair_256x256"),  # M = 200: 235 narrow tiles on 74 pairs
+    ("pair_wide_many_tiles", 5, 59, 0, "umma_pair_256x256"),    # M = 300: 235 wide tiles (160 + 144 rows)
+    ("pair_wide_two_row_tiles", 10, 59, 0, "umma_pair_256x256"),  # M = 600: 470 wide tiles, two row tiles (160 + 144 rows each)
+]
+
+
+@pytest.mark.parametrize("shape", MANY_TILES, ids=[s[0] for s in MANY_TILES])
+def test_every_kernel_walks_several_tiles_per_cta(shape):
+    name, B, K, flags, path = shape
+    cfg = gen.Config(name, B=B, K=K, d=128, d_draft=64, V=60000, sigma_W=0.2, sigma_w=0.05, match_lo=0.5, match_hi=0.95, seed=21)
+    reps = _full_parity(cfg, (0.0, 0.5, 1.0), flags=flags, expect_path=path)
+    assert all(r.seqs_exempt <= r.seqs // 2 + 1 for r in reps)
+
+
+def test_largest_window_the_interface_accepts():
+    """K = 1024, the largest window a handle may be created for: the scan kernel's shared-memory
+    layout there needs four bytes more than the default limit."""
+    cfg = gen.Config("k1024", B=2, K=1024, d=64, d_draft=64, V=300, sigma_W=0.2, sigma_w=0.05, match_lo=0.9, match_hi=0.99, seed=22)
+    _full_parity(cfg, (0.0, 0.5, 1.0))
 
 
 @pytest.mark.parametrize("layout", [0, 1])
@@ -195,7 +224,7 @@ def test_ties_zeros_and_out_of_range_draft_tokens():
     tok = gen.plant_draft_tokens(cfg, y)
     tok[0, 1] = -5          # ids outside the vocabulary are data: they simply never match
     tok[1, 2] = cfg.V + 9
-    for flags in (0, 8, 4, 1):
+    for flags in (0, 8, 1):
         case = DeviceCase(cfg, W, ht, hd, w, flags=flags)
         try:
             o = orc.verify(ht, hd, W, tok, w, 0.0, 0.5, cfg.dtype)
@@ -209,7 +238,7 @@ def test_ties_zeros_and_out_of_range_draft_tokens():
     # +0 and -0 logits still ties
     Wz = np.zeros_like(W)
     hneg = ht.copy()
-    for flags in (0, 4, 1):
+    for flags in (0, 1):
         case = DeviceCase(cfg, Wz, hneg, hd, w, flags=flags)
         try:
             g = case.run(np.zeros((cfg.B, cfg.K), np.int32), 0.5)
@@ -265,7 +294,7 @@ def test_all_negative_logits_are_not_beaten_by_the_zero_filled_tail():
     y = _oracle_y(cfg, W, ht)
     tok = gen.plant_draft_tokens(cfg, y)
     o = orc.verify(ht, None, W, tok, w, 0.0, 0.5, cfg.dtype)
-    for flags in (0, 8, 4):  # M = 153: two-SM kernel, one-SM kernel, row tiles
+    for flags in (0, 8):  # M = 153: two-SM kernel, one-SM kernel
         case = DeviceCase(cfg, W, ht, None, w, flags=flags)
         try:
             g = case.run(tok, 0.5)

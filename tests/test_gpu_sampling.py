@@ -184,9 +184,3 @@ def test_sampling_is_refused_where_it_is_not_defined():
         h.set_top_k(4)
     finally:
         h.destroy()
-    h = aj.Handle(0, 2, 4, 128, 0, 512, flags=aj.AJ_FLAG_ROW_TILES)
-    try:
-        assert h.set_sampling(1.0, check=False) == aj.AJ_ERR_UNSUPPORTED
-        assert h.set_sampling(0.0, check=False) == aj.AJ_OK
-    finally:
-        h.destroy()

@@ -144,6 +144,8 @@ class GpuWorkload:
         self.handle_t = aj.Handle(device, cfg.B, cfg.K, cfg.d, cfg.d_draft, cfg.V, aj.AJ_BF16, aj.AJ_W_VD,
                                   flags | aj.AJ_FLAG_TIME_KERNELS, shard=shard[1])
         for h in (self.handle, self.handle_t):  # the variants of the acceptance step: top-K rule, sampled target tokens
+            if rule and rule.get("fuse_judge"):
+                h.fuse_judge(self.w, stream=torch.cuda.current_stream().cuda_stream)
             if rule and rule.get("top_k"):
                 h.set_top_k(rule["top_k"])
             if rule and rule.get("temperature"):
@@ -443,6 +445,7 @@ def main():
     ap.add_argument("--flags", type=int, default=0, help="extra aj_create flags (kernel selection switches, for comparisons)")
     ap.add_argument("--top-k", type=int, default=0, help="time the top-K acceptance rule (paper Section 4.1) instead of the classifier")
     ap.add_argument("--temperature", type=float, default=0.0, help="time sampled verification (paper Appendix A) at this temperature instead of greedy")
+    ap.add_argument("--fuse-judge", action="store_true", help="compute the classifier's target half inside the projection kernel (paper Section 3.2)")
     ap.add_argument("--w-copies", type=int, default=None, help="copies of W_lm to rotate over (default 3, or 2 for the 70B shape)")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -468,7 +471,7 @@ def main():
     copies = args.w_copies or (3 if head.d * head.V * 2 < 1.5e9 else 2)
 
     vocab = args.sharding == "vocab"
-    rule = {k: v for k, v in (("top_k", args.top_k), ("temperature", args.temperature)) if v}
+    rule = {k: v for k, v in (("top_k", args.top_k), ("temperature", args.temperature), ("fuse_judge", args.fuse_judge)) if v}
     if not vocab:
         head = ajd.rank_config(head, rank)  # every rank verifies its own sequences
     W_host = gen.make_W(head)

@@ -113,6 +113,25 @@ aj_status aj_verify(aj_handle h, const void *h_target, const void *h_draft, cons
                     float *top1_val, float *judge_p, void *cuda_stream);
 
 /*
+ * Fold the target half of the classifier into the LM-head projection (the paper's Section 3.2,
+ * "Classifier model & training": the classifier "can be fused with the existing LM head layer", which
+ * makes its computation nearly free).  judge_w . [h_draft ; h_target] splits into a draft half and a
+ * target half, and the target half, w_target . h_target[row], has the shape of one more logit.  This call
+ * appends w_target = judge_w[d_draft ..] to the vocabulary as three bf16 rows b0 + b1 + b2 that add up to
+ * w_target to fp32 precision (each the bf16 rounding of what the earlier ones leave); later cycles on
+ * this handle compute their dot products with every row of h_target in one extra vocabulary block of the
+ * projection kernel (tensor cores, fp32 accumulation; the rows lie past V and never enter the argmax)
+ * and the judge kernel then reads only the h_draft rows of the mismatching positions (nothing when
+ * d_draft == 0).  Results agree with the unfused path within the tolerance stated for judge_p.
+ *   judge_w  [d_draft + d] f32 DEVICE: read by a small kernel enqueued on cuda_stream; later calls of
+ *            aj_verify and its variants on this handle must pass weights with the same target half
+ *            (the draft half and judge_b are still taken from each call).  NULL switches back.
+ * Only on the tensor-core path (AJ_BF16, d % 64 == 0): AJ_ERR_UNSUPPORTED otherwise.  Ignored while the
+ * top-K rule is in force.  Errors: AJ_ERR_INVALID_ARG, AJ_ERR_UNSUPPORTED, AJ_ERR_CUDA.
+ */
+aj_status aj_fuse_judge(aj_handle h, const float *judge_w, void *cuda_stream);
+
+/*
  * Switch the acceptance rule of a handle to the top-K rule of the paper's Section 4.1 (the lossy
  * baseline it compares with): a mismatching draft token is accepted iff it is among the top_k most
  * likely tokens of the target, i.e. iff fewer than top_k vocabulary entries have a larger logit

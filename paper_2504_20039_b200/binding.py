@@ -21,6 +21,7 @@ EXPORTS = (
     "aj_create", "aj_verify", "aj_verify_host", "aj_last_status", "aj_last_gemm_ms", "aj_gemm_ms_stats", "aj_last_launch_count",
     "aj_last_gemm_path", "aj_pair_schedule", "aj_destroy", "aj_set_top_k", "aj_set_sampling", "aj_verify_tree", "aj_lr_fit", "aj_shard_exchange_bytes", "aj_shard_exchange_alloc", "aj_shard_exchange_free", "aj_shard_range", "aj_create_sharded",
     "aj_shard_project", "aj_shard_finish", "aj_ipc_export", "aj_ipc_import", "aj_ipc_close", "aj_status_string", "aj_version", "aj_verify_static",
+    "aj_fuse_judge",
 )
 
 _lib = None
@@ -92,6 +93,8 @@ def lib() -> ctypes.CDLL:
         L.aj_ipc_import.restype = ci
         L.aj_ipc_close.argtypes = [vp]
         L.aj_ipc_close.restype = ci
+        L.aj_fuse_judge.argtypes = [vp, vp, vp]
+        L.aj_fuse_judge.restype = ci
         L.aj_set_top_k.argtypes = [vp, ci]
         L.aj_set_top_k.restype = ci
         L.aj_set_sampling.argtypes = [vp, ctypes.c_float, ctypes.c_uint64, ctypes.c_uint64]
@@ -287,6 +290,13 @@ class Handle:
                                   _ptr(target_tok), stream or None)
         if check and st != AJ_OK:
             raise AjError(st, "aj_verify_host")
+        return st
+
+    def fuse_judge(self, judge_w=None, stream: int = 0, check: bool = True) -> int:
+        """aj_fuse_judge: compute the classifier's target half in the projection kernel (None: back to the judge kernel)."""
+        st = lib().aj_fuse_judge(self._h, _ptr(judge_w), stream or None)
+        if check and st != AJ_OK:
+            raise AjError(st, "aj_fuse_judge")
         return st
 
     def set_top_k(self, top_k: int, check: bool = True) -> int:

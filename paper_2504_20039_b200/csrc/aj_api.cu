@@ -19,7 +19,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
 struct TmapSlot {
     const void *ptr = nullptr;
     long long rows = 0;
-    int box_rows = 0;  // -1: the [d, V] map of W_lm (64 entries x 64 k-rows per box)
+    int box_rows = 0;  // -1: a [d, rows] map, W_lm stored [d, V] (64 entries x 64 k-rows per box)
     unsigned long long stamp = 0;
     CUtensorMap map;
 };
@@ -64,6 +64,10 @@ struct aj_handle_s {
     float *rk_thr = nullptr;         // [max_M] the draft tokens' own logits
     int *rk_tok = nullptr;           // [max_M]
     unsigned *rk_cnt = nullptr;      // [max_M] entries that outrank them
+    // the classifier's target half folded into the projection (aj_fuse_judge)
+    bool fold = false;
+    void *fold_rows = nullptr;       // three bf16 rows that add up to w_target, laid out like W_lm
+    float *fold_parts = nullptr;     // [3][max_M] their dot products with every row of h_target
 };
 
 // Exchange buffer of one GPU: 256 bytes of flags (one 8-byte epoch per source GPU), then two slot
@@ -230,7 +234,9 @@ aj_status aj_create(aj_handle *out, int device, int max_B, int max_K, int d, int
               cudaMalloc(&h->st_acc, (size_t)max_B * 4) == cudaSuccess &&
               cudaMalloc(&h->st_next, (size_t)max_B * 4) == cudaSuccess && cudaMalloc(&h->st_tt, max_M * 4) == cudaSuccess &&
               cudaMalloc(&h->rk_thr, max_M * 4) == cudaSuccess && cudaMalloc(&h->rk_tok, max_M * 4) == cudaSuccess &&
-              cudaMalloc(&h->rk_cnt, max_M * 4) == cudaSuccess;
+              cudaMalloc(&h->rk_cnt, max_M * 4) == cudaSuccess &&
+              cudaMalloc(&h->fold_rows, (size_t)8 * d * 2) == cudaSuccess &&
+              cudaMalloc(&h->fold_parts, (size_t)JUDGE_FOLD_ROWS * max_M * 4) == cudaSuccess;
     if (ok && (flags & AJ_FLAG_TIME_KERNELS))
         for (int i = 0; ok && i < EVENT_RING; i++)
             ok = cudaEventCreate(&h->ev0[i]) == cudaSuccess && cudaEventCreate(&h->ev1[i]) == cudaSuccess;
@@ -267,6 +273,8 @@ aj_status aj_destroy(aj_handle h) {
     cudaFree(h->rk_thr);
     cudaFree(h->rk_tok);
     cudaFree(h->rk_cnt);
+    cudaFree(h->fold_rows);
+    cudaFree(h->fold_parts);
     for (int i = 0; i < EVENT_RING; i++) {
         if (h->ev0[i]) cudaEventDestroy(h->ev0[i]);
         if (h->ev1[i]) cudaEventDestroy(h->ev1[i]);
@@ -330,6 +338,12 @@ static aj_status enqueue_project(aj_handle h, const void *h_target, const void *
     g.w_layout = h->layout;
     g.keys = h->keys;
     g.status = h->status;
+    const bool fold = h->fold && h->umma_ok && h->top_k == 0;  // the top-K rule does not consult the classifier
+    if (fold) {
+        g.fold.rows = h->fold_rows;
+        g.fold.parts = h->fold_parts;
+        g.fold.stride = h->max_B * (h->max_K + 1);
+    }
     if (h->world) {
         ++h->epoch;
         const size_t max_M = (size_t)h->max_B * (h->max_K + 1);
@@ -352,12 +366,14 @@ static aj_status enqueue_project(aj_handle h, const void *h_target, const void *
         // tensor-bound regime: two-SM tiles of 256 vocabulary entries x up to 256 rows
         UmmaPlan p;
         p.bn = 256;
-        const PairSched sc = pair_schedule(M, V, d);
+        const PairSched sc = pair_schedule(M, V, d, fold);
         const CUtensorMap *tw = get_tmap(h, W_lm, V, h->layout == AJ_W_DV ? -1 : 128);
         const CUtensorMap *th = get_tmap(h, h_target, M, sc.box_rows);
-        if (!th || !tw) return AJ_ERR_CUDA;
+        const CUtensorMap *tj = fold ? get_tmap(h, h->fold_rows, h->layout == AJ_W_DV ? 8 : JUDGE_FOLD_ROWS, h->layout == AJ_W_DV ? -1 : 128) : tw;
+        if (!th || !tw || !tj) return AJ_ERR_CUDA;
         p.tmap_h = *th;
         p.tmap_w = *tw;
+        p.tmap_j = *tj;
         const long long tiles = (long long)sc.n_n * sc.n_v;
         const int pairs = umma_pair_max_pairs();
         p.grid = 2 * (int)(tiles < pairs ? tiles : pairs);
@@ -368,10 +384,12 @@ static aj_status enqueue_project(aj_handle h, const void *h_target, const void *
         p.bn = vm_choose_bn(M);
         const CUtensorMap *tw = get_tmap(h, W_lm, V, h->layout == AJ_W_DV ? -1 : 128);
         const CUtensorMap *th = get_tmap(h, h_target, M, p.bn);
-        if (!th || !tw) return AJ_ERR_CUDA;
+        const CUtensorMap *tj = fold ? get_tmap(h, h->fold_rows, h->layout == AJ_W_DV ? 8 : JUDGE_FOLD_ROWS, h->layout == AJ_W_DV ? -1 : 128) : tw;
+        if (!th || !tw || !tj) return AJ_ERR_CUDA;
         p.tmap_h = *th;
         p.tmap_w = *tw;
-        const long long tiles = (long long)((M + p.bn - 1) / p.bn) * ((V + 127) / 128);
+        p.tmap_j = *tj;
+        const long long tiles = (long long)((M + p.bn - 1) / p.bn) * ((V + 127) / 128 + (fold ? 1 : 0));
         p.grid = (int)(tiles < h->num_sms ? tiles : h->num_sms);
         e = launch_umma_vm(g, p, stream);
         h->last_path = umma_vm_path_name(p.bn);
@@ -423,6 +441,10 @@ static aj_status enqueue_finish(aj_handle h, const void *h_target, const void *h
     j.top_k = h->top_k;
     j.V = h->V;
     j.rank_cnt = h->rk_cnt;
+    if (h->fold && h->umma_ok && h->top_k == 0) {
+        j.fold_parts = h->fold_parts;
+        j.fold_stride = h->max_B * (h->max_K + 1);
+    }
     j.accept_len = accept_len;
     j.next_tok = next_tok;
     j.target_tok = target_tok;
@@ -707,11 +729,26 @@ aj_status aj_set_sampling(aj_handle h, float temperature, uint64_t seed, uint64_
     return AJ_OK;
 }
 
+aj_status aj_fuse_judge(aj_handle h, const float *judge_w, void *cuda_stream) {
+    if (!h) return AJ_ERR_INVALID_ARG;
+    if (!judge_w) {
+        h->fold = false;
+        return AJ_OK;
+    }
+    if (!h->umma_ok) return AJ_ERR_UNSUPPORTED;  // the CUDA-core kernel has no extra rows to offer
+    DeviceGuard guard(h->device);
+    if (!guard.ok()) return AJ_ERR_CUDA;
+    if (launch_judge_split(judge_w + h->d_draft, h->d, h->layout, h->fold_rows, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+        return AJ_ERR_CUDA;
+    h->fold = true;
+    return AJ_OK;
+}
+
 int aj_last_launch_count(aj_handle h) { return h ? h->last_launches : 0; }
 
 aj_status aj_pair_schedule(int M, int d, int V, int32_t out[10]) {
     if (!out || M < 1 || d < 1 || V < 1) return AJ_ERR_INVALID_ARG;
-    const PairSched sc = pair_schedule(M, V, d);
+    const PairSched sc = pair_schedule(M, V, d, 0);
     out[0] = sc.n_v;
     out[1] = sc.n_n;
     out[2] = sc.u_base;

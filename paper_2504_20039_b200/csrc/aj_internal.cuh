@@ -235,6 +235,22 @@ __device__ inline void add_gumbel_noise(const Noise &nz, float (&x)[32], int v, 
 }
 #endif
 
+// ------------------------------------------------ the classifier's target half as rows of the LM head
+//
+// z = b + w_draft . h_draft[row] + w_target . h_target[row]: the second dot product has the shape of
+// one more logit.  When it is folded into the projection, w_target is appended to the vocabulary as
+// THREE bf16 rows whose sum is w_target to fp32 precision (w = b0 + b1 + b2, each the bf16 rounding of
+// what the previous ones leave), in one extra vocabulary block that follows the real ones.  Its
+// entries lie past V, so they never enter the argmax; the epilogue stores the three partial dot
+// products of every row to parts[3][stride] and the scan kernel adds them in a fixed order.
+struct JudgeFold {
+    const void *rows = nullptr;  // bf16, laid out like W_lm: [3, d], or [d, 8] (3 of 8 entries used); nullptr: not folded
+    float *parts = nullptr;      // [3][stride]
+    int stride = 0;
+};
+constexpr int JUDGE_FOLD_ROWS = 3;
+cudaError_t launch_judge_split(const float *w_target, int d, int w_layout, void *rows_out, cudaStream_t stream);
+
 struct RankPrepArgs {
     const void *h;             // [M, d]
     const void *W;             // LM head
@@ -260,6 +276,7 @@ struct GemmArgs {
     Publish pub;
     RankArgs rank;       // thr != nullptr: also count, per row, the entries that outrank the draft token
     Noise noise;         // temperature > 0: the argmax is taken over logit + temperature * Gumbel noise
+    JudgeFold fold;      // rows != nullptr: one more vocabulary block computes the classifier's target half
 };
 
 // What a projection kernel's epilogue does besides the argmax.
@@ -272,6 +289,7 @@ cudaError_t launch_simt_gemm_argmax(const GemmArgs &a, int num_sms, cudaStream_t
 struct UmmaPlan {
     CUtensorMap tmap_h;  // rows of h, 128-byte swizzle
     CUtensorMap tmap_w;  // rows of W (or, for [d, V], 64 entries x 64 k-rows)
+    CUtensorMap tmap_j;  // the folded classifier rows, same box as tmap_w (only with GemmArgs::fold)
     int bn;              // rows of h per tile
     int grid;
 };
@@ -285,7 +303,8 @@ const char *umma_vm_path_name(int bn);
 // per tile.  tmap_w has a 64 x 128 box, tmap_h a 64 x pair_schedule().box_rows box; p.grid = 2 *
 // number of pairs.
 struct PairSched {
-    int n_v;               // blocks of 256 vocabulary entries
+    int n_v;               // blocks of 256 vocabulary entries, the block of the folded classifier rows included
+    int fold;              // 1: the last block holds the classifier rows instead of vocabulary entries
     int n_n;               // row tiles
     int u_base, u_rem;     // row tile i holds u_base + (i < u_rem) units of 16 rows
     int box_rows;          // rows of h each CTA of a pair stages per k-block and accumulator
@@ -294,7 +313,7 @@ struct PairSched {
     int n_groups;          // row tiles are walked in groups ...
     int g_base, g_rem;     // ... group g holds g_base + (g < g_rem) row tiles
 };
-PairSched pair_schedule(int M, int V, int d);
+PairSched pair_schedule(int M, int V, int d, int fold);
 cudaError_t umma_pair_prepare(int num_sms);
 int umma_pair_max_pairs();
 cudaError_t launch_umma_pair(const GemmArgs &a, const UmmaPlan &p, cudaStream_t stream);
@@ -313,6 +332,8 @@ struct JudgeArgs {
     int top_k = 0;                   // > 0: the top-K rule replaces the classifier
     int V = 0;                       // vocabulary size (top-K rule: ids outside it are never accepted)
     unsigned *rank_cnt = nullptr;    // [B*R] counts from the projection kernel (top-K rule)
+    const float *fold_parts = nullptr;  // [3][fold_stride] the target half of the classifier from the projection kernel, else nullptr
+    int fold_stride = 0;
     const int32_t *parent = nullptr; // [B, K] tree drafts: parent node of every node (-1 = the root), else nullptr
     int32_t *best_node = nullptr;    // [B] tree drafts: the deepest accepted node (-1 = the root), optional
     int32_t *accept_len, *next_tok, *target_tok;

@@ -17,6 +17,9 @@
 // (the root always is) and it matches or is forgiven; the result is the deepest accepted node, the
 // lowest index among equally deep ones.  A chain (parent[i] = i - 1) is the window case.
 //
+// When the projection kernel has computed the target half of w . x as three extra rows of the LM head
+// (a.fold_parts), only the draft half is read here and the three partial sums are added to it.
+//
 // The kernel is launched as a programmatic dependent of the projection kernel: its blocks may
 // become resident while that kernel still runs and wait at the grid dependency before they
 // read the keys.  Each key is cleared right after it is read, so the next cycle finds zeros.
@@ -136,7 +139,7 @@ __global__ void __maxnreg__(96) judge_scan_kernel(JudgeArgs a) {
         for (size_t l = threadIdx.x; l < wlines; l += blockDim.x)
             asm volatile("prefetch.global.L2 [%0];" ::"l"(wbytes + l * 128));
         if ((long long)gridDim.x * K <= 256) {
-            const size_t lt = (row_bytes_t + 127) / 128, ld = a.h_draft ? (row_bytes_d + 127) / 128 : 0;
+            const size_t lt = a.fold_parts ? 0 : (row_bytes_t + 127) / 128, ld = a.h_draft ? (row_bytes_d + 127) / 128 : 0;
             const size_t per_row = lt + ld;
             for (size_t l = threadIdx.x; l < per_row * (R - 1); l += blockDim.x) {
                 const size_t row = (size_t)b * R + 1 + l / per_row, o = l % per_row;
@@ -204,7 +207,7 @@ __global__ void __maxnreg__(96) judge_scan_kernel(JudgeArgs a) {
                      ((reinterpret_cast<uintptr_t>(a.h_draft) & 15) == 0) &&
                      ((reinterpret_cast<uintptr_t>(a.judge_w) & 15) == 0);
     const int split = a.d_draft / epc;                 // chunks that belong to the draft row
-    const int chunks = (a.d_draft + a.d) / epc;
+    const int chunks = (a.d_draft + (a.fold_parts ? 0 : a.d)) / epc;  // the target half may come from the projection kernel
     for (int it = warp; it < K * SEGS; it += nwarps) {
         const int i = it / SEGS, seg = it % SEGS;
         if (!mis_s[i] || i + 1 >= R || a.top_k > 0) continue;  // at mismatches only, where the features exist; not under the top-K rule
@@ -219,7 +222,7 @@ __global__ void __maxnreg__(96) judge_scan_kernel(JudgeArgs a) {
                              : segment_dot<false>(xd, xt, a.judge_w, split, c0, c1, lane);
         } else {
             s = seg == 0 ? scalar_dot(xd, a.judge_w, a.d_draft, a.dtype, lane) +
-                               scalar_dot(xt, a.judge_w + a.d_draft, a.d, a.dtype, lane)
+                               (a.fold_parts ? 0.0f : scalar_dot(xt, a.judge_w + a.d_draft, a.d, a.dtype, lane))
                          : 0.0f;
         }
 #pragma unroll
@@ -246,6 +249,10 @@ __global__ void __maxnreg__(96) judge_scan_kernel(JudgeArgs a) {
             float z = a.judge_b;
 #pragma unroll
             for (int seg = 0; seg < SEGS; seg++) z += part_s[i * SEGS + seg];
+            if (a.fold_parts) {
+                const float *fp = a.fold_parts + (size_t)b * R + (i + 1);  // the row that encodes draft token i
+                z += (__ldcg(fp) + __ldcg(fp + a.fold_stride)) + __ldcg(fp + 2 * (size_t)a.fold_stride);
+            }
             p = 1.0f / (1.0f + expf(-z));
             const bool forgiven = (a.tau <= 0.0f) ? false : (a.tau >= 1.0f) ? true : (p < a.tau);
             rej = forgiven ? 0 : 1;
@@ -295,7 +302,34 @@ __global__ void __maxnreg__(96) judge_scan_kernel(JudgeArgs a) {
     }
 }
 
+// w_target as three bf16 rows whose sum is w_target to fp32 precision, laid out like the LM head:
+// [3, d] for a [V, d] head, [d, 8] (entries 0..2) for a [d, V] head.
+__global__ void judge_split_kernel(const float *__restrict__ w, int d, int w_layout, __nv_bfloat16 *__restrict__ out) {
+    const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= d) return;
+    float r = w[k];
+    __nv_bfloat16 b[JUDGE_FOLD_ROWS];
+#pragma unroll
+    for (int i = 0; i < JUDGE_FOLD_ROWS; i++) {
+        b[i] = __float2bfloat16_rn(r);
+        r -= __bfloat162float(b[i]);  // exact: the remainder has fewer significant bits than r
+    }
+#pragma unroll
+    for (int i = 0; i < 8; i++) {
+        const __nv_bfloat16 x = i < JUDGE_FOLD_ROWS ? b[i] : __float2bfloat16_rn(0.0f);
+        if (w_layout)
+            out[(size_t)k * 8 + i] = x;
+        else if (i < JUDGE_FOLD_ROWS)
+            out[(size_t)i * d + k] = x;
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_judge_split(const float *w_target, int d, int w_layout, void *rows_out, cudaStream_t stream) {
+    judge_split_kernel<<<(d + 255) / 256, 256, 0, stream>>>(w_target, d, w_layout, static_cast<__nv_bfloat16 *>(rows_out));
+    return cudaGetLastError();
+}
 
 cudaError_t launch_judge_scan(const JudgeArgs &a, cudaStream_t stream) {
     cudaLaunchConfig_t cfg = {};

@@ -116,9 +116,9 @@ __device__ inline Tile decode_tile(const PairSched &sc, int t) {
 template <bool DUAL, bool WDV, int EPI>
 __global__ void __launch_bounds__(num_threads(DUAL), 1)
 umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_h,
-                 int M, int V, int d, PairSched sc, int stream_w, int v_offset,
+                 const __grid_constant__ CUtensorMap tmap_j, int M, int V, int d, PairSched sc, int stream_w, int v_offset,
                  unsigned long long *__restrict__ keys, int *__restrict__ status, const Publish pub, const RankArgs rk,
-                 const Noise nz) {
+                 const Noise nz, float *__restrict__ fold_parts, int fold_stride) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;  // the same offset in both CTAs: one descriptor serves both
@@ -139,6 +139,7 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
     const int num_pairs = gridDim.x >> 1;
     const int num_kb = d / BK;
     const int num_tiles = sc.n_n * sc.n_v;
+    const int fold_tile = sc.fold ? sc.n_v - 1 : -1;  // the vocabulary block that holds the classifier rows
     const int stages = sc.stages;
     const uint32_t b_bytes = (uint32_t)sc.box_rows * BK * 2;       // one accumulator's rows of h staged by this CTA
     constexpr int n_acc = DUAL ? 2 : 1;
@@ -187,7 +188,9 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
             bool ok = true;
             for (int t = pair; ok && t < num_tiles; t += num_pairs) {
                 const Tile tl = decode_tile(sc, t);
-                const int w_row = tl.v_tile * BV + (int)rank * BV_CTA;
+                const bool fold = tl.v_tile == fold_tile;
+                const CUtensorMap *tw = fold ? &tmap_j : &tmap_w;  // the classifier rows start at entry 0 of their own map
+                const int w_row = (fold ? 0 : tl.v_tile * BV) + (int)rank * BV_CTA;
                 const int h_row0 = tl.row0[0] + (int)rank * (tl.n_inst[0] >> 1);
                 const int h_row1 = tl.row0[1] + (int)rank * (tl.n_inst[1] >> 1);
                 for (int kb = 0; kb < num_kb; kb++) {
@@ -200,10 +203,10 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
                     if (rank == 0) mbar_expect_tx(full_bar(s), stage_tx);
                     const uint32_t a_dst = base + s * stage_bytes;
                     if (WDV) {  // W stored [d, V]: two boxes of 64 entries x 64 k-rows
-                        tma_load_2d_pair(a_dst, &tmap_w, w_row, kb * BK, leader_full, pol_w);
-                        tma_load_2d_pair(a_dst + A_BYTES / 2, &tmap_w, w_row + 64, kb * BK, leader_full, pol_w);
+                        tma_load_2d_pair(a_dst, tw, w_row, kb * BK, leader_full, pol_w);
+                        tma_load_2d_pair(a_dst + A_BYTES / 2, tw, w_row + 64, kb * BK, leader_full, pol_w);
                     } else {
-                        tma_load_2d_pair(a_dst, &tmap_w, kb * BK, w_row, leader_full, pol_w);
+                        tma_load_2d_pair(a_dst, tw, kb * BK, w_row, leader_full, pol_w);
                     }
                     tma_load_2d_pair(a_dst + A_BYTES, &tmap_h, kb * BK, h_row0, leader_full, pol_h);
                     if (n_acc == 2) tma_load_2d_pair(a_dst + A_BYTES + b_bytes, &tmap_h, kb * BK, h_row1, leader_full, pol_h);
@@ -310,6 +313,18 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
                 {
                     float v[32];
                     tmem_ld32(tbase + acc_col(it, a) + (uint32_t)(c * 32), v);
+                    if (tl.v_tile == fold_tile) {
+                        // the classifier rows: lanes 0..2 of the leader's first quadrant hold the three partial
+                        // dot products of 32 rows of h; they are stored, and nothing of this block is a logit
+                        if (rank == 0 && q == 0 && lane < JUDGE_FOLD_ROWS) {
+#pragma unroll
+                            for (int j = 0; j < 32; j++) {
+                                const int row = row_a + c * 32 + j;
+                                if (c * 32 + j < n_inst && row < M) fold_parts[(size_t)lane * fold_stride + row] = v[j];
+                            }
+                        }
+                        continue;
+                    }
                     if (EPI == EPI_COUNT) count_outranking(rk, v, v_first, v_ok, row_a + c * 32, n_inst - c * 32, M, lane);
                     if (EPI == EPI_SAMPLE) add_gumbel_noise(nz, v, v_first + lane + v_offset, row_a + c * 32);
                     // the lowest threshold of the chunk (a row without a key yet: everything qualifies)
@@ -414,8 +429,9 @@ cudaError_t umma_pair_prepare(int num_sms) {
 
 int umma_pair_max_pairs() { return g_max_pairs; }
 
-PairSched pair_schedule(int M, int V, int d) {
+PairSched pair_schedule(int M, int V, int d, int fold) {
     PairSched sc;
+    sc.fold = fold ? 1 : 0;
     const int units = (M + 15) / 16;  // rows in units of 16 (the UMMA N granule)
     // Wide tiles (up to 512 rows on two accumulators with an issuing warp each) for every batch of more
     // than 256 rows; up to 256 rows one narrow tile per vocabulary block, double-buffered.
@@ -424,7 +440,7 @@ PairSched pair_schedule(int M, int V, int d) {
     sc.n_n = (units + cap - 1) / cap;
     sc.u_base = units / sc.n_n;
     sc.u_rem = units % sc.n_n;
-    sc.n_v = (V + BV - 1) / BV;
+    sc.n_v = (V + BV - 1) / BV + sc.fold;
     const int u_max = sc.u_base + (sc.u_rem ? 1 : 0);
     // rows of h each CTA stages per accumulator: half of the largest accumulator
     sc.box_rows = 8 * (sc.dual ? (u_max + 1) / 2 : u_max);
@@ -441,7 +457,7 @@ PairSched pair_schedule(int M, int V, int d) {
 }
 
 cudaError_t launch_umma_pair(const GemmArgs &a, const UmmaPlan &p, cudaStream_t stream) {
-    const PairSched sc = pair_schedule(a.M, a.V, a.d);
+    const PairSched sc = pair_schedule(a.M, a.V, a.d, a.fold.rows != nullptr);
     const int stream_w = (sc.n_n == 1) ? 1 : 0;  // W is read by one pair only: do not keep it in L2
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)p.grid);  // 2 CTAs per pair
@@ -465,8 +481,8 @@ cudaError_t launch_umma_pair(const GemmArgs &a, const UmmaPlan &p, cudaStream_t 
     auto kernel = a.noise.temperature > 0.0f ? pick(std::integral_constant<int, EPI_SAMPLE>{})
                   : a.rank.thr               ? pick(std::integral_constant<int, EPI_COUNT>{})
                                              : pick(std::integral_constant<int, EPI_PLAIN>{});
-    return cudaLaunchKernelEx(&cfg, kernel, p.tmap_w, p.tmap_h, a.M, a.V, a.d, sc, stream_w, a.v_offset, a.keys, a.status,
-                              a.pub, a.rank, a.noise);
+    return cudaLaunchKernelEx(&cfg, kernel, p.tmap_w, p.tmap_h, a.fold.rows ? p.tmap_j : p.tmap_w, a.M, a.V, a.d, sc, stream_w,
+                              a.v_offset, a.keys, a.status, a.pub, a.rank, a.noise, a.fold.parts, a.fold.stride);
 }
 
 }  // namespace aj

@@ -55,9 +55,9 @@ template <int BN> struct VCfg {
 template <int BN, bool WDV, int EPI>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 umma_vm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_h,
-               int M, int V, int d, int n_n, int n_v, int stream_w, int v_offset,
-               unsigned long long *__restrict__ keys, int *__restrict__ status, const Publish pub, const RankArgs rk,
-               const Noise nz) {
+               const __grid_constant__ CUtensorMap tmap_j, int M, int V, int d, int n_n, int n_v, int fold_tile,
+               int stream_w, int v_offset, unsigned long long *__restrict__ keys, int *__restrict__ status, const Publish pub,
+               const RankArgs rk, const Noise nz, float *__restrict__ fold_parts, int fold_stride) {
     using C = VCfg<BN>;
     constexpr int STAGES = C::STAGES;
     extern __shared__ uint8_t smem_raw[];
@@ -116,6 +116,9 @@ umma_vm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
             bool ok = true;
             for (int t = blockIdx.x; ok && t < num_tiles; t += gridDim.x) {
                 const int n_tile = t % n_n, v_tile = t / n_n;
+                const bool fold = v_tile == fold_tile;  // the block after the vocabulary: the classifier rows, entry 0 of their own map
+                const CUtensorMap *tw = fold ? &tmap_j : &tmap_w;
+                const int w_row = fold ? 0 : v_tile * BV;
                 for (int kb = 0; kb < num_kb; kb++) {
                     if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) {
                         give_up();
@@ -125,10 +128,10 @@ umma_vm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                     mbar_expect_tx(full_bar(s), C::STAGE_BYTES);
                     const uint32_t a_dst = base + s * C::STAGE_BYTES;
                     if (WDV) {  // W stored [d, V]: two boxes of 64 entries x 64 k-rows
-                        tma_load_2d(a_dst, &tmap_w, v_tile * BV, kb * BK, full_bar(s), pol_w);
-                        tma_load_2d(a_dst + A_BYTES / 2, &tmap_w, v_tile * BV + 64, kb * BK, full_bar(s), pol_w);
+                        tma_load_2d(a_dst, tw, w_row, kb * BK, full_bar(s), pol_w);
+                        tma_load_2d(a_dst + A_BYTES / 2, tw, w_row + 64, kb * BK, full_bar(s), pol_w);
                     } else {
-                        tma_load_2d(a_dst, &tmap_w, kb * BK, v_tile * BV, full_bar(s), pol_w);
+                        tma_load_2d(a_dst, tw, kb * BK, w_row, full_bar(s), pol_w);
                     }
                     tma_load_2d(a_dst + A_BYTES, &tmap_h, kb * BK, n_tile * BN, full_bar(s), pol_h);
                     if (++s == STAGES) {
@@ -221,6 +224,18 @@ umma_vm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                 if (c * 32 < n_inst) {  // warp-uniform
                     float v[32];
                     tmem_ld32(taddr + c * 32, v);
+                    if (v_tile == fold_tile) {
+                        // the classifier rows: lanes 0..2 of the first quadrant hold the three partial dot
+                        // products of 32 rows of h; they are stored, and nothing of this block is a logit
+                        if (q == 0 && lane < JUDGE_FOLD_ROWS) {
+#pragma unroll
+                            for (int j = 0; j < 32; j++) {
+                                const int row = n_tile * BN + c * 32 + j;
+                                if (c * 32 + j < n_inst && row < M) fold_parts[(size_t)lane * fold_stride + row] = v[j];
+                            }
+                        }
+                        continue;
+                    }
                     if (EPI == EPI_COUNT) count_outranking(rk, v, v_first, v_ok, n_tile * BN + c * 32, n_inst - c * 32, M, lane);
                     if (EPI == EPI_SAMPLE) add_gumbel_noise(nz, v, v_first + lane + v_offset, n_tile * BN + c * 32);
                     // all 32 reductions are issued before any result is used, so that their
@@ -265,7 +280,8 @@ umma_vm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
 template <int BN>
 cudaError_t launch_vm(const GemmArgs &a, const UmmaPlan &p, cudaStream_t stream) {
     const int n_n = (a.M + BN - 1) / BN;
-    const int n_v = (a.V + BV - 1) / BV;
+    const int fold = a.fold.rows ? 1 : 0;
+    const int n_v = (a.V + BV - 1) / BV + fold;  // one more block for the folded classifier rows
     const int stream_w = (n_n == 1) ? 1 : 0;  // W is read by one CTA only: do not keep it in L2
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)p.grid);
@@ -284,8 +300,9 @@ cudaError_t launch_vm(const GemmArgs &a, const UmmaPlan &p, cudaStream_t stream)
     auto kernel = a.noise.temperature > 0.0f ? pick(std::integral_constant<int, EPI_SAMPLE>{})
                   : a.rank.thr               ? pick(std::integral_constant<int, EPI_COUNT>{})
                                              : pick(std::integral_constant<int, EPI_PLAIN>{});
-    return cudaLaunchKernelEx(&cfg, kernel, p.tmap_w, p.tmap_h, a.M, a.V, a.d, n_n, n_v, stream_w, a.v_offset, a.keys,
-                              a.status, a.pub, a.rank, a.noise);
+    return cudaLaunchKernelEx(&cfg, kernel, p.tmap_w, p.tmap_h, fold ? p.tmap_j : p.tmap_w, a.M, a.V, a.d, n_n, n_v,
+                              fold ? n_v - 1 : -1, stream_w, a.v_offset, a.keys, a.status, a.pub, a.rank, a.noise, a.fold.parts,
+                              a.fold.stride);
 }
 
 }  // namespace

@@ -81,6 +81,13 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.rows.append((time.time(), [x.strip() for x in line.split(",")]))
 
+    def wait_first(self, timeout: float = 4.0):
+        """nvidia-smi takes a few hundred milliseconds to print its first row: wait for it, so that a
+        timed region that starts now falls inside the sampled time."""
+        t = time.time()
+        while self.proc and not self.rows and time.time() - t < timeout and self.proc.poll() is None:
+            time.sleep(0.01)
+
     def __exit__(self, *exc):
         if self.proc:
             time.sleep(0.03)
@@ -217,15 +224,18 @@ class GpuWorkload:
 
 
 # DRAM traffic per launch of the projection kernel (dram__bytes_read.sum + dram__bytes_write.sum of one
-# ncu capture; summaries under profiles/).  A figure is reported only while the kernel's sources still
-# hash to what was captured.
+# profiler capture each), kept as data next to the capture summaries.  A figure is reported only while
+# the kernel's sources still hash to what was captured.
 CSRC = os.path.join(ROOT, "paper_2504_20039_b200", "csrc")
-NCU_TRAFFIC = {
-    # (workload, kernel configuration): (bytes per launch, kernel source files, sha1 of those files)
-    ("c2_8b_b1_k16", "umma_vm_128x32"): (1.0547e9, ["aj_umma_vm.cu"], "e8fb306d3308"),        # profiles/umma_vm_128x32_c2_8b_b1_k16.md
-    ("c3_8b_b64_k32", "umma_pair_256x256"): (1.0809e9, ["aj_umma_pair.cu"], "82740e3d26df"),  # profiles/umma_pair_256x256_c3_8b_b64_k32.md
-    ("c4_70b_b32_k64", "umma_pair_256x256"): (3.1834e9, ["aj_umma_pair.cu"], "82740e3d26df"),  # profiles/umma_pair_256x256_c4_70b_b32_k64.md
-}
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "dram_traffic.json")
+
+
+def _traffic_table():
+    try:
+        with open(TRAFFIC_FILE) as f:
+            return {(e["workload"], e["kernel"]): (float(e["bytes_per_launch"]), e["sources"], e["sources_sha1_12"]) for e in json.load(f)["captures"]}
+    except (OSError, ValueError, KeyError):
+        return {}
 
 
 def _sources_sha(files):
@@ -239,7 +249,7 @@ def _sources_sha(files):
 
 
 def traffic_of(cfg: gen.Config, path: str):
-    ent = NCU_TRAFFIC.get((cfg.name, path))
+    ent = _traffic_table().get((cfg.name, path))
     if not ent:
         return None
     byts, files, sha = ent
@@ -249,9 +259,12 @@ def traffic_of(cfg: gen.Config, path: str):
         return None
 
 
-def roofline_of(cfg: gen.Config, gemm_ms: float, pk, v_count=None):
+def roofline_of(cfg: gen.Config, gemm_ms: float, pk, v_count=None, gemm_ms_min=None, step_ms=None):
     """Roofline of the projection kernel: W streamed once from HBM vs 2*M*d*V flops on the tensor pipe
-    (V = the vocabulary entries this GPU projects)."""
+    (V = the vocabulary entries this GPU projects).  gemm_ms is the kernel's mean duration inside the
+    timed loop (CUDA events around the launch); gemm_ms_min its shortest launch, what the kernel does
+    before the power cap pulls the clock down (the peaks are burst figures of the same kind);
+    step_ms the whole cycle measured in the same pass, for a fraction of the cycle, not of the kernel."""
     V = cfg.V if v_count is None else v_count
     flops = 2.0 * cfg.M * cfg.d * V
     byts = 2.0 * cfg.d * V + 2.0 * cfg.M * cfg.d + 8.0 * cfg.M
@@ -260,36 +273,64 @@ def roofline_of(cfg: gen.Config, gemm_ms: float, pk, v_count=None):
     s = gemm_ms * 1e-3
     if t_hbm >= t_tc:
         a = byts / s / 1e9
-        return {"bound": "hbm", "achieved": a, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": a / pk["hbm_gbs"],
-                "traffic": None, "peak_source": f"of {pk['source']}", "kernel_ms": gemm_ms, "algorithmic_bytes": byts}
-    a = flops / s / 1e12
-    return {"bound": "tensor", "achieved": a, "peak": pk["bf16_tflops"], "unit": "TFLOP/s", "frac": a / pk["bf16_tflops"],
-            "frac_of_sustained_peak": a / pk["bf16_tflops_sustained"], "traffic": None, "peak_source": f"of {pk['source']}",
-            "kernel_ms": gemm_ms, "algorithmic_flops": flops}
+        r = {"bound": "hbm", "achieved": a, "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": a / pk["hbm_gbs"],
+             "traffic": None, "peak_source": f"of {pk['source']}", "kernel_ms": gemm_ms, "algorithmic_bytes": byts}
+    else:
+        a = flops / s / 1e12
+        r = {"bound": "tensor", "achieved": a, "peak": pk["bf16_tflops"], "unit": "TFLOP/s", "frac": a / pk["bf16_tflops"],
+             "frac_of_sustained_peak": a / pk["bf16_tflops_sustained"], "traffic": None, "peak_source": f"of {pk['source']}",
+             "kernel_ms": gemm_ms, "algorithmic_flops": flops}
+    t_roof = max(t_hbm, t_tc)
+    r["roofline_ms"] = t_roof * 1e3
+    if gemm_ms_min:
+        r["kernel_ms_min"] = gemm_ms_min
+        r["frac_shortest_launch"] = t_roof / (gemm_ms_min * 1e-3)
+    if step_ms:
+        r["cycle_ms_same_pass"] = step_ms  # this pass records two events per cycle, which lengthens a cycle a little
+    return r
+
+
+MAX_REGIONS = 200  # --max-regions
 
 
 def bench_one(cfg, device, steps, warmup, barrier, reduce_max, pk, w_copies, W_host=None, with_e2e=True, flags=0, group=None, rule=None):
     wl = GpuWorkload(cfg, device, w_copies, W_host, flags, group, rule)
     try:
-        wl.run(wl.handle, warmup)
         with ClockSampler(device) as cs:
-            ms, t0, t1 = wl.timed(wl.handle, steps, barrier)
-        clocks = cs.summary(t0, t1)
-        ms = reduce_max(ms)
-        # the same loop again with events around the projection kernel (ring of 512 launches)
-        wl.run(wl.handle_t, min(warmup, 8))
-        wl.handle_t.gemm_ms_stats()
-        prof_steps = min(steps, 512)
-        wl.timed(wl.handle_t, prof_steps, barrier)
-        gemm_mean, gemm_min, n = wl.handle_t.gemm_ms_stats()
+            cs.wait_first()
+            wl.run(wl.handle, warmup)
+            # The timed region is exactly `steps` cycles.  A short region (20 cycles of 160 us) ends before
+            # the clock sampler's first tick and is noisy, so it is repeated, every repeat bracketed by its
+            # own events, until about 0.35 s have been timed; the median region is reported.
+            first, t_begin, t_end = wl.timed(wl.handle, steps, barrier)
+            regions = [reduce_max(first)]
+            repeats = int(min(MAX_REGIONS, max(1, -(-350.0 // max(regions[0], 1e-3)))))
+            for _ in range(repeats - 1):
+                ms_r, _, t_end = wl.timed(wl.handle, steps, barrier)
+                regions.append(reduce_max(ms_r))
+            # a second pass of the same loop with events around the projection kernel (ring of 512
+            # launches); the cycle time of THIS pass is reported beside the kernel time, since the event
+            # records lengthen a cycle a little and the two passes are separate measurements
+            wl.run(wl.handle_t, min(warmup, 8))
+            wl.handle_t.gemm_ms_stats()
+            prof_steps = min(max(steps, 64), 512)
+            pass_ms, _, t_end = wl.timed(wl.handle_t, prof_steps, barrier)
+            gemm_mean, gemm_min, n = wl.handle_t.gemm_ms_stats()
+        clocks = cs.summary(t_begin, t_end)
+        ms = statistics.median(regions)
         assert wl.handle.last_status() == wl.aj.AJ_OK and wl.handle_t.last_status() == wl.aj.AJ_OK
         res = {
             "ms_per_step": ms / steps, "clocks": clocks, "path": wl.handle.last_gemm_path(),
-            "roofline": dict(roofline_of(cfg, gemm_mean, pk, wl.v_count), traffic=None if (group is not None or rule) else traffic_of(cfg, wl.handle.last_gemm_path())),
+            "timing": {"regions_of_steps": len(regions), "ms_per_step_min": min(regions) / steps, "ms_per_step_max": max(regions) / steps,
+                       "reported": "median region"},
+            "roofline": dict(roofline_of(cfg, gemm_mean, pk, wl.v_count, gemm_min, pass_ms / prof_steps),
+                             traffic=None if (group is not None or rule) else traffic_of(cfg, wl.handle.last_gemm_path())),
             "gemm_ms_min": gemm_min, "gemm_launches_timed": n,
             "launches_per_step": wl.handle.last_launch_count(),
             "mean_accept_len": float(wl.acc.float().mean().item()),
         }
+        # the whole cycle (both kernels, as timed in the main pass) against the same roofline
+        res["roofline"]["frac_whole_cycle"] = res["roofline"]["roofline_ms"] / res["ms_per_step"]
         if with_e2e:
             s, h2d, d2h = wl.e2e(max(10, min(steps, 300)), 5)
             res["e2e_s_per_step"] = reduce_max(s)
@@ -436,6 +477,8 @@ def main():
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--workload", default="c2", choices=["c2", "c3", "c4", "sweep", "lr_fit"])
+    ap.add_argument("--point", default=None, metavar="BxK", help="one point of the sweep on the 8B shape as the workload, e.g. 8x32")
+    ap.add_argument("--max-regions", type=int, default=200, help="most repeats of the timed region (1 for profiler captures)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-extra", action="store_true", help="skip the batched configurations reported under 'extra'")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline")
@@ -463,9 +506,13 @@ def main():
     group = ajd.Group(info, backend="nccl", device=torch.device(f"cuda:{local}"))
     barrier, reduce_max = group.barrier, group.max_over_ranks
 
+    global MAX_REGIONS
+    MAX_REGIONS = max(1, args.max_regions)
     pk = peaks()
     head = workload("c2" if args.workload == "sweep" else args.workload)
-    default_steps = {"c2": 4000, "c3": 400, "c4": 200}[head.name[:2]]
+    if args.point:
+        head = gen.sweep_config(*map(int, args.point.lower().split("x")))
+    default_steps = {"c2": 4000, "c3": 400, "c4": 200, "c5": max(20, int(0.4 / max(2.0 * head.M * head.d * head.V / 1.2e15, 1.7e-4)))}[head.name[:2]]
     steps = args.steps if args.steps is not None else default_steps
     warmup = max(3, args.warmup if args.warmup is not None else 10)
     copies = args.w_copies or (3 if head.d * head.V * 2 < 1.5e9 else 2)
@@ -488,7 +535,7 @@ def main():
                    "l2": f"W_lm rotates over {copies} copies of {head.d * head.V * 2 / 1e9:.2f} GB each (inputs larger than the 126 MB L2)",
                    "gemm_path": r["path"], "mean_accept_len": r["mean_accept_len"],
                    "rule": rule or "classifier at tau on greedy target tokens"},
-        "clocks": r["clocks"], "roofline": r["roofline"],
+        "clocks": r["clocks"], "roofline": r["roofline"], "timing": r["timing"],
         "gpu_launches": r["launches_per_step"] * steps,
     }
     if "e2e_s_per_step" in r:
@@ -502,8 +549,10 @@ def main():
         todo = []
         if args.workload == "sweep":
             todo = [gen.sweep_config(B, K) for B in gen.SWEEP_B for K in gen.SWEEP_K]
-        elif args.workload == "c2" and not vocab:
-            todo = [gen.C3, gen.C4]
+        elif args.workload == "c2" and not vocab and not args.point:
+            # the batched 8B- and 70B-shaped workloads, and the three points of the sweep around the crossover
+            # from HBM-bound to tensor-bound (264, 520 and 576 rows)
+            todo = [gen.C3, gen.sweep_config(8, 32), gen.sweep_config(8, 64), gen.sweep_config(64, 8), gen.C4]
         for cfg in todo:
             cfg = ajd.rank_config(cfg, rank)
             same_W = cfg.d == head.d and cfg.V == head.V
@@ -512,6 +561,21 @@ def main():
             extra.append({"workload": cfg.name, "B": cfg.B, "K": cfg.K, "d": cfg.d, "V": cfg.V, "steps": n,
                           "ms_per_step": rr["ms_per_step"], "value": cfg.B * cfg.K * world / (rr["ms_per_step"] * 1e-3), "unit": UNIT,
                           "gemm_path": rr["path"], "roofline": rr["roofline"], "clocks": rr["clocks"]})
+    if world > 1 and not vocab and args.workload == "c2" and not args.no_extra:
+        # Strong scaling of the headline workload with the LM head split by vocabulary over the ranks: one batch,
+        # every rank streams 1/N of W_lm, per-row keys exchanged by peer stores inside the kernels.  Recorded
+        # beside the replicas above so that a multi-GPU run exercises the exchange; a failure here is reported,
+        # not fatal (set-up fails on every rank or on none).
+        c2 = gen.C2
+        try:
+            rr = bench_one(c2, local, steps, warmup, barrier, reduce_max, pk, copies, W_host if (c2.d, c2.V, c2.seed) == (head.d, head.V, head.seed) else None,
+                           with_e2e=False, flags=args.flags, group=group, rule=rule)
+            extra.append({"workload": c2.name, "sharding": "vocab", "scaling": "strong", "n_gpus": world, "B": c2.B, "K": c2.K, "steps": steps,
+                          "ms_per_step": rr["ms_per_step"], "value": c2.B * c2.K / (rr["ms_per_step"] * 1e-3), "unit": UNIT,
+                          "gemm_path": rr["path"], "roofline": rr["roofline"], "clocks": rr["clocks"], "timing": rr["timing"],
+                          "parallelism": f"W_lm split by vocabulary over {world} GPUs, one batch, keys exchanged by peer stores inside the kernels"})
+        except Exception as e:  # noqa: BLE001
+            extra.append({"workload": c2.name, "sharding": "vocab", "n_gpus": world, "error": repr(e)[:300]})
     line["extra"] = extra
 
     if rank == 0 and world == 1 and not args.no_cpu:

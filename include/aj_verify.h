@@ -287,7 +287,13 @@ const char *aj_last_gemm_path(aj_handle h);
  * Arguments are those of aj_create and aj_verify together; the device is the CURRENT CUDA device;
  * all pointers are device pointers with the layouts aj_verify documents; optional outputs may be
  * NULL.  dev_status (optional, device, int32) receives 0, or AJ_ERR_TIMEOUT if a bounded wait in a
- * kernel ran out; read it after the stream has finished.
+ * kernel ran out; read it after the stream has finished.  Without it a timeout goes unreported (there
+ * is no handle to ask), so pass it wherever the result matters.
+ * The cycle runs on the same kernels, chosen the same way, as aj_verify runs it on a plain handle: the
+ * one-SM tensor-core kernel up to 128 rows, the two-SM kernel above (AJ_BF16, AJ_W_VD, d % 64 == 0), the
+ * CUDA-core kernel for everything else (AJ_F32, AJ_W_DV, other widths).  The variants a handle can be
+ * switched to (top-K rule, sampling, tree drafts, the folded classifier, vocabulary sharding) need a
+ * handle's workspace and are not offered here.
  *   B * (K + 1) > AJ_STATIC_MAX_ROWS  ->  AJ_ERR_WORKSPACE, nothing enqueued.
  * The first call on each device looks up the array's device address (cudaGetSymbolAddress) and
  * prepares the kernels; make that first call outside any stream capture.  Later calls only enqueue.

@@ -313,7 +313,7 @@ struct PairSched {
     int n_groups;          // row tiles are walked in groups ...
     int g_base, g_rem;     // ... group g holds g_base + (g < g_rem) row tiles
 };
-PairSched pair_schedule(int M, int V, int d, int fold);
+PairSched pair_schedule(int M, int V, int d, int fold, int epi = 0);  // epi: EPI_PLAIN / EPI_COUNT / EPI_SAMPLE
 cudaError_t umma_pair_prepare(int num_sms);
 int umma_pair_max_pairs();
 cudaError_t launch_umma_pair(const GemmArgs &a, const UmmaPlan &p, cudaStream_t stream);

@@ -38,6 +38,7 @@ struct DeviceSetup {
     aj_status error = AJ_OK;
     unsigned char *scratch = nullptr;  // device address of g_static_scratch on this device
     int num_sms = 0;
+    bool pair_ok = false;  // the two-SM kernel can be launched on this device
     EncodeTiledFn encode = nullptr;
 };
 
@@ -77,6 +78,7 @@ const DeviceSetup *setup_current_device(aj_status *st) {
         } else {
             s.scratch = static_cast<unsigned char *>(ptr);
             s.encode = reinterpret_cast<EncodeTiledFn>(fn);
+            s.pair_ok = umma_pair_prepare(s.num_sms) == cudaSuccess && umma_pair_max_pairs() > 0;  // an occupancy query, no allocation
         }
         if (s.error != AJ_OK) cudaGetLastError();
     }
@@ -137,8 +139,18 @@ extern "C" aj_status aj_verify_static(const void *h_target, const void *h_draft,
     g.keys = keys;
     g.status = status;
 
+    // the same choice of projection kernel as aj_verify makes
     cudaError_t e;
-    if (dtype == AJ_BF16 && layout == AJ_W_VD && d % 64 == 0) {
+    if (dtype == AJ_BF16 && layout == AJ_W_VD && d % 64 == 0 && M > 128 && s->pair_ok) {
+        UmmaPlan p;
+        p.bn = 256;
+        const PairSched sc = pair_schedule(M, V, d, 0);
+        if (!encode_rows(s, &p.tmap_w, W_lm, d, V, 128) || !encode_rows(s, &p.tmap_h, h_target, d, M, sc.box_rows)) return AJ_ERR_CUDA;
+        const long long tiles = (long long)sc.n_n * sc.n_v;
+        const int pairs = umma_pair_max_pairs();
+        p.grid = 2 * (int)(tiles < pairs ? tiles : pairs);
+        e = launch_umma_pair(g, p, stream);
+    } else if (dtype == AJ_BF16 && layout == AJ_W_VD && d % 64 == 0) {
         UmmaPlan p;
         p.bn = vm_choose_bn(M);
         if (!encode_rows(s, &p.tmap_w, W_lm, d, V, 128) || !encode_rows(s, &p.tmap_h, h_target, d, M, p.bn)) return AJ_ERR_CUDA;

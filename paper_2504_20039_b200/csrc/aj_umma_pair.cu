@@ -429,13 +429,15 @@ cudaError_t umma_pair_prepare(int num_sms) {
 
 int umma_pair_max_pairs() { return g_max_pairs; }
 
-PairSched pair_schedule(int M, int V, int d, int fold) {
+PairSched pair_schedule(int M, int V, int d, int fold, int epi) {
     PairSched sc;
     sc.fold = fold ? 1 : 0;
     const int units = (M + 15) / 16;  // rows in units of 16 (the UMMA N granule)
     // Wide tiles (up to 512 rows on two accumulators with an issuing warp each) for every batch of more
-    // than 256 rows; up to 256 rows one narrow tile per vocabulary block, double-buffered.
-    sc.dual = units > 16 ? 1 : 0;
+    // than 256 rows; up to 256 rows one narrow tile per vocabulary block, double-buffered.  The epilogue
+    // of a wide tile is not hidden under MMAs; the counting epilogue of the top-K rule is long enough for
+    // narrow tiles to win where a tile is short (d = 4096, 2112 rows: 1.78 vs 2.01 ms; d = 8192: wide).
+    sc.dual = (units > 16 && !(epi == EPI_COUNT && d < 8192 && units > 32)) ? 1 : 0;
     const int cap = sc.dual ? 32 : 16;
     sc.n_n = (units + cap - 1) / cap;
     sc.u_base = units / sc.n_n;
@@ -457,7 +459,8 @@ PairSched pair_schedule(int M, int V, int d, int fold) {
 }
 
 cudaError_t launch_umma_pair(const GemmArgs &a, const UmmaPlan &p, cudaStream_t stream) {
-    const PairSched sc = pair_schedule(a.M, a.V, a.d, a.fold.rows != nullptr);
+    const int epi = a.noise.temperature > 0.0f ? EPI_SAMPLE : a.rank.thr ? EPI_COUNT : EPI_PLAIN;
+    const PairSched sc = pair_schedule(a.M, a.V, a.d, a.fold.rows != nullptr, epi);
     const int stream_w = (sc.n_n == 1) ? 1 : 0;  // W is read by one pair only: do not keep it in L2
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)p.grid);  // 2 CTAs per pair

@@ -63,14 +63,44 @@ class Exchange:
     ranks swap over the process group.  `buffers[r]` is rank r's; pass the list to Handle(shard=...)."""
 
     def __init__(self, group: "Group", max_B: int, max_K: int):
+        """Fails on EVERY rank if it fails on one (a rank that raised alone would leave the others waiting at
+        the next barrier): after each step the ranks vote, and a rank that succeeded undoes its part."""
         from . import binding as aj
 
         self._aj, self.group = aj, group
         rank, world = group.info.rank, group.info.world
-        self.own = aj.shard_exchange_alloc(max_B, max_K, world)
-        handles = group.all_gather_bytes(aj.ipc_export(self.own))
-        self.buffers = [self.own if r == rank else aj.ipc_import(handles[r]) for r in range(world)]
-        group.barrier()  # every rank has mapped every buffer
+        self.own, self.buffers, err, handle = None, [], None, b""
+        try:
+            self.own = aj.shard_exchange_alloc(max_B, max_K, world)
+            handle = aj.ipc_export(self.own)
+        except Exception as e:  # noqa: BLE001 - reported to every rank below
+            err = e
+        handles = group.all_gather_bytes(handle)
+        if not group.all_ok(err is None):
+            self._undo()
+            raise RuntimeError(f"exchange buffer could not be allocated or exported on some rank (this rank: {err!r})")
+        try:
+            self.buffers = [self.own if r == rank else aj.ipc_import(handles[r]) for r in range(world)]
+        except Exception as e:  # noqa: BLE001
+            err = e
+        if not group.all_ok(err is None):  # also: every rank has mapped every buffer
+            self._undo()
+            raise RuntimeError(f"a peer's exchange buffer could not be mapped on some rank (this rank: {err!r})")
+
+    def _undo(self) -> None:
+        for r, p in enumerate(self.buffers):
+            if r != self.group.info.rank and p:
+                try:
+                    self._aj.ipc_close(p)
+                except Exception:  # noqa: BLE001
+                    pass
+        self.buffers = []
+        if self.own:
+            try:
+                self._aj.shard_exchange_free(self.own)
+            except Exception:  # noqa: BLE001
+                pass
+            self.own = None
 
     def ready(self) -> None:
         """Call after every rank has created its handle (which clears its own buffer) and before the first cycle."""
@@ -129,6 +159,10 @@ class Group:
 
     def sum_over_ranks(self, x: float) -> float:
         return self._reduce(x, "SUM")
+
+    def all_ok(self, ok: bool) -> bool:
+        """True iff `ok` is true on every rank (a collective: all ranks get the same answer)."""
+        return self._reduce(1.0 if ok else 0.0, "MIN") > 0.5
 
     def all_gather_bytes(self, payload: bytes):
         """Every rank's `payload`, in rank order (used to exchange IPC handles of exchange buffers)."""

@@ -14,6 +14,37 @@ TOL_P = 1e-4       # |judge probability (device) - (oracle)|
 GAP_EXEMPT = 1e-2  # a row whose top-1/top-2 gap is at most this may legitimately pick the runner-up
 
 
+GUARD_BYTES = 256   # on each side of a guarded tensor
+GUARD_FILL = 0xA5
+
+
+class Guarded:
+    """A device tensor in the middle of a larger allocation whose first and last GUARD_BYTES hold a fixed
+    byte pattern.  Kernels that write a byte before or after a tensor they were given (or scribble over a
+    neighbouring input) change the pattern; check() finds that after the call.  Stands in for a memory
+    checker on the buffers the caller owns."""
+
+    def __init__(self, src, name: str, device="cuda:0"):
+        import torch
+
+        src = src.contiguous()
+        raw = src.view(torch.uint8).reshape(-1) if src.numel() else torch.empty(0, dtype=torch.uint8, device=src.device)
+        self.name = name
+        self.whole = torch.full((2 * GUARD_BYTES + raw.numel(),), GUARD_FILL, dtype=torch.uint8, device=device)
+        self.whole[GUARD_BYTES : GUARD_BYTES + raw.numel()] = raw.to(device)
+        self.t = self.whole[GUARD_BYTES : GUARD_BYTES + raw.numel()].view(src.dtype).reshape(src.shape)
+
+    def check(self):
+        lo, hi = self.whole[:GUARD_BYTES], self.whole[-GUARD_BYTES:]
+        assert bool((lo == GUARD_FILL).all()) and bool((hi == GUARD_FILL).all()), f"bytes next to {self.name} were overwritten"
+
+
+def guarded_full(shape, fill, dtype, name):
+    import torch
+
+    return Guarded(torch.full(shape, fill, dtype=dtype), name)
+
+
 def to_device(a: np.ndarray, dtype: int, device="cuda:0"):
     import torch
 
@@ -46,10 +77,21 @@ class DeviceCase:
         self.cfg = cfg
         self.aj = aj
         self.torch = torch
-        self.W = W if hasattr(W, "data_ptr") else to_device(W, cfg.dtype)
-        self.ht = to_device(ht, cfg.dtype)
-        self.hd = to_device(hd, cfg.dtype)
-        self.w = to_device(w, gen.F32)
+        # inputs copied here sit between guard bands (a full-size LM head that is already on the device is shared
+        # between cases and used as it is)
+        self.guards = []
+
+        def guard(t, name):
+            if t is None:
+                return None
+            g = Guarded(t, name)
+            self.guards.append(g)
+            return g.t
+
+        self.W = W if hasattr(W, "data_ptr") else guard(to_device(W, cfg.dtype, "cpu"), "W_lm")
+        self.ht = guard(to_device(ht, cfg.dtype, "cpu"), "h_target")
+        self.hd = guard(to_device(hd, cfg.dtype, "cpu"), "h_draft")
+        self.w = guard(to_device(w, gen.F32, "cpu"), "judge_w")
         self.extra_row = not (flags & aj.AJ_FLAG_NO_EXTRA_ROW)  # K + 1 rows per sequence, or K
         self.handle = aj.Handle(0, max_B or cfg.B, max_K or cfg.K, cfg.d, cfg.d_draft, cfg.V, cfg.dtype, layout, flags)
 
@@ -60,22 +102,22 @@ class DeviceCase:
         hd = None if self.hd is None else self.hd[seqs]
         B = ht.shape[0] if B is None else B
         K = cfg.K if K is None else K
-        tok_d = torch.from_numpy(np.ascontiguousarray(tok, dtype=np.int32)).cuda()
-        i32 = dict(dtype=torch.int32, device="cuda")
-        f32 = dict(dtype=torch.float32, device="cuda")
         fill_i = -7 if fill is None else fill
-        acc = torch.full((B,), fill_i, **i32)
-        nxt = torch.full((B,), fill_i, **i32)
         R = K + 1 if self.extra_row else K
-        tt = torch.full((B, R), fill_i, **i32)
-        top1 = torch.full((B, R), 12345.0, **f32)
-        jp = torch.full((B, K), 12345.0, **f32)
+        # every output, and the draft tokens, between guard bands; outputs pre-filled with values no call writes
+        gs = [Guarded(torch.from_numpy(np.ascontiguousarray(tok, dtype=np.int32)), "draft_tok"),
+              guarded_full((B,), fill_i, torch.int32, "accept_len"), guarded_full((B,), fill_i, torch.int32, "next_tok"),
+              guarded_full((B, R), fill_i, torch.int32, "target_tok"), guarded_full((B, R), 12345.0, torch.float32, "top1_val"),
+              guarded_full((B, K), 12345.0, torch.float32, "judge_p")]
+        tok_d, acc, nxt, tt, top1, jp = (g.t for g in gs)
         stream = torch.cuda.current_stream().cuda_stream
         self.handle.verify(ht.contiguous(), None if hd is None else hd.contiguous(), self.W, tok_d, self.w,
                            cfg.judge_b if judge_b is None else judge_b, tau, B, K, acc, nxt, tt, top1, jp, stream=stream)
         torch.cuda.synchronize()
         st = self.handle.last_status()
         assert st == self.aj.AJ_OK, self.aj.status_string(st)
+        for g in gs + self.guards:
+            g.check()
         return GpuResult(acc.cpu().numpy(), nxt.cpu().numpy(), tt.cpu().numpy(), top1.cpu().numpy(), jp.cpu().numpy(),
                          self.handle.last_gemm_path(), self.handle.last_launch_count())
 

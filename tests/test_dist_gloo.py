@@ -28,7 +28,33 @@ def _worker(rank, world, port, out):
         handles = g.all_gather_bytes(bytes([rank]) * 64)  # stand-ins for 64-byte IPC handles
         seeds = g.all_gather_bytes(ajd.sampling_seed(77, rank).to_bytes(8, "little"))
         assert len({bytes(s) for s in seeds}) == world and ajd.sampling_seed(77, rank, "vocab") == 77
-        out.put((rank, cfg.seed, float(ht.astype("float64").sum()), slowest, total, [h[0] for h in handles], len(handles[0])))
+        votes = (g.all_ok(True), g.all_ok(rank != 1))       # one rank's failure is every rank's answer
+        # Exchange set-up against a fake of the CUDA calls: rank 1 cannot map rank 0's buffer; both ranks must
+        # raise, and both must give back what they had allocated and mapped
+        from paper_2504_20039_b200 import binding
+
+        log = []
+        binding.shard_exchange_alloc = lambda B, K, w: 1000 + rank
+        binding.shard_exchange_free = lambda p: log.append(("free", p))
+        binding.ipc_export = lambda p: bytes([rank]) * 64
+        binding.ipc_close = lambda p: log.append(("close", p))
+
+        def fake_import(h):
+            if rank == 1:
+                raise RuntimeError("peer mapping refused")
+            return 2000 + h[0]
+
+        binding.ipc_import = fake_import
+        try:
+            ajd.Exchange(g, 4, 8)
+            raised = False
+        except RuntimeError:
+            raised = True
+        binding.ipc_import = lambda h: 2000 + h[0]
+        ex = ajd.Exchange(g, 4, 8)                            # and with every call succeeding it is built
+        built = ex.buffers == ([1000, 2001] if rank == 0 else [2000, 1001])
+        out.put((rank, cfg.seed, float(ht.astype("float64").sum()), slowest, total, [h[0] for h in handles], len(handles[0]),
+                 votes, raised, sorted(log), built))
     finally:
         g.close()
 
@@ -46,7 +72,11 @@ def test_two_ranks_over_gloo():
     for p in procs:
         p.join(timeout=60)
         assert p.exitcode == 0
-    (r0, seed0, sum0, slow0, tot0, hs0, n0), (r1, seed1, sum1, slow1, tot1, hs1, n1) = res
+    (r0, seed0, sum0, slow0, tot0, hs0, n0, *more0), (r1, seed1, sum1, slow1, tot1, hs1, n1, *more1) = res
+    assert more0[0] == more1[0] == (True, False)
+    assert more0[1] and more1[1]                                           # the failure on rank 1 raised on both ranks
+    assert more0[2] == [("close", 2001), ("free", 1000)] and more1[2] == [("free", 1001)]
+    assert more0[3] and more1[3]
     assert (r0, r1) == (0, 1)
     assert seed0 == gen.C1.seed and seed1 != seed0 and sum0 != sum1      # each rank verifies its own sequences
     assert slow0 == slow1 == 11.0                                          # every rank reports the slowest rank's time

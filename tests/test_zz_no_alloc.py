@@ -11,11 +11,12 @@ import aj_inputs as gen
 pytestmark = pytest.mark.gpu
 
 
-def _both(cfg, seed_shift=0):
+def _both(cfg, seed_shift=0, expect_path=None):
     import torch
 
     import paper_2504_20039_b200 as aj
-    from aj_testlib import DeviceCase
+    from aj_testlib import DeviceCase, GpuResult, check_parity
+    from oracle import aj_oracle as orc
 
     cfg = gen.scaled(cfg, seed=cfg.seed + seed_shift)
     W = gen.make_W(cfg)
@@ -23,9 +24,12 @@ def _both(cfg, seed_shift=0):
     w = gen.make_judge(cfg)
     case = DeviceCase(cfg, W, ht, hd, w)
     try:
-        first = case.run(gen.random_draft_tokens(cfg), cfg.tau)      # the device's own greedy tokens ...
-        tok = gen.plant_draft_tokens(cfg, first.target_tok)          # ... give a realistic mix of matches
+        # draft tokens planted against the oracle's greedy tokens: a realistic mix of matches
+        y = np.stack([[orc.argmax(r)[0] for r in orc.logits(ht[b], W, cfg.dtype)] for b in range(cfg.B)])
+        tok = gen.plant_draft_tokens(cfg, y)
         want = case.run(tok, cfg.tau)
+        if expect_path:
+            assert want.path == expect_path  # the kernel aj_verify chose; the static entry point makes the same choice
 
         i32 = dict(dtype=torch.int32, device="cuda")
         f32 = dict(dtype=torch.float32, device="cuda")
@@ -34,11 +38,24 @@ def _both(cfg, seed_shift=0):
         tt = torch.full((cfg.B, cfg.K + 1), -3, **i32)
         top1, jp = torch.full((cfg.B, cfg.K + 1), 7.0, **f32), torch.full((cfg.B, cfg.K), 7.0, **f32)
         status = torch.full((1,), 99, **i32)
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]  # what the driver has left: it counts every allocation of the process
         aj.verify_static(case.ht, case.hd, case.W, tok_d, case.w, cfg.judge_b, cfg.tau, cfg.B, cfg.K, cfg.d, cfg.d_draft,
                          cfg.V, cfg.dtype, aj.AJ_W_VD, acc, nxt, tt, top1, jp, status,
                          stream=torch.cuda.current_stream().cuda_stream)
         torch.cuda.synchronize()
         assert int(status.item()) == 0
+        # one more call, now that the first call on this device has done its set-up: no byte of device memory may go
+        free_mid = torch.cuda.mem_get_info()[0]
+        aj.verify_static(case.ht, case.hd, case.W, tok_d, case.w, cfg.judge_b, cfg.tau, cfg.B, cfg.K, cfg.d, cfg.d_draft,
+                         cfg.V, cfg.dtype, aj.AJ_W_VD, acc, nxt, tt, top1, jp, status,
+                         stream=torch.cuda.current_stream().cuda_stream)
+        torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info()[0] == free_mid and free_mid <= free_before
+        assert int(status.item()) == 0
+        # against the oracle, under the tolerances of every other parity test
+        got = GpuResult(acc.cpu().numpy(), nxt.cpu().numpy(), tt.cpu().numpy(), top1.cpu().numpy(), jp.cpu().numpy(), want.path, 2)
+        check_parity(orc.verify(ht, hd, W, tok, w, cfg.judge_b, cfg.tau, cfg.dtype), got, tok, cfg.tau)
         np.testing.assert_array_equal(tt.cpu().numpy(), want.target_tok)
         np.testing.assert_array_equal(acc.cpu().numpy(), want.accept_len)
         np.testing.assert_array_equal(nxt.cpu().numpy(), want.next_tok)
@@ -53,9 +70,11 @@ def test_static_scratch_entry_point_matches_handle_entry_point_twice():
     # call's keys in the shared array and must not be disturbed by them
     big = gen.Config("static_a", B=5, K=40, d=512, d_draft=256, V=5000, sigma_W=0.2, sigma_w=0.05, match_lo=0.5, match_hi=0.9, seed=30)
     small = gen.Config("static_b", B=2, K=9, d=256, d_draft=128, V=3001, sigma_W=0.2, sigma_w=0.05, match_lo=0.5, match_hi=0.9, seed=31)
-    _both(big)
-    _both(small)
-    _both(gen.scaled(small, dtype=gen.F32, d=200, d_draft=72))  # the CUDA-core kernel shares the same scratch
+    _both(big, expect_path="umma_pair_256x256")   # 205 rows: the two-SM kernel, as aj_verify chooses
+    _both(small, expect_path="umma_vm_128x32")
+    _both(gen.scaled(small, dtype=gen.F32, d=200, d_draft=72), expect_path="simt")  # the CUDA-core kernel shares the same scratch
+    wide = gen.Config("static_c", B=9, K=40, d=256, d_draft=128, V=3000, sigma_W=0.2, sigma_w=0.05, match_lo=0.5, match_hi=0.9, seed=32)
+    _both(wide, expect_path="umma_pair_256x256")  # 369 rows: wide tiles on two accumulators
 
 
 def test_static_scratch_entry_point_rejects_what_does_not_fit():

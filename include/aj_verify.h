@@ -206,13 +206,18 @@ aj_status aj_verify_tree(aj_handle h, const void *h_target, const void *h_draft,
  *           {the largest absolute component of the gradient of f at the result, the milliseconds the
  *           evaluations' loss + gradient kernel took in total (CUDA events)}.
  * Stops when that component is <= tol, after max_iter iterations, or when no step lowers f any more
- * (evaluations are fp32 per row, fp64 across rows).  Synchronous; allocates and frees its own workspace
- * ((SMs + 2) * F floats).  Errors: AJ_ERR_INVALID_ARG, AJ_ERR_UNSUPPORTED (alignment, or rows wider than
- * 48 KB: 24 576 features in bf16, 12 288 in fp32), AJ_ERR_NOT_SM100, AJ_ERR_CUDA.
+ * (evaluations are fp32 per row, fp64 across rows).  Synchronous.  The first fit on a device allocates a
+ * workspace ((SMs + 2) * F floats of device memory, 2 * F floats of pinned host memory) that later fits on
+ * that device reuse (it grows if a later fit needs more); aj_lr_release frees it.  Fits in one process
+ * take turns.  Errors: AJ_ERR_INVALID_ARG, AJ_ERR_UNSUPPORTED (alignment, or rows wider than 48 KB: 24 576
+ * features in bf16, 12 288 in fp32), AJ_ERR_NOT_SM100, AJ_ERR_CUDA.
  */
 aj_status aj_lr_fit(int device, const void *X, const uint8_t *labels, long long n, int F, aj_dtype dtype, float C,
                     int max_iter, float tol, float *w_out, float *b_out, int *iters_out, float *stats_out,
                     void *cuda_stream);
+
+/* Free the workspace aj_lr_fit keeps on `device` (-1: on every device).  Errors: AJ_ERR_INVALID_ARG, AJ_ERR_CUDA. */
+aj_status aj_lr_release(int device);
 
 /*
  * The same cycle for a caller whose per-cycle tensors live in host memory: h_target, h_draft and

@@ -21,7 +21,7 @@ EXPORTS = (
     "aj_create", "aj_verify", "aj_verify_host", "aj_last_status", "aj_last_gemm_ms", "aj_gemm_ms_stats", "aj_last_launch_count",
     "aj_last_gemm_path", "aj_pair_schedule", "aj_destroy", "aj_set_top_k", "aj_set_sampling", "aj_verify_tree", "aj_lr_fit", "aj_shard_exchange_bytes", "aj_shard_exchange_alloc", "aj_shard_exchange_free", "aj_shard_range", "aj_create_sharded",
     "aj_shard_project", "aj_shard_finish", "aj_ipc_export", "aj_ipc_import", "aj_ipc_close", "aj_status_string", "aj_version", "aj_verify_static",
-    "aj_fuse_judge",
+    "aj_fuse_judge", "aj_lr_release",
 )
 
 _lib = None
@@ -93,6 +93,8 @@ def lib() -> ctypes.CDLL:
         L.aj_ipc_import.restype = ci
         L.aj_ipc_close.argtypes = [vp]
         L.aj_ipc_close.restype = ci
+        L.aj_lr_release.argtypes = [ci]
+        L.aj_lr_release.restype = ci
         L.aj_fuse_judge.argtypes = [vp, vp, vp]
         L.aj_fuse_judge.restype = ci
         L.aj_set_top_k.argtypes = [vp, ci]
@@ -118,6 +120,11 @@ def lr_fit(device: int, X, labels, n: int, F: int, dtype: int, C: float, w_out, 
         raise AjError(st, "aj_lr_fit")
     lr_fit.kernel_ms = stats[1]
     return st, b.value, it[0], it[1], stats[0]
+
+
+def lr_release(device: int = -1) -> int:
+    """aj_lr_release: free the workspace aj_lr_fit keeps between fits."""
+    return lib().aj_lr_release(device)
 
 
 def status_string(status: int) -> str:

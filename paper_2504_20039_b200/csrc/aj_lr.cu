@@ -17,6 +17,7 @@
 #include <math.h>
 #include <stdint.h>
 
+#include <mutex>
 #include <type_traits>
 #include <vector>
 
@@ -208,9 +209,13 @@ __global__ void lr_reduce_kernel(const float *__restrict__ partial_g, int parts,
     g[f] = s;
 }
 
-// One device allocation and one pinned host allocation per fit, carved into the pieces below.
+// One device allocation and one pinned host allocation, carved into the pieces below.  A device's
+// workspace is kept between fits (allocating and freeing the pinned and device memory took longer than
+// the fit's kernels) and grows when a fit needs more; aj_lr_release gives it back.
 struct Workspace {
     char *dev = nullptr, *host = nullptr;
+    size_t dev_bytes = 0, host_bytes = 0;
+    cudaEvent_t ev0 = nullptr, ev1 = nullptr;
     size_t head_bytes = 0;         // partial losses, w and the gradient: the part mirrored on the host
     double *partial_ld = nullptr;  // device [2 * grid]: losses, then intercept gradients
     float *w_dev = nullptr, *g_dev = nullptr, *partial_g = nullptr;
@@ -219,8 +224,19 @@ struct Workspace {
     bool alloc(int F, int grid) {
         const size_t ld = (2 * (size_t)grid * sizeof(double) + 255) & ~(size_t)255;  // every piece starts on a 256-byte boundary
         const size_t vec = ((size_t)F * sizeof(float) + 255) & ~(size_t)255;
-        if (cudaMalloc(&dev, ld + 2 * vec + (size_t)grid * F * sizeof(float)) != cudaSuccess) return false;
-        if (cudaMallocHost(&host, ld + 2 * vec) != cudaSuccess) return false;
+        const size_t need_dev = ld + 2 * vec + (size_t)grid * F * sizeof(float), need_host = ld + 2 * vec;
+        if (need_dev > dev_bytes || need_host > host_bytes) {
+            release();
+            if (cudaMalloc(&dev, need_dev) != cudaSuccess || cudaMallocHost(&host, need_host) != cudaSuccess) {
+                release();
+                return false;
+            }
+            dev_bytes = need_dev, host_bytes = need_host;
+        }
+        if (!ev0 && (cudaEventCreate(&ev0) != cudaSuccess || cudaEventCreate(&ev1) != cudaSuccess)) {
+            release();
+            return false;
+        }
         head_bytes = ld + 2 * vec;
         partial_ld = reinterpret_cast<double *>(dev);
         w_dev = reinterpret_cast<float *>(dev + ld);
@@ -231,11 +247,20 @@ struct Workspace {
         g_host = reinterpret_cast<float *>(reinterpret_cast<char *>(w_host) + vec);
         return true;
     }
-    ~Workspace() {
-        cudaFree(dev);
-        cudaFreeHost(host);
+    void release() {
+        if (dev) cudaFree(dev);
+        if (host) cudaFreeHost(host);
+        if (ev0) cudaEventDestroy(ev0);
+        if (ev1) cudaEventDestroy(ev1);
+        dev = host = nullptr;
+        ev0 = ev1 = nullptr;
+        dev_bytes = host_bytes = 0;
     }
 };
+
+constexpr int LR_MAX_DEVICES = 64;
+std::mutex g_lr_mutex;  // a fit holds it from start to end: fits in one process take turns
+Workspace g_lr_ws[LR_MAX_DEVICES];
 
 }  // namespace
 
@@ -270,6 +295,7 @@ extern "C" aj_status aj_lr_fit(int device, const void *X, const uint8_t *labels,
         cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess)
         return AJ_ERR_CUDA;
     if (cc_major != 10) return AJ_ERR_NOT_SM100;
+    if (device >= LR_MAX_DEVICES) return AJ_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     using Kernel = void (*)(const LrArgs);
     auto pick_g = [&](auto bf, auto cp) -> Kernel {
@@ -298,7 +324,8 @@ extern "C" aj_status aj_lr_fit(int device, const void *X, const uint8_t *labels,
     const long long want = (n + groups - 1) / groups;  // CTAs that would have a row for every group
     const int grid = (int)(want < num_sms ? want : num_sms);
 
-    Workspace ws;
+    std::lock_guard<std::mutex> lock(g_lr_mutex);
+    Workspace &ws = g_lr_ws[device];
     if (!ws.alloc(F, grid)) {
         cudaGetLastError();
         return AJ_ERR_CUDA;
@@ -306,15 +333,7 @@ extern "C" aj_status aj_lr_fit(int device, const void *X, const uint8_t *labels,
 
     const int D = F + 1;  // the intercept is the last coordinate
     bool cuda_ok = true;
-    cudaEvent_t ev0 = nullptr, ev1 = nullptr;
-    if (cudaEventCreate(&ev0) != cudaSuccess || cudaEventCreate(&ev1) != cudaSuccess) return AJ_ERR_CUDA;
-    struct Events {
-        cudaEvent_t a, b;
-        ~Events() {
-            cudaEventDestroy(a);
-            cudaEventDestroy(b);
-        }
-    } events{ev0, ev1};
+    cudaEvent_t ev0 = ws.ev0, ev1 = ws.ev1;
     double kernel_ms = 0.0;
     // f and its gradient at v (fp64 on the host, w rounded to fp32 for the device)
     auto eval = [&](const std::vector<double> &v, std::vector<double> &grad) -> double {
@@ -447,5 +466,23 @@ extern "C" aj_status aj_lr_fit(int device, const void *X, const uint8_t *labels,
         stats_out[0] = (float)max_abs(g);
         stats_out[1] = (float)kernel_ms;
     }
+    return AJ_OK;
+}
+
+extern "C" aj_status aj_lr_release(int device) {
+    using namespace aj;
+    if (device >= LR_MAX_DEVICES) return AJ_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(g_lr_mutex);
+    int prev = 0;
+    if (cudaGetDevice(&prev) != cudaSuccess) return AJ_ERR_CUDA;
+    for (int dev = 0; dev < LR_MAX_DEVICES; dev++) {
+        if ((device >= 0 && dev != device) || (!g_lr_ws[dev].dev && !g_lr_ws[dev].ev0)) continue;
+        if (cudaSetDevice(dev) != cudaSuccess) {
+            cudaGetLastError();
+            continue;
+        }
+        g_lr_ws[dev].release();
+    }
+    cudaSetDevice(prev);
     return AJ_OK;
 }

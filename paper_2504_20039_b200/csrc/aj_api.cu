@@ -505,18 +505,20 @@ aj_status aj_verify_host(aj_handle h, const void *h_target_host, const void *h_d
     if (!guard.ok()) return AJ_ERR_CUDA;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const size_t M = (size_t)B * rows_per_seq(h, K), esz = elem_size(h->dtype);
+    // The hidden states are always copied (the projection kernel reads them a thousand times over), and
+    // their copies are enqueued first: everything the host does next runs while they are on their way.
+    bool ok = cudaMemcpyAsync(h->st_ht, h_target_host, M * d * esz, cudaMemcpyHostToDevice, stream) == cudaSuccess &&
+              (h->d_draft == 0 ||
+               cudaMemcpyAsync(h->st_hd, h_draft_host, M * h->d_draft * esz, cudaMemcpyHostToDevice, stream) == cudaSuccess);
+    if (!ok) return AJ_ERR_CUDA;
     // Small host buffers that are pinned (and therefore mapped into the device's address space) are
     // used in place by the judge kernel: it reads the draft tokens and writes the results over PCIe,
-    // which saves three copy operations per cycle.  The hidden states are always copied: the
-    // projection kernel reads them a thousand times over.
+    // which saves three copy operations per cycle.
     int32_t *tok_dev = static_cast<int32_t *>(device_view(draft_tok_host));
     int32_t *acc_dev = static_cast<int32_t *>(device_view(accept_len_host));
     int32_t *next_dev = static_cast<int32_t *>(device_view(next_tok_host));
     int32_t *tt_dev = target_tok_host ? static_cast<int32_t *>(device_view(target_tok_host)) : nullptr;
-    bool ok = cudaMemcpyAsync(h->st_ht, h_target_host, M * d * esz, cudaMemcpyHostToDevice, stream) == cudaSuccess &&
-              (h->d_draft == 0 ||
-               cudaMemcpyAsync(h->st_hd, h_draft_host, M * h->d_draft * esz, cudaMemcpyHostToDevice, stream) == cudaSuccess) &&
-              (tok_dev || cudaMemcpyAsync(h->st_tok, draft_tok_host, (size_t)B * K * 4, cudaMemcpyHostToDevice, stream) == cudaSuccess);
+    ok = tok_dev || cudaMemcpyAsync(h->st_tok, draft_tok_host, (size_t)B * K * 4, cudaMemcpyHostToDevice, stream) == cudaSuccess;
     if (!ok) return AJ_ERR_CUDA;
     st = aj_verify(h, h->st_ht, h->d_draft ? h->st_hd : nullptr, W_lm, tok_dev ? tok_dev : h->st_tok, judge_w, judge_b, tau, B, K,
                    d, V, acc_dev ? acc_dev : h->st_acc, next_dev ? next_dev : h->st_next,

@@ -259,7 +259,7 @@ def traffic_of(cfg: gen.Config, path: str):
         return None
 
 
-def roofline_of(cfg: gen.Config, gemm_ms: float, pk, v_count=None, gemm_ms_min=None, step_ms=None):
+def roofline_of(cfg: gen.Config, gemm_ms: float, pk, v_count=None, gemm_ms_min=None, step_ms=None, alone_ms=None):
     """Roofline of the projection kernel: W streamed once from HBM vs 2*M*d*V flops on the tensor pipe
     (V = the vocabulary entries this GPU projects).  gemm_ms is the kernel's mean duration inside the
     timed loop (CUDA events around the launch); gemm_ms_min its shortest launch, what the kernel does
@@ -285,6 +285,9 @@ def roofline_of(cfg: gen.Config, gemm_ms: float, pk, v_count=None, gemm_ms_min=N
     if gemm_ms_min:
         r["kernel_ms_min"] = gemm_ms_min
         r["frac_shortest_launch"] = t_roof / (gemm_ms_min * 1e-3)
+    if alone_ms:
+        r["kernel_ms_alone"] = alone_ms  # best of 10 single launches after 50 ms of idle: comparable with the burst peak
+        r["frac_alone"] = t_roof / (alone_ms * 1e-3)
     if step_ms:
         r["cycle_ms_same_pass"] = step_ms  # this pass records two events per cycle, which lengthens a cycle a little
     return r
@@ -317,13 +320,24 @@ def bench_one(cfg, device, steps, warmup, barrier, reduce_max, pk, w_copies, W_h
             pass_ms, _, t_end = wl.timed(wl.handle_t, prof_steps, barrier)
             gemm_mean, gemm_min, n = wl.handle_t.gemm_ms_stats()
         clocks = cs.summary(t_begin, t_end)
+        # the kernel timed alone, the way the burst peak it is compared with was taken (best of 10 single
+        # launches, the GPU left idle for 50 ms before each so that the clock is not held down by the power cap)
+        burst = []
+        for i in range(10):
+            torch_sync = wl.torch.cuda.synchronize
+            torch_sync()
+            time.sleep(0.05)
+            wl.step(wl.handle_t, i)
+            torch_sync()
+            burst.append(wl.handle_t.last_gemm_ms())
+        wl.handle_t.gemm_ms_stats()
         ms = statistics.median(regions)
         assert wl.handle.last_status() == wl.aj.AJ_OK and wl.handle_t.last_status() == wl.aj.AJ_OK
         res = {
             "ms_per_step": ms / steps, "clocks": clocks, "path": wl.handle.last_gemm_path(),
             "timing": {"regions_of_steps": len(regions), "ms_per_step_min": min(regions) / steps, "ms_per_step_max": max(regions) / steps,
                        "reported": "median region"},
-            "roofline": dict(roofline_of(cfg, gemm_mean, pk, wl.v_count, gemm_min, pass_ms / prof_steps),
+            "roofline": dict(roofline_of(cfg, gemm_mean, pk, wl.v_count, gemm_min, pass_ms / prof_steps, min(burst)),
                              traffic=None if (group is not None or rule) else traffic_of(cfg, wl.handle.last_gemm_path())),
             "gemm_ms_min": gemm_min, "gemm_launches_timed": n,
             "launches_per_step": wl.handle.last_launch_count(),

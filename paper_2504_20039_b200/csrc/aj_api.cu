@@ -338,6 +338,7 @@ static aj_status enqueue_project(aj_handle h, const void *h_target, const void *
     g.w_layout = h->layout;
     g.keys = h->keys;
     g.status = h->status;
+    g.sched = reinterpret_cast<unsigned *>(h->status) + 32;  // zeroed with the status block; the kernel leaves it zero
     const bool fold = h->fold && h->umma_ok && h->top_k == 0;  // the top-K rule does not consult the classifier
     if (fold) {
         g.fold.rows = h->fold_rows;

@@ -277,6 +277,10 @@ struct GemmArgs {
     RankArgs rank;       // thr != nullptr: also count, per row, the entries that outrank the draft token
     Noise noise;         // temperature > 0: the argmax is taken over logit + temperature * Gumbel noise
     JudgeFold fold;      // rows != nullptr: one more vocabulary block computes the classifier's target half
+    // Two words, zero between launches, through which the CTA pairs of the two-SM kernel share out their
+    // tiles as they become free (a tile counter and a count of the pairs that are done with it);
+    // nullptr: every pair takes the tiles pair, pair + pairs, ... in a fixed order.
+    unsigned *sched = nullptr;
 };
 
 // What a projection kernel's epilogue does besides the argmax.

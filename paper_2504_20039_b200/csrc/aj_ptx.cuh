@@ -193,6 +193,38 @@ __device__ inline void mbar_arrive_cluster(uint32_t cluster_bar) {
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar) : "memory");
 }
 
+// The waiting side of a hand-over of ordinary data between the two CTAs: what the arriving thread
+// wrote (to either CTA's shared memory) before its release-arrive is visible after this wait.
+__device__ inline bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ inline bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+    if (mbar_try_wait_cluster(bar, parity)) return true;
+    unsigned long long t0 = 0;
+    for (uint32_t spin = 1;; ++spin) {
+        if (mbar_try_wait_cluster(bar, parity)) return true;
+        if ((spin & 0xFF) == 0) {
+            if (*abort_flag) return false;
+            const unsigned long long now = globaltimer_ns();
+            if (t0 == 0)
+                t0 = now;
+            else if (now - t0 > WAIT_LIMIT_NS)
+                return false;
+        }
+    }
+}
+__device__ inline void st_shared_cluster_u32(uint32_t cluster_addr, uint32_t value) {
+    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(cluster_addr), "r"(value) : "memory");
+}
+
 // 2-D tiled TMA load into THIS CTA's shared memory whose completion bytes are counted on an
 // mbarrier given by its cluster-wide address (the leader's barrier).  No multicast: every CTA
 // fetches its own half-tiles.

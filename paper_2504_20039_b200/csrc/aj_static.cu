@@ -138,6 +138,8 @@ extern "C" aj_status aj_verify_static(const void *h_target, const void *h_draft,
     g.w_layout = layout;
     g.keys = keys;
     g.status = status;
+    // the tile counter of the two-SM kernel: zero when the library is loaded, put back to zero by every launch
+    g.sched = reinterpret_cast<unsigned *>(s->scratch + (size_t)STATIC_MAX_ROWS * 8) + 32;
 
     // the same choice of projection kernel as aj_verify makes
     cudaError_t e;

@@ -7,9 +7,16 @@
 // A tile is 256 vocabulary entries (UMMA M = 256, 128 per SM = the 128 TMEM lanes of each SM) by a
 // block of rows of hidden states (UMMA N, any multiple of 16).  The rows are cut into the fewest
 // tiles and spread over them evenly in units of 16 rows, so no tensor work is spent on padding and
-// all tiles take nearly the same time, which keeps the pairs that share a block of W in step and
-// that block in L2.  When h_target outgrows L2 the row tiles are walked in groups, each group
-// against the whole vocabulary.
+// all tiles take nearly the same time.  When h_target outgrows L2 the row tiles are walked in groups,
+// each group against the whole vocabulary.
+//
+// Tiles are numbered so that consecutive tiles share a block of W, and the pairs take them in that
+// order from a counter in global memory as they become free.  A fixed assignment (pair p takes tiles
+// p, p + pairs, ...) loses the sharing: SM pairs do not run at one speed (measured on one GPU: some
+// pairs, the same ones in every launch, take 3 % longer per tile), after thirty tiles neighbouring
+// pairs are a whole tile apart, and a block of W has left L2 before its last reader asks for it.  With
+// the counter the readers of a block start within microseconds of one another at every point of the
+// launch, W can be marked evict-first, h_target stays in L2, and a slower pair simply takes fewer tiles.
 //
 // Two forms (512 columns of tensor memory either way):
 //   narrow tiles (DUAL = false, batches of at most 256 rows): one accumulator of up to 256 columns in
@@ -34,7 +41,9 @@
 // tiled TMA loads, and the follower's loads report their bytes to the leader's barrier.
 //
 // Roles in each CTA:
-//   warp 0      TMA producer (one thread): waits for its own stage to be free, then loads
+//   warp 0      TMA producer (one thread).  The leader's draws the pair's next tile from the counter and
+//               announces it, through a small ring of slots in shared memory with their own barriers,
+//               to every other warp of both CTAs (-1: no more tiles).  Both wait for a free stage and load
 //               W[v0 + 128*rank .. +128, kb] and, per accumulator a, h[row0[a] + (N[a]/2)*rank .. , kb];
 //   warp 1, 2   warp 1 allocates tensor memory (both CTAs); in the leader one thread of each issues
 //               the MMAs of accumulator 0 / 1 (warp 2 only for wide tiles) and commits stage-release
@@ -70,7 +79,8 @@ constexpr int A_BYTES = BV_CTA * BK * 2;   // 16 KB: this CTA's 128 rows of W, o
 constexpr int RING_BYTES = 224 * 1024;     // shared memory given to the stage ring (the SM has 227 KB per CTA)
 constexpr int MAX_STAGES = 8;
 constexpr int TMEM_COLS = 2 * BN;
-constexpr int BAR_BYTES = 8 * (2 * MAX_STAGES + 8) + 16;
+constexpr int SCHED_SLOTS = 4;  // tiles a pair may have announced to its warps and not yet retired
+constexpr int BAR_BYTES = 8 * (2 * MAX_STAGES + 8) + 16 + 8 * 2 * SCHED_SLOTS + 4 * SCHED_SLOTS;
 constexpr int SMEM_BYTES = RING_BYTES + BAR_BYTES + 1024;
 
 struct Tile {
@@ -83,11 +93,11 @@ struct Tile {
 };
 
 // Tile t of the schedule.  Row tiles come in groups; a group is walked against every vocabulary
-// block (row tile fastest) before the next group starts.  Consecutive tiles, which run on
-// neighbouring pairs at the same time, share a block of W.  Which row tile of the group a pair gets
-// rotates with the vocabulary block, so that pairs whose number is a multiple of the group size
-// apart do not always get the larger (or the smaller) row tiles and drift away from the pairs they
-// share W with.  A wide tile's units of 16 rows are split over the two accumulators, the larger half first.
+// block (row tile fastest) before the next group starts.  Consecutive tiles, which are taken at
+// nearly the same time, share a block of W.  Which row tile of the group comes first rotates with the
+// vocabulary block (with a fixed assignment of tiles to pairs this keeps a pair from always getting the
+// larger, or the smaller, row tiles).  A wide tile's units of 16 rows are split over the two accumulators,
+// the larger half first.
 __device__ inline Tile decode_tile(const PairSched &sc, int t) {
     int g = 0, start = 0, sz = sc.g_base + (0 < sc.g_rem ? 1 : 0);
     while (g + 1 < sc.n_groups && t >= start + sz * sc.n_v) {
@@ -118,7 +128,7 @@ __global__ void __launch_bounds__(num_threads(DUAL), 1)
 umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_h,
                  const __grid_constant__ CUtensorMap tmap_j, int M, int V, int d, PairSched sc, int stream_w, int v_offset,
                  unsigned long long *__restrict__ keys, int *__restrict__ status, const Publish pub, const RankArgs rk,
-                 const Noise nz, float *__restrict__ fold_parts, int fold_stride) {
+                 const Noise nz, float *__restrict__ fold_parts, int fold_stride, unsigned *__restrict__ sched) {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;  // the same offset in both CTAs: one descriptor serves both
@@ -131,6 +141,12 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
     auto acc_empty_bar = [&](int a) { return bar_base + 8u * (2 * MAX_STAGES + 4 + a); };      // used in the leader only
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem + RING_BYTES + 8 * (2 * MAX_STAGES + 8));
     volatile int *abort_flag = reinterpret_cast<volatile int *>(tmem_slot + 1);
+    // The tiles of this pair, announced one by one by the leader's producer to every warp of both CTAs.
+    const uint32_t sched_base = bar_base + 8u * (2 * MAX_STAGES + 8) + 16u;
+    auto sched_full_bar = [&](int i) { return sched_base + 8u * i; };                   // one in each CTA
+    auto sched_empty_bar = [&](int i) { return sched_base + 8u * (SCHED_SLOTS + i); };  // used in the leader only
+    auto sched_tile_addr = [&](int i) { return sched_base + 8u * (2 * SCHED_SLOTS) + 4u * i; };
+    volatile int *sched_tile = reinterpret_cast<volatile int *>(smem + RING_BYTES + 8 * (2 * MAX_STAGES + 8) + 16 + 8 * 2 * SCHED_SLOTS);
 
     const int warp = threadIdx.x >> 5;  // warp-uniform
     const int lane = threadIdx.x & 31;
@@ -155,6 +171,11 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
             mbar_init(acc_full_bar(a), 1);   // the accumulator's issuing thread
             mbar_init(acc_empty_bar(a), 8);  // the four warps that drain it, in both CTAs
         }
+        for (int i = 0; i < SCHED_SLOTS; i++) {
+            mbar_init(sched_full_bar(i), 1);  // the leader's producer
+            // every reader of the slot: the issuing threads and the follower's producer, and the epilogue warps of both CTAs
+            mbar_init(sched_empty_bar(i), (DUAL ? 2 : 1) * 9 + 1);
+        }
         *abort_flag = 0;
         fence_barrier_init();
     }
@@ -177,6 +198,13 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
     auto acc_id = [&](int it, int a) { return DUAL ? a : (it & 1); };
     auto acc_col = [&](int it, int a) { return (uint32_t)(acc_id(it, a) * BN); };
     auto acc_phase = [&](int it) { return (uint32_t)(DUAL ? it : (it >> 1)) & 1u; };
+    // A reader's side of the tile announcements: the it-th tile of this pair, -1 after the last one
+    // (or when the wait ran out); the slot is given back once the caller's warp has read it.
+    auto announced_tile = [&](int it) {
+        const int slot = it & (SCHED_SLOTS - 1);
+        return mbar_wait_cluster(sched_full_bar(slot), (uint32_t)(it / SCHED_SLOTS) & 1u, abort_flag) ? sched_tile[slot] : -2;
+    };
+    auto retire_slot = [&](int it) { mbar_arrive_cluster(map_to_cta(sched_empty_bar(it & (SCHED_SLOTS - 1)), 0)); };
 
     if (warp == 0) {
         if (lane == 0) {
@@ -186,14 +214,43 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
             int s = 0;
             uint32_t ph = 0;
             bool ok = true;
-            for (int t = pair; ok && t < num_tiles; t += num_pairs) {
+            // The leader's producer decides which tile comes next.  With a tile counter the pairs take
+            // tiles in order as they become free: the tiles that share a block of W are then taken within
+            // a short time of one another however far the pairs have drifted apart (some SM pairs run a
+            // few percent slower than others), and a slower pair ends up with fewer tiles.  The first
+            // tile of a pair is its own number; the counter hands out the rest.  The next tile is
+            // asked for some k-blocks before the current one has been loaded, so that the answer is
+            // there when it is needed.
+            const int kb_ask = num_kb > 16 ? num_kb - 16 : 0;
+            int t = pair < num_tiles ? pair : -1;
+            for (int it = 0; ok; ++it) {
+                const int slot = it & (SCHED_SLOTS - 1);
+                if (rank == 0) {
+                    if (it >= SCHED_SLOTS &&
+                        !mbar_wait_cluster(sched_empty_bar(slot), (uint32_t)(it / SCHED_SLOTS - 1) & 1u, abort_flag)) {
+                        give_up();
+                        t = -1;  // still announced below: the other warps must not wait for a tile that never comes
+                    }
+                    sched_tile[slot] = t;
+                    st_shared_cluster_u32(map_to_cta(sched_tile_addr(slot), 1), (uint32_t)t);
+                    mbar_arrive_cluster(map_to_cta(sched_full_bar(slot), 0));
+                    mbar_arrive_cluster(map_to_cta(sched_full_bar(slot), 1));
+                } else {
+                    t = announced_tile(it);
+                    if (t == -2) give_up();
+                    retire_slot(it);
+                }
+                if (t < 0) break;
                 const Tile tl = decode_tile(sc, t);
                 const bool fold = tl.v_tile == fold_tile;
                 const CUtensorMap *tw = fold ? &tmap_j : &tmap_w;  // the classifier rows start at entry 0 of their own map
                 const int w_row = (fold ? 0 : tl.v_tile * BV) + (int)rank * BV_CTA;
                 const int h_row0 = tl.row0[0] + (int)rank * (tl.n_inst[0] >> 1);
                 const int h_row1 = tl.row0[1] + (int)rank * (tl.n_inst[1] >> 1);
+                int next = -1;
                 for (int kb = 0; kb < num_kb; kb++) {
+                    // (the answer is not looked at before the loop ends: the thread does not wait for it here)
+                    if (rank == 0 && kb == kb_ask) next = sched ? (int)atomicAdd(sched, 1u) + num_pairs : t + num_pairs;
                     if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) {
                         give_up();
                         ok = false;
@@ -215,6 +272,15 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
                         ph ^= 1u;
                     }
                 }
+                t = next < num_tiles ? next : -1;
+            }
+            if (rank == 0) {
+                // The pair that leaves last puts the counter back to zero for the next launch; each pair has
+                // drawn its last number from it before it is counted here.
+                if (sched) {
+                    __threadfence();
+                    if (atomicInc(sched + 1, (unsigned)num_pairs - 1u) == (unsigned)num_pairs - 1u) atomicExch(sched, 0u);
+                }
             }
         }
     } else if (warp <= 2) {
@@ -229,8 +295,11 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
             int s = 0;
             uint32_t ph = 0;
             bool ok = true;
-            int it = 0;
-            for (int t = pair; ok && t < num_tiles; t += num_pairs, ++it) {
+            for (int it = 0; ok; ++it) {
+                const int t = announced_tile(it);
+                if (t == -2) give_up();
+                retire_slot(it);
+                if (t < 0) break;
                 const Tile tl = decode_tile(sc, t);
                 const int n_inst = tl.rows(a);  // 0: this accumulator has no rows in this tile (one unit of 16); the barriers still turn
                 const uint32_t idesc = instr_desc(BV, n_inst) | a_major;
@@ -289,8 +358,15 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
         // All of the accumulator's keys are fetched before it is ready, so no chunk waits for an L2
         // round trip.  The chunk loop is kept rolled, one copy of its code stays in the instruction
         // cache: the keys rotate through kk[0].
-        int it = 0;
-        for (int t = pair; t < num_tiles; t += num_pairs, ++it) {
+        for (int it = 0;; ++it) {
+            int t = announced_tile(it);
+            if (__any_sync(0xffffffffu, t == -2)) {  // the whole warp takes one decision
+                give_up();
+                t = -2;
+            }
+            __syncwarp();
+            if (lane == 0) retire_slot(it);
+            if (t < 0) break;
             const Tile tl = decode_tile(sc, t);
             uint32_t kk[CH];
 #pragma unroll
@@ -461,7 +537,11 @@ PairSched pair_schedule(int M, int V, int d, int fold, int epi) {
 cudaError_t launch_umma_pair(const GemmArgs &a, const UmmaPlan &p, cudaStream_t stream) {
     const int epi = a.noise.temperature > 0.0f ? EPI_SAMPLE : a.rank.thr ? EPI_COUNT : EPI_PLAIN;
     const PairSched sc = pair_schedule(a.M, a.V, a.d, a.fold.rows != nullptr, epi);
-    const int stream_w = (sc.n_n == 1) ? 1 : 0;  // W is read by one pair only: do not keep it in L2
+    // W is not kept in L2 when one pair reads each block, nor when the tiles are shared out by the counter:
+    // the pairs that share a block then read it within microseconds of one another, and a block of W that
+    // lingers only pushes h_target out (2080 x 8192 rows against 128256 entries: 2.21 GB of DRAM reads per
+    // launch instead of 2.80, and 3.9 with the fixed order, against 2.14 GB of operands)
+    const int stream_w = (sc.n_n == 1 || a.sched) ? 1 : 0;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)p.grid);  // 2 CTAs per pair
     cfg.blockDim = dim3(num_threads(sc.dual != 0));
@@ -485,7 +565,7 @@ cudaError_t launch_umma_pair(const GemmArgs &a, const UmmaPlan &p, cudaStream_t 
                   : a.rank.thr               ? pick(std::integral_constant<int, EPI_COUNT>{})
                                              : pick(std::integral_constant<int, EPI_PLAIN>{});
     return cudaLaunchKernelEx(&cfg, kernel, p.tmap_w, p.tmap_h, a.fold.rows ? p.tmap_j : p.tmap_w, a.M, a.V, a.d, sc, stream_w,
-                              a.v_offset, a.keys, a.status, a.pub, a.rank, a.noise, a.fold.parts, a.fold.stride);
+                              a.v_offset, a.keys, a.status, a.pub, a.rank, a.noise, a.fold.parts, a.fold.stride, a.sched);
 }
 
 }  // namespace aj

@@ -286,8 +286,9 @@ const char *aj_last_gemm_path(aj_handle h);
  * pool at start-up, that runs under a per-allocation memory audit, or whose allocator is frozen by
  * the time it needs a cycle verified cannot use a handle.  This function takes no handle and calls
  * no cudaMalloc, cudaFree or any allocating routine: its only scratch memory, one 8-byte key per row
- * of hidden states plus a status word, is a fixed array inside the library's device image, so every
- * GPU that loads the library holds AJ_STATIC_MAX_ROWS * 8 + 256 bytes (about 256 KB) until exit.
+ * of hidden states plus a 256-byte block (a status word, and the two words through which the CTA pairs
+ * of the two-SM kernel share out their tiles), is a fixed array inside the library's device image, so
+ * every GPU that loads the library holds AJ_STATIC_MAX_ROWS * 8 + 256 bytes (about 256 KB) until exit.
  *
  * Arguments are those of aj_create and aj_verify together; the device is the CURRENT CUDA device;
  * all pointers are device pointers with the layouts aj_verify documents; optional outputs may be

@@ -164,6 +164,24 @@ void *device_view(const void *host_ptr) {
 
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
+// Brings one cycle's hidden states from pinned host memory into the handle's staging buffers: every
+// thread fetches 16-byte pieces over PCIe (all of a small batch's pieces are in flight at once).  For the
+// few hundred KB of a small batch this takes less than two copy operations do, and the projection
+// kernel, launched as a programmatic dependent, sets itself up meanwhile.
+__global__ void stage_hidden_kernel(const uint4 *__restrict__ a_src, uint4 *__restrict__ a_dst, unsigned n_a,
+                                    const uint4 *__restrict__ b_src, uint4 *__restrict__ b_dst, unsigned n_b) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const unsigned stride = gridDim.x * blockDim.x;
+    for (unsigned i = blockIdx.x * blockDim.x + threadIdx.x; i < n_a + n_b; i += stride) {
+        // the host rewrites these buffers between cycles: never a cached copy
+        if (i < n_a)
+            a_dst[i] = __ldcv(a_src + i);
+        else
+            b_dst[i - n_a] = __ldcv(b_src + (i - n_a));
+    }
+}
+constexpr size_t STAGE_KERNEL_MAX_BYTES = 1u << 20;  // above this the copy engines are at least as fast
+
 }  // namespace
 
 extern "C" {
@@ -508,9 +526,25 @@ aj_status aj_verify_host(aj_handle h, const void *h_target_host, const void *h_d
     const size_t M = (size_t)B * rows_per_seq(h, K), esz = elem_size(h->dtype);
     // The hidden states are always copied (the projection kernel reads them a thousand times over), and
     // their copies are enqueued first: everything the host does next runs while they are on their way.
-    bool ok = cudaMemcpyAsync(h->st_ht, h_target_host, M * d * esz, cudaMemcpyHostToDevice, stream) == cudaSuccess &&
-              (h->d_draft == 0 ||
-               cudaMemcpyAsync(h->st_hd, h_draft_host, M * h->d_draft * esz, cudaMemcpyHostToDevice, stream) == cudaSuccess);
+    // A small batch in pinned memory is fetched by a kernel, anything else by the copy engines.
+    const size_t ht_bytes = M * d * esz, hd_bytes = M * h->d_draft * esz;
+    bool ok = true, staged = false;
+    if (ht_bytes + hd_bytes <= STAGE_KERNEL_MAX_BYTES && ht_bytes % 16 == 0 && hd_bytes % 16 == 0) {
+        const void *ht_view = device_view(h_target_host);
+        const void *hd_view = hd_bytes ? device_view(h_draft_host) : nullptr;
+        if (ht_view && aligned16(ht_view) && (hd_bytes == 0 || (hd_view && aligned16(hd_view)))) {
+            const unsigned n_a = (unsigned)(ht_bytes / 16), n_b = (unsigned)(hd_bytes / 16);
+            const unsigned blocks = (n_a + n_b + 255) / 256;
+            stage_hidden_kernel<<<blocks < 1024 ? blocks : 1024, 256, 0, stream>>>(
+                static_cast<const uint4 *>(ht_view), static_cast<uint4 *>(h->st_ht), n_a, static_cast<const uint4 *>(hd_view),
+                static_cast<uint4 *>(h->st_hd), n_b);
+            ok = cudaGetLastError() == cudaSuccess;
+            staged = true;
+        }
+    }
+    if (!staged)
+        ok = cudaMemcpyAsync(h->st_ht, h_target_host, ht_bytes, cudaMemcpyHostToDevice, stream) == cudaSuccess &&
+             (hd_bytes == 0 || cudaMemcpyAsync(h->st_hd, h_draft_host, hd_bytes, cudaMemcpyHostToDevice, stream) == cudaSuccess);
     if (!ok) return AJ_ERR_CUDA;
     // Small host buffers that are pinned (and therefore mapped into the device's address space) are
     // used in place by the judge kernel: it reads the draft tokens and writes the results over PCIe,
@@ -525,7 +559,7 @@ aj_status aj_verify_host(aj_handle h, const void *h_target_host, const void *h_d
                    d, V, acc_dev ? acc_dev : h->st_acc, next_dev ? next_dev : h->st_next,
                    target_tok_host ? (tt_dev ? tt_dev : h->st_tt) : nullptr, nullptr, nullptr, cuda_stream);
     if (st != AJ_OK) return st;
-    const int launches = h->last_launches;
+    const int launches = h->last_launches + (staged ? 1 : 0);
     ok = (acc_dev || cudaMemcpyAsync(accept_len_host, h->st_acc, (size_t)B * 4, cudaMemcpyDeviceToHost, stream) == cudaSuccess) &&
          (next_dev || cudaMemcpyAsync(next_tok_host, h->st_next, (size_t)B * 4, cudaMemcpyDeviceToHost, stream) == cudaSuccess) &&
          (!target_tok_host || tt_dev ||

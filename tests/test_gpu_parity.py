@@ -405,6 +405,44 @@ def test_host_buffer_entry_point_matches_device_entry_point():
         case.close()
 
 
+def test_host_entry_point_reads_the_host_buffers_afresh_every_cycle():
+    """The same pinned buffers are rewritten by the host between cycles (a small batch is fetched from them by
+    a kernel, a large one by the copy engines): every cycle must see what they hold then.  Also the
+    target-only classifier, where there is no second tensor to fetch."""
+    import torch
+
+    orc = _oracle()
+    for name, B, K, d, dd, V in (("host_small", 4, 20, 512, 256, 9000), ("host_target_only", 3, 12, 256, 0, 4000),
+                                 ("host_large", 24, 40, 768, 256, 3000)):  # 24 x 41 x (768 + 256) x 2 B = 2 MB: copy engines
+        cfg = gen.Config(name, B=B, K=K, d=d, d_draft=dd, V=V, sigma_W=0.2, sigma_w=0.05, match_lo=0.5, match_hi=0.9, seed=19)
+        W, ht, hd, w = _host_case(cfg)
+        tok = gen.plant_draft_tokens(cfg, _oracle_y(cfg, W, ht))
+        case = DeviceCase(cfg, W, ht, hd, w)
+        try:
+            pin = lambda a: torch.from_numpy(a.view(np.int16) if a.dtype == np.uint16 else a).pin_memory()
+            ht_h, tok_h = pin(ht.copy()), pin(tok.copy())
+            hd_h = pin(hd.copy()) if dd else None
+            acc = torch.full((cfg.B,), -1, dtype=torch.int32).pin_memory()
+            nxt = torch.full((cfg.B,), -1, dtype=torch.int32).pin_memory()
+            tt = torch.full((cfg.B, cfg.K + 1), -1, dtype=torch.int32).pin_memory()
+            order = np.arange(cfg.B)
+            for cycle in range(4):
+                # rotate the sequences through the same buffers, in place
+                order = np.roll(order, 1)
+                ht_h.numpy()[:] = ht[order].view(np.int16)
+                tok_h.numpy()[:] = tok[order]
+                if dd:
+                    hd_h.numpy()[:] = hd[order].view(np.int16)
+                case.handle.verify_host(ht_h, hd_h, case.W, tok_h, case.w, cfg.judge_b, 0.5, cfg.B, cfg.K, acc, nxt, tt,
+                                        stream=torch.cuda.current_stream().cuda_stream)
+                o = orc.verify(ht[order], hd[order] if dd else None, W, tok[order], w, cfg.judge_b, 0.5, cfg.dtype)
+                np.testing.assert_array_equal(tt.numpy(), o.target_tok)
+                np.testing.assert_array_equal(acc.numpy(), o.accept_len)
+                np.testing.assert_array_equal(nxt.numpy(), o.next_tok)
+        finally:
+            case.close()
+
+
 def test_a_cycle_captured_in_a_cuda_graph_replays_with_new_inputs():
     """aj_verify only enqueues (two kernel launches, no allocation, no synchronisation), so a cycle can be
     captured in a CUDA graph and replayed: the replay reads whatever the input buffers hold then."""

@@ -138,7 +138,8 @@ aj_status aj_fuse_judge(aj_handle h, const float *judge_w, void *cuda_stream);
  * (among equal logits the lower index ranks first; a draft token outside the vocabulary is never
  * accepted).  The classifier is then not consulted: judge_w and h_draft may be NULL and judge_b, tau
  * are ignored; judge_p, if given, receives the draft token's rank (as a float, 0 = the target's own
- * token) at every mismatching position and NaN elsewhere.  A cycle then launches three kernels (the
+ * token) at every mismatching position and NaN elsewhere; a rank below top_k is exact, a rejected
+ * token's is some value from top_k up to its rank (the count stops once top_k entries outrank it).  A cycle then launches three kernels (the
  * draft tokens' own logits, the projection with the count fused into its epilogue, the scan).
  * top_k = 0 switches back to the classifier.  Not available on vocabulary-parallel handles or with
  * AJ_FLAG_NO_EXTRA_ROW (AJ_ERR_UNSUPPORTED).  Errors: AJ_ERR_INVALID_ARG.

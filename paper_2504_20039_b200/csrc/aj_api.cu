@@ -337,6 +337,7 @@ static aj_status enqueue_project(aj_handle h, const void *h_target, const void *
         g.rank.thr = h->rk_thr;
         g.rank.tok = h->rk_tok;
         g.rank.cnt = h->rk_cnt;
+        g.rank.top_k = h->top_k;
     }
     if (h->temperature > 0.0f) {
         g.noise.temperature = h->temperature;
@@ -385,7 +386,7 @@ static aj_status enqueue_project(aj_handle h, const void *h_target, const void *
         // tensor-bound regime: two-SM tiles of 256 vocabulary entries x up to 256 rows
         UmmaPlan p;
         p.bn = 256;
-        const PairSched sc = pair_schedule(M, V, d, fold, h->temperature > 0.0f ? EPI_SAMPLE : h->top_k > 0 ? EPI_COUNT : EPI_PLAIN);
+        const PairSched sc = pair_schedule(M, V, d, fold);
         const CUtensorMap *tw = get_tmap(h, W_lm, V, h->layout == AJ_W_DV ? -1 : 128);
         const CUtensorMap *th = get_tmap(h, h_target, M, sc.box_rows);
         const CUtensorMap *tj = fold ? get_tmap(h, h->fold_rows, h->layout == AJ_W_DV ? 8 : JUDGE_FOLD_ROWS, h->layout == AJ_W_DV ? -1 : 128) : tw;

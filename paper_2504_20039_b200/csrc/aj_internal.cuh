@@ -126,21 +126,29 @@ __device__ inline void publish_keys(const Publish &p, unsigned long long *keys) 
 // threshold); the projection kernels then also count, per row, the entries that outrank it
 // (larger logit, or equal logit and lower index), and the judge kernel compares the count with top_k.
 struct RankArgs {
-    const float *thr = nullptr;  // [M] the draft token's logit; +inf where the row has no draft token
+    float *thr = nullptr;        // [M] the draft token's logit; +inf where the row has no draft token, and
+                                 //     raised to +inf by the tensor-core kernels once top_k entries outrank it
     const int *tok = nullptr;    // [M] the draft token, -1 where there is none or it is outside the vocabulary
     unsigned *cnt = nullptr;     // [M] entries that outrank it (zeroed by the threshold kernel)
+    int top_k = 0;               // the rule asks only whether fewer than top_k entries outrank the token
 };
 
 #ifdef __CUDACC__
 // Epilogue add-on for the vocabulary-major kernels: the warp holds 32 consecutive vocabulary entries
-// (lane = entry v_first + lane) of 32 columns (rows row_first .. + 32 of h) in v[]; lane j is
-// responsible for column j.
-__device__ inline void count_outranking(const RankArgs &rk, const float (&v)[32], int v_first, bool v_ok, int row_first,
-                                        int n_cols, int M, int lane) {
-    const int row = row_first + lane;
-    const bool valid = lane < n_cols && row < M;
-    const float th = valid ? __ldg(rk.thr + row) : INFINITY;
-    const int tk = valid ? __ldg(rk.tok + row) : -1;
+// (lane = entry v_first + lane) of 32 columns (32 consecutive rows of h) in v[]; lane j is responsible
+// for column j: `row` is its row of h, th / tk that row's threshold and draft token (+inf / -1 where the
+// column is not a row of the batch), vmax the largest of this lane's 32 logits.
+// A row whose count has reached top_k is settled (the rule only asks whether fewer than top_k entries
+// outrank the token): its threshold is raised to +inf in global memory, so later tiles read that and leave
+// it alone.  And a chunk none of whose logits reaches the lowest of its 32 thresholds is left after one
+// reduction and one vote, which is nearly every chunk once the settled rows are out of the way.
+__device__ inline float rank_threshold(const RankArgs &rk, int row, bool valid) {
+    return valid ? __ldcg(rk.thr + row) : INFINITY;  // from L2: other SMs raise it while this kernel runs
+}
+__device__ inline void count_outranking(const RankArgs &rk, const float (&v)[32], float vmax, int v_first, bool v_ok, float th,
+                                        int tk, int row, bool valid, int lane) {
+    const uint32_t tmin = warp_min_u32(ordered_image(th));
+    if (!__any_sync(0xffffffffu, v_ok && ordered_image(vmax) >= tmin)) return;
     const int vidx = v_first + lane;
     unsigned mine = 0;
 #pragma unroll
@@ -151,7 +159,10 @@ __device__ inline void count_outranking(const RankArgs &rk, const float (&v)[32]
         const unsigned b = __ballot_sync(0xffffffffu, ahead);
         if (lane == j) mine = __popc(b);
     }
-    if (valid && mine) atomicAdd(rk.cnt + row, mine);
+    if (valid && mine) {
+        const unsigned before = atomicAdd(rk.cnt + row, mine);
+        if (before < (unsigned)rk.top_k && before + mine >= (unsigned)rk.top_k) rk.thr[row] = INFINITY;
+    }
 }
 #endif
 
@@ -317,7 +328,7 @@ struct PairSched {
     int n_groups;          // row tiles are walked in groups ...
     int g_base, g_rem;     // ... group g holds g_base + (g < g_rem) row tiles
 };
-PairSched pair_schedule(int M, int V, int d, int fold, int epi = 0);  // epi: EPI_PLAIN / EPI_COUNT / EPI_SAMPLE
+PairSched pair_schedule(int M, int V, int d, int fold);
 cudaError_t umma_pair_prepare(int num_sms);
 int umma_pair_max_pairs();
 cudaError_t launch_umma_pair(const GemmArgs &a, const UmmaPlan &p, cudaStream_t stream);

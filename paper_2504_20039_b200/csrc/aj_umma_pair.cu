@@ -371,6 +371,18 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
             uint32_t kk[CH];
 #pragma unroll
             for (int i = 0; i < CH; i++) kk[i] = load_key(tl, i);
+            // top-K rule: the thresholds and draft tokens of the accumulator's rows, fetched ahead like the keys
+            float thp[EPI == EPI_COUNT ? CH : 1];
+            int tkp[EPI == EPI_COUNT ? CH : 1];
+            if (EPI == EPI_COUNT) {
+#pragma unroll
+                for (int i = 0; i < CH; i++) {
+                    const int col = i * 32 + lane, row = tl.first_row(a) + col;
+                    const bool valid = col < tl.rows(a) && row < M;
+                    thp[i] = rank_threshold(rk, row, valid);
+                    tkp[i] = valid ? __ldg(rk.tok + row) : -1;
+                }
+            }
             const int v_first = tl.v_tile * BV + (int)rank * BV_CTA + q * 32;  // vocabulary entry of lane 0
             const bool v_ok = v_first + lane < V;                            // entries past V hold zero-filled junk
             const uint32_t tbase = tmem_base + ((uint32_t)(q * 32) << 16);
@@ -386,6 +398,12 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
                 const uint32_t kthr = kk[0];
 #pragma unroll
                 for (int i = 0; i + 1 < CH; i++) kk[i] = kk[i + 1];
+                const float th_c = thp[0];
+                const int tk_c = tkp[0];
+                if (EPI == EPI_COUNT) {
+#pragma unroll
+                    for (int i = 0; i + 1 < CH; i++) thp[i] = thp[i + 1], tkp[i] = tkp[i + 1];
+                }
                 {
                     float v[32];
                     tmem_ld32(tbase + acc_col(it, a) + (uint32_t)(c * 32), v);
@@ -401,13 +419,16 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
                         }
                         continue;
                     }
-                    if (EPI == EPI_COUNT) count_outranking(rk, v, v_first, v_ok, row_a + c * 32, n_inst - c * 32, M, lane);
                     if (EPI == EPI_SAMPLE) add_gumbel_noise(nz, v, v_first + lane + v_offset, row_a + c * 32);
-                    // the lowest threshold of the chunk (a row without a key yet: everything qualifies)
-                    const uint32_t tmin = warp_min_u32(kthr);
                     float vmax = v[0];
 #pragma unroll
                     for (int j = 1; j < 32; j++) vmax = fmaxf(vmax, v[j]);
+                    if (EPI == EPI_COUNT) {
+                        const int row = row_a + c * 32 + lane;
+                        count_outranking(rk, v, vmax, v_first, v_ok, th_c, tk_c, row, c * 32 + lane < n_inst && row < M, lane);
+                    }
+                    // the lowest threshold of the chunk (a row without a key yet: everything qualifies)
+                    const uint32_t tmin = warp_min_u32(kthr);
                     if (__any_sync(0xffffffffu, v_ok && ordered_image(vmax) >= tmin)) {
                         const float thr = kthr == NO_ROW ? __int_as_float(0x7fc00000)  // NaN: no comparison with it is ever true
                                           : kthr == 0u  ? -INFINITY
@@ -505,15 +526,13 @@ cudaError_t umma_pair_prepare(int num_sms) {
 
 int umma_pair_max_pairs() { return g_max_pairs; }
 
-PairSched pair_schedule(int M, int V, int d, int fold, int epi) {
+PairSched pair_schedule(int M, int V, int d, int fold) {
     PairSched sc;
     sc.fold = fold ? 1 : 0;
     const int units = (M + 15) / 16;  // rows in units of 16 (the UMMA N granule)
     // Wide tiles (up to 512 rows on two accumulators with an issuing warp each) for every batch of more
-    // than 256 rows; up to 256 rows one narrow tile per vocabulary block, double-buffered.  The epilogue
-    // of a wide tile is not hidden under MMAs; the counting epilogue of the top-K rule is long enough for
-    // narrow tiles to win where a tile is short (d = 4096, 2112 rows: 1.78 vs 2.01 ms; d = 8192: wide).
-    sc.dual = (units > 16 && !(epi == EPI_COUNT && d < 8192 && units > 32)) ? 1 : 0;
+    // than 256 rows; up to 256 rows one narrow tile per vocabulary block, double-buffered.
+    sc.dual = units > 16 ? 1 : 0;
     const int cap = sc.dual ? 32 : 16;
     sc.n_n = (units + cap - 1) / cap;
     sc.u_base = units / sc.n_n;
@@ -535,8 +554,7 @@ PairSched pair_schedule(int M, int V, int d, int fold, int epi) {
 }
 
 cudaError_t launch_umma_pair(const GemmArgs &a, const UmmaPlan &p, cudaStream_t stream) {
-    const int epi = a.noise.temperature > 0.0f ? EPI_SAMPLE : a.rank.thr ? EPI_COUNT : EPI_PLAIN;
-    const PairSched sc = pair_schedule(a.M, a.V, a.d, a.fold.rows != nullptr, epi);
+    const PairSched sc = pair_schedule(a.M, a.V, a.d, a.fold.rows != nullptr);
     // W is not kept in L2 when one pair reads each block, nor when the tiles are shared out by the counter:
     // the pairs that share a block then read it within microseconds of one another, and a block of W that
     // lingers only pushes h_target out (2080 x 8192 rows against 128256 entries: 2.21 GB of DRAM reads per

@@ -236,7 +236,15 @@ umma_vm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                         }
                         continue;
                     }
-                    if (EPI == EPI_COUNT) count_outranking(rk, v, v_first, v_ok, n_tile * BN + c * 32, n_inst - c * 32, M, lane);
+                    if (EPI == EPI_COUNT) {
+                        const int row = n_tile * BN + c * 32 + lane;
+                        const bool valid = c * 32 + lane < n_inst && row < M;
+                        float vmax = v[0];
+#pragma unroll
+                        for (int j = 1; j < 32; j++) vmax = fmaxf(vmax, v[j]);
+                        count_outranking(rk, v, vmax, v_first, v_ok, rank_threshold(rk, row, valid), valid ? __ldg(rk.tok + row) : -1, row,
+                                         valid, lane);
+                    }
                     if (EPI == EPI_SAMPLE) add_gumbel_noise(nz, v, v_first + lane + v_offset, n_tile * BN + c * 32);
                     // all 32 reductions are issued before any result is used, so that their
                     // latencies overlap instead of adding up

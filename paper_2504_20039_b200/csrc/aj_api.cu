@@ -312,6 +312,8 @@ static aj_status enqueue_project(aj_handle h, const void *h_target, const void *
     if (h->keys_dirty) {
         const size_t all = (size_t)h->max_B * (h->max_K + 1) * sizeof(unsigned long long);
         if (cudaMemsetAsync(h->keys, 0, all, stream) != cudaSuccess) return AJ_ERR_CUDA;
+        // (and the two-SM kernel's tile counter, which a cycle that gave up may not have put back)
+        if (cudaMemsetAsync(reinterpret_cast<unsigned *>(h->status) + 32, 0, 2 * sizeof(unsigned), stream) != cudaSuccess) return AJ_ERR_CUDA;
     }
     h->keys_dirty = true;
 

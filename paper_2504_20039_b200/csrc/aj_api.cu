@@ -343,6 +343,7 @@ static aj_status enqueue_project(aj_handle h, const void *h_target, const void *
     }
     if (h->temperature > 0.0f) {
         g.noise.temperature = h->temperature;
+        g.noise.inv_temperature = 1.0f / h->temperature;
         g.noise.key0 = (uint32_t)h->seed;
         g.noise.key1 = (uint32_t)(h->seed >> 32);
         g.noise.step0 = (uint32_t)h->step;

@@ -176,6 +176,7 @@ __device__ inline void count_outranking(const RankArgs &rk, const float (&v)[32]
 // u = ((x >> 9) + 0.5) * 2^-23 (exact in fp32, never 0 or 1); g = -ln(-ln u).
 struct Noise {
     float temperature = 0.0f;  // 0: greedy, no noise
+    float inv_temperature = 0.0f;
     uint32_t key0 = 0, key1 = 0;    // seed
     uint32_t step0 = 0, step1 = 0;  // cycle counter
 };
@@ -232,17 +233,59 @@ __device__ inline float noisy_score(const Noise &nz, float logit, int row, int v
     return fmaf(nz.temperature * -0.693147180559945f, lg2_neg_ln_uniform(x), logit);
 }
 
+// Which draws can matter.  A thread holds 32 logits of one vocabulary entry, none above vmax, and the rows
+// they belong to have each a best noisy score so far, none below `lowest`: an element can only take its
+// row over if its noise is at least need = (lowest - vmax) / T.  The noise grows with the random word, so
+// that is a cutoff on the word's upper 23 bits: k >= u(need) 2^23 with u(g) = exp(-exp(-g)), taken with a
+// margin (need lowered by 2e-3, 16 counts off) that covers the approximate exponentials.  0: every draw
+// may matter (no row has a score yet, or need is small); that is also the answer to a NaN.
+__device__ inline float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ inline uint32_t noise_cutoff(float lowest, float vmax, float inv_temperature) {
+    const float need = (lowest - vmax) * inv_temperature - 2e-3f;
+    if (!(need > -3.0f)) return 0u;
+    const float e = ex2_approx(-1.4426950408889634f * need);  // exp(-need) <= e^3
+    const float u = ex2_approx(-1.4426950408889634f * e);
+    const float k = u * 8388608.0f - 16.0f;
+    return k > 0.0f ? (uint32_t)k : 0u;
+}
+
 // Epilogue add-on for the vocabulary-major kernels: this thread holds entry v of the 32 rows
-// row_first .. + 32 (row_first a multiple of 4) in x[]; one Philox call serves four rows.
-__device__ inline void add_gumbel_noise(const Noise &nz, float (&x)[32], int v, int row_first) {
+// row_first .. + 32 (row_first a multiple of 4) in x[]; one Philox call serves four rows.  Every word
+// is drawn (the eight generator calls of a chunk back to back, so that their multiply chains overlap); the
+// two logarithms are only taken of the words that reach k_need (see noise_cutoff), the other elements
+// cannot take their row over and become -inf.  False: no element of the warp's chunk can matter and x[] is
+// left as it was.  The whole warp must call this together.
+__device__ inline bool add_gumbel_noise(const Noise &nz, float (&x)[32], int v, int row_first, uint32_t k_need) {
     const float scale = nz.temperature * -0.693147180559945f;
+    uint32_t w[32];
 #pragma unroll
     for (int q = 0; q < 8; q++) {
-        uint32_t w[4];
-        philox4x32_10((uint32_t)v, (uint32_t)((row_first >> 2) + q), nz.step0, nz.step1, nz.key0, nz.key1, w);
-#pragma unroll
-        for (int i = 0; i < 4; i++) x[4 * q + i] = fmaf(scale, lg2_neg_ln_uniform(w[i]), x[4 * q + i]);
+        uint32_t o[4];
+        philox4x32_10((uint32_t)v, (uint32_t)((row_first >> 2) + q), nz.step0, nz.step1, nz.key0, nz.key1, o);
+        w[4 * q + 0] = o[0], w[4 * q + 1] = o[1], w[4 * q + 2] = o[2], w[4 * q + 3] = o[3];
     }
+    uint32_t top = w[0];
+#pragma unroll
+    for (int i = 1; i < 32; i++) top = w[i] > top ? w[i] : top;
+    if (!__any_sync(0xffffffffu, (top >> 9) >= k_need)) return false;  // one decision per warp: a real branch
+#pragma unroll
+    for (int q = 0; q < 8; q++) {
+        const bool c0 = (w[4 * q] >> 9) >= k_need, c1 = (w[4 * q + 1] >> 9) >= k_need, c2 = (w[4 * q + 2] >> 9) >= k_need,
+                   c3 = (w[4 * q + 3] >> 9) >= k_need;
+        if (__any_sync(0xffffffffu, c0 || c1 || c2 || c3)) {
+            x[4 * q + 0] = c0 ? fmaf(scale, lg2_neg_ln_uniform(w[4 * q + 0]), x[4 * q + 0]) : -INFINITY;
+            x[4 * q + 1] = c1 ? fmaf(scale, lg2_neg_ln_uniform(w[4 * q + 1]), x[4 * q + 1]) : -INFINITY;
+            x[4 * q + 2] = c2 ? fmaf(scale, lg2_neg_ln_uniform(w[4 * q + 2]), x[4 * q + 2]) : -INFINITY;
+            x[4 * q + 3] = c3 ? fmaf(scale, lg2_neg_ln_uniform(w[4 * q + 3]), x[4 * q + 3]) : -INFINITY;
+        } else {
+            x[4 * q + 0] = x[4 * q + 1] = x[4 * q + 2] = x[4 * q + 3] = -INFINITY;
+        }
+    }
+    return true;
 }
 #endif
 

@@ -419,7 +419,15 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
                         }
                         continue;
                     }
-                    if (EPI == EPI_SAMPLE) add_gumbel_noise(nz, v, v_first + lane + v_offset, row_a + c * 32);
+                    // the lowest threshold of the chunk (a row without a key yet: everything qualifies)
+                    const uint32_t tmin = warp_min_u32(kthr);
+                    if (EPI == EPI_SAMPLE) {
+                        float pmax = v[0];  // of the plain logits
+#pragma unroll
+                        for (int j = 1; j < 32; j++) pmax = fmaxf(pmax, v[j]);
+                        const uint32_t k_need = noise_cutoff(key_value((unsigned long long)tmin << 32), pmax, nz.inv_temperature);
+                        if (!add_gumbel_noise(nz, v, v_first + lane + v_offset, row_a + c * 32, k_need)) continue;
+                    }
                     float vmax = v[0];
 #pragma unroll
                     for (int j = 1; j < 32; j++) vmax = fmaxf(vmax, v[j]);
@@ -427,8 +435,6 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
                         const int row = row_a + c * 32 + lane;
                         count_outranking(rk, v, vmax, v_first, v_ok, th_c, tk_c, row, c * 32 + lane < n_inst && row < M, lane);
                     }
-                    // the lowest threshold of the chunk (a row without a key yet: everything qualifies)
-                    const uint32_t tmin = warp_min_u32(kthr);
                     if (__any_sync(0xffffffffu, v_ok && ordered_image(vmax) >= tmin)) {
                         const float thr = kthr == NO_ROW ? __int_as_float(0x7fc00000)  // NaN: no comparison with it is ever true
                                           : kthr == 0u  ? -INFINITY

@@ -245,7 +245,16 @@ umma_vm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                         count_outranking(rk, v, vmax, v_first, v_ok, rank_threshold(rk, row, valid), valid ? __ldg(rk.tok + row) : -1, row,
                                          valid, lane);
                     }
-                    if (EPI == EPI_SAMPLE) add_gumbel_noise(nz, v, v_first + lane + v_offset, n_tile * BN + c * 32);
+                    if (EPI == EPI_SAMPLE) {
+                        // the lowest of the chunk's running maxima bounds the noise an element needs to matter
+                        const int row = n_tile * BN + c * 32 + lane;
+                        const uint32_t tmin = warp_min_u32((c * 32 + lane < n_inst && row < M) ? rb_u[c] : 0xFFFFFFFFu);
+                        float pmax = v[0];
+#pragma unroll
+                        for (int j = 1; j < 32; j++) pmax = fmaxf(pmax, v[j]);
+                        const uint32_t k_need = noise_cutoff(key_value((unsigned long long)tmin << 32), pmax, nz.inv_temperature);
+                        if (!add_gumbel_noise(nz, v, v_first + lane + v_offset, n_tile * BN + c * 32, k_need)) continue;
+                    }
                     // all 32 reductions are issued before any result is used, so that their
                     // latencies overlap instead of adding up
                     uint32_t u[32], m[32];

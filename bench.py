@@ -5,8 +5,9 @@
 A step is one whole cycle (LM-head projection + argmax, then judge + prefix scan: two launches) over one
 batch of seeded synthetic inputs shaped like the paper's Llama-3.x pairs.  The headline workload is
 the batch-1 8B-shaped configuration (B=1, K=16, d=4096, V=128256, bf16), the setting the paper's own
-measurements use (batch size 1); the batched 8B- and 70B-shaped configurations are reported under
-"extra" in the same JSON line.  Metric: verified draft positions per second (B*K per cycle).
+measurements use (batch size 1); the batched 8B- and 70B-shaped configurations, three points of the sweep
+around the HBM / tensor crossover, and two variants of the acceptance step (sampled target tokens, the top-K
+rule) are reported under "extra" in the same JSON line.  Metric: verified draft positions per second (B*K per cycle).
 
 Rank layout for N > 1: one process per GPU, every rank verifies its own batch against its own copy
 of W_lm (sequences are independent, there is no data-path collective): weak scaling.
@@ -568,14 +569,20 @@ def main():
             # the batched 8B- and 70B-shaped workloads, and the three points of the sweep around the crossover
             # from HBM-bound to tensor-bound (264, 520 and 576 rows)
             todo = [gen.C3, gen.sweep_config(8, 32), gen.sweep_config(8, 64), gen.sweep_config(64, 8), gen.C4]
-        for cfg in todo:
+            if not rule:
+                # and the two variants of the acceptance step whose epilogues do more, each right after the
+                # default rule on the same workload: sampled target tokens at C3, the top-K rule at C4
+                todo = [gen.C3, (gen.C3, {"temperature": 1.0})] + todo[1:] + [(gen.C4, {"top_k": 8})]
+        for item in todo:
+            cfg, item_rule = item if isinstance(item, tuple) else (item, rule)
             cfg = ajd.rank_config(cfg, rank)
             same_W = cfg.d == head.d and cfg.V == head.V
             n = max(20, int(0.4 / max(2.0 * cfg.M * cfg.d * cfg.V / 1.2e15, 1.7e-4)))
-            rr = bench_one(cfg, local, n, 5, barrier, reduce_max, pk, 2 if not same_W else copies, W_host if same_W else None, with_e2e=False, flags=args.flags, rule=rule)
+            rr = bench_one(cfg, local, n, 5, barrier, reduce_max, pk, 2 if not same_W else copies, W_host if same_W else None, with_e2e=False, flags=args.flags, rule=item_rule)
             extra.append({"workload": cfg.name, "B": cfg.B, "K": cfg.K, "d": cfg.d, "V": cfg.V, "steps": n,
                           "ms_per_step": rr["ms_per_step"], "value": cfg.B * cfg.K * world / (rr["ms_per_step"] * 1e-3), "unit": UNIT,
-                          "gemm_path": rr["path"], "roofline": rr["roofline"], "clocks": rr["clocks"]})
+                          "gemm_path": rr["path"], "rule": item_rule or "classifier at tau on greedy target tokens",
+                          "roofline": rr["roofline"], "clocks": rr["clocks"]})
     if world > 1 and not vocab and args.workload == "c2" and not args.no_extra:
         # Strong scaling of the headline workload with the LM head split by vocabulary over the ranks: one batch,
         # every rank streams 1/N of W_lm, per-row keys exchanged by peer stores inside the kernels.  Recorded

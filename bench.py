@@ -279,7 +279,10 @@ def roofline_of(cfg: gen.Config, gemm_ms: float, pk, v_count=None, gemm_ms_min=N
     else:
         a = flops / s / 1e12
         r = {"bound": "tensor", "achieved": a, "peak": pk["bf16_tflops"], "unit": "TFLOP/s", "frac": a / pk["bf16_tflops"],
-             "frac_of_sustained_peak": a / pk["bf16_tflops_sustained"], "traffic": None, "peak_source": f"of {pk['source']}",
+             "frac_of_sustained_peak": a / pk["bf16_tflops_sustained"], "sustained_peak": pk["bf16_tflops_sustained"],
+             "peak_kind": "burst; kernel_ms is the mean launch of a loop that runs under the power cap, for which the sustained "
+                          "peak is the like-for-like figure (frac_of_sustained_peak); frac_alone is the launch timed alone against the burst peak",
+             "traffic": None, "peak_source": f"of {pk['source']}",
              "kernel_ms": gemm_ms, "algorithmic_flops": flops}
     t_roof = max(t_hbm, t_tc)
     r["roofline_ms"] = t_roof * 1e3

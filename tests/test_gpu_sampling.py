@@ -83,6 +83,30 @@ def test_sampled_cycle_matches_the_oracle(shape):
         case.close()
 
 
+@pytest.mark.parametrize("T", [0.02, 0.2, 6.0, 40.0])
+def test_very_low_and_very_high_temperatures(T):
+    """The tensor-core kernels take the logarithms only of the draws that can still take a row over; how many
+    those are depends on the temperature (nearly none when it is low, nearly all when it is high, where the
+    noise dwarfs the logits).  Both ends, on the one-SM kernel and on narrow and wide two-SM tiles, over several
+    vocabulary tiles per CTA."""
+    for name, B, K, d, dd, V, flags, path in (("t_one_sm", 2, 14, 128, 64, 40000, 0, "umma_vm_128x32"),
+                                              ("t_pair_narrow", 4, 49, 128, 0, 50000, 0, "umma_pair_256x256"),
+                                              ("t_pair_wide", 10, 59, 128, 64, 60000, 0, "umma_pair_256x256")):
+        orc, cfg, W, ht, hd, w = _inputs(name, B, K, d, dd, V, gen.BF16, 0, seed=77)
+        case = DeviceCase(cfg, W, ht, hd, w, flags=flags)
+        try:
+            drawn = orc.verify(ht, hd, W, np.zeros((B, K), np.int32), w, cfg.judge_b, 0.0, gen.BF16, temperature=T, seed=5, step=9).target_tok
+            tok = gen.plant_draft_tokens(cfg, drawn)
+            case.handle.set_sampling(T, 5, 9)
+            o = orc.verify(ht, hd, W, tok, w, cfg.judge_b, 0.5, gen.BF16, temperature=T, seed=5, step=9)
+            g = case.run(tok, 0.5)
+            assert g.path == path
+            rep = check_parity(o, g, tok, 0.5)
+            assert rep.rows_exempt <= max(3, rep.rows // 10), rep
+        finally:
+            case.close()
+
+
 def test_every_kernel_draws_the_same_tokens():
     """One input, one random state: the one-SM kernel, the CTA-pair kernel, and the CUDA-core kernel see the
     same noise, so they agree wherever the noisy scores are not too close to call."""

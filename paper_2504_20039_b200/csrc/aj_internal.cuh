@@ -368,6 +368,7 @@ struct PairSched {
     int box_rows;          // rows of h each CTA of a pair stages per k-block and accumulator
     int dual;              // 1: every tile uses two accumulators that share the staged block of W
     int stages;            // depth of the shared-memory ring
+    int kps;               // k-blocks of 64 per stage (1 or 2)
     int n_groups;          // row tiles are walked in groups ...
     int g_base, g_rem;     // ... group g holds g_base + (g < g_rem) row tiles
 };

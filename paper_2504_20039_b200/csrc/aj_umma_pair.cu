@@ -159,7 +159,11 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
     const int stages = sc.stages;
     const uint32_t b_bytes = (uint32_t)sc.box_rows * BK * 2;       // one accumulator's rows of h staged by this CTA
     constexpr int n_acc = DUAL ? 2 : 1;
-    const uint32_t stage_bytes = A_BYTES + n_acc * b_bytes;         // a multiple of 1024
+    // A stage holds kps k-blocks (1 or 2), each [W | h of accumulator 0 | h of accumulator 1]: with two, the
+    // issuing thread tests one barrier and commits once per 8 MMAs instead of per 4.
+    const int kps = sc.kps;
+    const uint32_t sub_bytes = A_BYTES + n_acc * b_bytes;           // one k-block of a stage: a multiple of 1024
+    const uint32_t stage_bytes = (uint32_t)kps * sub_bytes;
     const uint32_t stage_tx = 2u * stage_bytes;                     // bytes both CTAs load per stage
 
     if (threadIdx.x == 0) {
@@ -248,9 +252,9 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
                 const int h_row0 = tl.row0[0] + (int)rank * (tl.n_inst[0] >> 1);
                 const int h_row1 = tl.row0[1] + (int)rank * (tl.n_inst[1] >> 1);
                 int next = -1;
-                for (int kb = 0; kb < num_kb; kb++) {
+                for (int kb = 0; kb < num_kb; kb += kps) {
                     // (the answer is not looked at before the loop ends: the thread does not wait for it here)
-                    if (rank == 0 && kb == kb_ask) next = sched ? (int)atomicAdd(sched, 1u) + num_pairs : t + num_pairs;
+                    if (rank == 0 && kb <= kb_ask && kb_ask < kb + kps) next = sched ? (int)atomicAdd(sched, 1u) + num_pairs : t + num_pairs;
                     if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) {
                         give_up();
                         ok = false;
@@ -258,15 +262,18 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
                     }
                     const uint32_t leader_full = map_to_cta(full_bar(s), 0);
                     if (rank == 0) mbar_expect_tx(full_bar(s), stage_tx);
-                    const uint32_t a_dst = base + s * stage_bytes;
-                    if (WDV) {  // W stored [d, V]: two boxes of 64 entries x 64 k-rows
-                        tma_load_2d_pair(a_dst, tw, w_row, kb * BK, leader_full, pol_w);
-                        tma_load_2d_pair(a_dst + A_BYTES / 2, tw, w_row + 64, kb * BK, leader_full, pol_w);
-                    } else {
-                        tma_load_2d_pair(a_dst, tw, kb * BK, w_row, leader_full, pol_w);
+                    for (int j = 0; j < kps; j++) {
+                        const uint32_t a_dst = base + s * stage_bytes + j * sub_bytes;
+                        const int kc = (kb + j) * BK;
+                        if (WDV) {  // W stored [d, V]: two boxes of 64 entries x 64 k-rows
+                            tma_load_2d_pair(a_dst, tw, w_row, kc, leader_full, pol_w);
+                            tma_load_2d_pair(a_dst + A_BYTES / 2, tw, w_row + 64, kc, leader_full, pol_w);
+                        } else {
+                            tma_load_2d_pair(a_dst, tw, kc, w_row, leader_full, pol_w);
+                        }
+                        tma_load_2d_pair(a_dst + A_BYTES, &tmap_h, kc, h_row0, leader_full, pol_h);
+                        if (n_acc == 2) tma_load_2d_pair(a_dst + A_BYTES + b_bytes, &tmap_h, kc, h_row1, leader_full, pol_h);
                     }
-                    tma_load_2d_pair(a_dst + A_BYTES, &tmap_h, kb * BK, h_row0, leader_full, pol_h);
-                    if (n_acc == 2) tma_load_2d_pair(a_dst + A_BYTES + b_bytes, &tmap_h, kb * BK, h_row1, leader_full, pol_h);
                     if (++s == stages) {
                         s = 0;
                         ph ^= 1u;
@@ -309,20 +316,22 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_consta
                 }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc_col(it, a);
-                for (int kb = 0; kb < num_kb; kb++) {
+                for (int kb = 0; kb < num_kb; kb += kps) {
                     if (!mbar_wait(full_bar(s), ph, abort_flag)) {
                         give_up();
                         ok = false;
                         break;
                     }
                     tc_fence_after();
-                    const uint32_t a_addr = base + s * stage_bytes;
-                    const unsigned long long adesc = WDV ? smem_desc_sw128_mn(a_addr) : smem_desc_sw128(a_addr);
-                    const unsigned long long bdesc = smem_desc_sw128(a_addr + b_off);
-                    if (n_inst) {
+                    for (int j = 0; j < kps; j++) {
+                        const uint32_t a_addr = base + s * stage_bytes + j * sub_bytes;
+                        const unsigned long long adesc = WDV ? smem_desc_sw128_mn(a_addr) : smem_desc_sw128(a_addr);
+                        const unsigned long long bdesc = smem_desc_sw128(a_addr + b_off);
+                        if (n_inst) {
 #pragma unroll
-                        for (int k = 0; k < BK / UMMA_K; k++)
-                            umma_bf16_pair(d_tmem, adesc + a_step * k, bdesc + 2ull * k, idesc, (uint32_t)((kb | k) != 0));
+                            for (int k = 0; k < BK / UMMA_K; k++)
+                                umma_bf16_pair(d_tmem, adesc + a_step * k, bdesc + 2ull * k, idesc, (uint32_t)((kb | j | k) != 0));
+                        }
                     }
                     umma_commit_pair(empty_bar(s));  // this accumulator is done with the stage, in both CTAs
                     if (++s == stages) {
@@ -547,7 +556,14 @@ PairSched pair_schedule(int M, int V, int d, int fold) {
     const int u_max = sc.u_base + (sc.u_rem ? 1 : 0);
     // rows of h each CTA stages per accumulator: half of the largest accumulator
     sc.box_rows = 8 * (sc.dual ? (u_max + 1) / 2 : u_max);
-    const int stage_bytes = A_BYTES + (sc.dual ? 2 : 1) * sc.box_rows * BK * 2;
+    // An issuing thread spends about 546 cycles on a k-block, 130 of them on the barrier test and the commit,
+    // and up to some 160 rows per accumulator that, not the tensor pipe, is what a tile waits for.  Two
+    // k-blocks per stage halve that share; taken where three such stages still fit (tiles of up to 320 rows:
+    // 136 rows 220 -> 191 us, 264 rows 267 -> 247, 520 rows 483 -> 436, 576 rows 503 -> 469; with two stages
+    // left, or on the tiles the pipe bounds, it costs 2 ... 8 % instead).
+    const int sub_bytes = A_BYTES + (sc.dual ? 2 : 1) * sc.box_rows * BK * 2;
+    sc.kps = ((d / BK) % 2 == 0 && RING_BYTES / (2 * sub_bytes) >= 3) ? 2 : 1;
+    const int stage_bytes = sc.kps * sub_bytes;
     sc.stages = RING_BYTES / stage_bytes < MAX_STAGES ? RING_BYTES / stage_bytes : MAX_STAGES;
     // row tiles per group: keep a group's rows of h (tile rows x d x 2 bytes) within about 40 MB of L2
     const long long tile_bytes = (sc.dual ? 512ll : 256ll) * d * 2;

@@ -56,7 +56,7 @@ template <int BN, bool WDV, int EPI>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 umma_vm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_h,
                const __grid_constant__ CUtensorMap tmap_j, int M, int V, int d, int n_n, int n_v, int fold_tile,
-               int stream_w, int v_offset, unsigned long long *__restrict__ keys, int *__restrict__ status, const Publish pub,
+               int stream_w, int kps, int v_offset, unsigned long long *__restrict__ keys, int *__restrict__ status, const Publish pub,
                const RankArgs rk, const Noise nz, float *__restrict__ fold_parts, int fold_stride) {
     using C = VCfg<BN>;
     constexpr int STAGES = C::STAGES;
@@ -77,6 +77,10 @@ umma_vm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
     const int lane = threadIdx.x & 31;
     const int num_kb = d / BK;
     const int num_tiles = n_n * n_v;
+    // A stage holds kps k-blocks (1 or 2), each [W | h], in the same ring: with two, the issuing thread tests
+    // one barrier and commits once per 8 MMAs instead of per 4.
+    const uint32_t stage_bytes = (uint32_t)kps * C::STAGE_BYTES;
+    const int stages = STAGES / kps;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; s++) {
@@ -119,22 +123,25 @@ umma_vm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                 const bool fold = v_tile == fold_tile;  // the block after the vocabulary: the classifier rows, entry 0 of their own map
                 const CUtensorMap *tw = fold ? &tmap_j : &tmap_w;
                 const int w_row = fold ? 0 : v_tile * BV;
-                for (int kb = 0; kb < num_kb; kb++) {
+                for (int kb = 0; kb < num_kb; kb += kps) {
                     if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) {
                         give_up();
                         ok = false;
                         break;
                     }
-                    mbar_expect_tx(full_bar(s), C::STAGE_BYTES);
-                    const uint32_t a_dst = base + s * C::STAGE_BYTES;
-                    if (WDV) {  // W stored [d, V]: two boxes of 64 entries x 64 k-rows
-                        tma_load_2d(a_dst, tw, w_row, kb * BK, full_bar(s), pol_w);
-                        tma_load_2d(a_dst + A_BYTES / 2, tw, w_row + 64, kb * BK, full_bar(s), pol_w);
-                    } else {
-                        tma_load_2d(a_dst, tw, kb * BK, w_row, full_bar(s), pol_w);
+                    mbar_expect_tx(full_bar(s), stage_bytes);
+                    for (int j = 0; j < kps; j++) {
+                        const uint32_t a_dst = base + s * stage_bytes + j * C::STAGE_BYTES;
+                        const int kc = (kb + j) * BK;
+                        if (WDV) {  // W stored [d, V]: two boxes of 64 entries x 64 k-rows
+                            tma_load_2d(a_dst, tw, w_row, kc, full_bar(s), pol_w);
+                            tma_load_2d(a_dst + A_BYTES / 2, tw, w_row + 64, kc, full_bar(s), pol_w);
+                        } else {
+                            tma_load_2d(a_dst, tw, kc, w_row, full_bar(s), pol_w);
+                        }
+                        tma_load_2d(a_dst + A_BYTES, &tmap_h, kc, n_tile * BN, full_bar(s), pol_h);
                     }
-                    tma_load_2d(a_dst + A_BYTES, &tmap_h, kb * BK, n_tile * BN, full_bar(s), pol_h);
-                    if (++s == STAGES) {
+                    if (++s == stages) {
                         s = 0;
                         ph ^= 1u;
                     }
@@ -161,22 +168,24 @@ umma_vm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                 }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(ab * BN);
-                for (int kb = 0; kb < num_kb; kb++) {
+                for (int kb = 0; kb < num_kb; kb += kps) {
                     if (!mbar_wait(full_bar(s), ph, abort_flag)) {
                         give_up();
                         ok = false;
                         break;
                     }
                     tc_fence_after();
-                    const uint32_t a_addr = base + s * C::STAGE_BYTES;
-                    const unsigned long long adesc = WDV ? smem_desc_sw128_mn(a_addr) : smem_desc_sw128(a_addr);
-                    constexpr unsigned long long a_step = WDV ? MN_KSTEP : 2ull;
-                    const unsigned long long bdesc = smem_desc_sw128(a_addr + A_BYTES);
+                    for (int j = 0; j < kps; j++) {
+                        const uint32_t a_addr = base + s * stage_bytes + j * C::STAGE_BYTES;
+                        const unsigned long long adesc = WDV ? smem_desc_sw128_mn(a_addr) : smem_desc_sw128(a_addr);
+                        constexpr unsigned long long a_step = WDV ? MN_KSTEP : 2ull;
+                        const unsigned long long bdesc = smem_desc_sw128(a_addr + A_BYTES);
 #pragma unroll
-                    for (int k = 0; k < BK / UMMA_K; k++)
-                        umma_bf16(d_tmem, adesc + a_step * k, bdesc + 2ull * k, idesc, (uint32_t)((kb | k) != 0));
+                        for (int k = 0; k < BK / UMMA_K; k++)
+                            umma_bf16(d_tmem, adesc + a_step * k, bdesc + 2ull * k, idesc, (uint32_t)((kb | j | k) != 0));
+                    }
                     umma_commit(empty_bar(s));  // the stage is free once these MMAs have read it
-                    if (++s == STAGES) {
+                    if (++s == stages) {
                         s = 0;
                         ph ^= 1u;
                     }
@@ -300,6 +309,9 @@ cudaError_t launch_vm(const GemmArgs &a, const UmmaPlan &p, cudaStream_t stream)
     const int fold = a.fold.rows ? 1 : 0;
     const int n_v = (a.V + BV - 1) / BV + fold;  // one more block for the folded classifier rows
     const int stream_w = (n_n == 1) ? 1 : 0;  // W is read by one CTA only: do not keep it in L2
+    // two k-blocks per stage where three such stages fit (every width but 256): the issuing thread's barrier
+    // test and commit then come once per 8 MMAs
+    const int kps = ((a.d / BK) % 2 == 0 && VCfg<BN>::STAGES / 2 >= 3) ? 2 : 1;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)p.grid);
     cfg.blockDim = dim3(NUM_THREADS);
@@ -318,7 +330,7 @@ cudaError_t launch_vm(const GemmArgs &a, const UmmaPlan &p, cudaStream_t stream)
                   : a.rank.thr               ? pick(std::integral_constant<int, EPI_COUNT>{})
                                              : pick(std::integral_constant<int, EPI_PLAIN>{});
     return cudaLaunchKernelEx(&cfg, kernel, p.tmap_w, p.tmap_h, fold ? p.tmap_j : p.tmap_w, a.M, a.V, a.d, n_n, n_v,
-                              fold ? n_v - 1 : -1, stream_w, a.v_offset, a.keys, a.status, a.pub, a.rank, a.noise, a.fold.parts,
+                              fold ? n_v - 1 : -1, stream_w, kps, a.v_offset, a.keys, a.status, a.pub, a.rank, a.noise, a.fold.parts,
                               a.fold.stride);
 }
 

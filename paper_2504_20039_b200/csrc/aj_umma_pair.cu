@@ -43,7 +43,8 @@
 // Roles in each CTA:
 //   warp 0      TMA producer (one thread).  The leader's draws the pair's next tile from the counter and
 //               announces it, through a small ring of slots in shared memory with their own barriers,
-//               to every other warp of both CTAs (-1: no more tiles).  Both wait for a free stage and load
+//               to every other warp of both CTAs (-1: no more tiles).  Both wait for a free stage (one or two
+//               k-blocks of 64, see pair_schedule) and load
 //               W[v0 + 128*rank .. +128, kb] and, per accumulator a, h[row0[a] + (N[a]/2)*rank .. , kb];
 //   warp 1, 2   warp 1 allocates tensor memory (both CTAs); in the leader one thread of each issues
 //               the MMAs of accumulator 0 / 1 (warp 2 only for wide tiles) and commits stage-release

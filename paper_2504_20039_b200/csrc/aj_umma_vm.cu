@@ -10,7 +10,8 @@
 //
 // Persistent CTAs, one per SM, three roles:
 //   warp 0      TMA producer: k-blocks of 64 columns of W (128 rows) and of h (BN rows) into a
-//               ring of shared-memory stages, 128-byte swizzle, completion on mbarriers;
+//               ring of shared-memory stages (one or two k-blocks per stage), 128-byte swizzle,
+//               completion on mbarriers;
 //   warp 1      MMA issuer: one thread issues tcgen05.mma (M=128, N=rows of the tile, K=16) into
 //               one of two accumulator buffers in tensor memory;
 //   warps 2..5  epilogue: a thread owns one TMEM lane = one vocabulary entry and reads 32 columns
@@ -42,7 +43,8 @@ template <int BN> struct VCfg {
     static constexpr int B_BYTES = BN * BK * 2;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
     // ring size: 224 of the SM's 227 KB per CTA, except for the narrowest tile, where 9 stages of
-    // 20 KB measured faster than 11 (161 vs 168 us on the batch-1 8B shape)
+    // 20 KB measured faster than 11 (161 vs 168 us on the batch-1 8B shape); with two k-blocks per
+    // stage that is four stages of 40 KB (five measured slower again: 163.5 vs 161.6 us)
     static constexpr int STAGES = ((BN <= 32 ? 192 : 224) * 1024) / STAGE_BYTES;
     static constexpr int TMEM_COLS = 2 * BN < 32 ? 32 : 2 * BN;
     static constexpr int NCH = (BN + 31) / 32;  // 32-column chunks per accumulator

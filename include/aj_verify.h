@@ -114,8 +114,8 @@ aj_status aj_verify(aj_handle h, const void *h_target, const void *h_draft, cons
 
 /*
  * Fold the target half of the classifier into the LM-head projection (the paper's Section 3.2,
- * "Classifier model & training": the classifier "can be fused with the existing LM head layer", which
- * makes its computation nearly free).  judge_w . [h_draft ; h_target] splits into a draft half and a
+ * "Classifier model & training": the paper remarks that a linear classifier can be computed together
+ * with the LM head, at next to no cost).  judge_w . [h_draft ; h_target] splits into a draft half and a
  * target half, and the target half, w_target . h_target[row], has the shape of one more logit.  This call
  * appends w_target = judge_w[d_draft ..] to the vocabulary as three bf16 rows b0 + b1 + b2 that add up to
  * w_target to fp32 precision (each the bf16 rounding of what the earlier ones leave); later cycles on

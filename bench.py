@@ -5,7 +5,7 @@
 A step is one whole cycle (LM-head projection + argmax, then judge + prefix scan: two launches) over one
 batch of seeded synthetic inputs shaped like the paper's Llama-3.x pairs.  The headline workload is
 the batch-1 8B-shaped configuration (B=1, K=16, d=4096, V=128256, bf16), the setting the paper's own
-measurements use (batch size 1); the batched 8B- and 70B-shaped configurations, three points of the sweep
+measurements use (batch size 1); the batched 8B- and 70B-shaped configurations, four points of the sweep
 around the HBM / tensor crossover, and two variants of the acceptance step (sampled target tokens, the top-K
 rule) are reported under "extra" in the same JSON line.  Metric: verified draft positions per second (B*K per cycle).
 
@@ -569,9 +569,9 @@ def main():
         if args.workload == "sweep":
             todo = [gen.sweep_config(B, K) for B in gen.SWEEP_B for K in gen.SWEEP_K]
         elif args.workload == "c2" and not vocab and not args.point:
-            # the batched 8B- and 70B-shaped workloads, and the three points of the sweep around the crossover
-            # from HBM-bound to tensor-bound (264, 520 and 576 rows)
-            todo = [gen.C3, gen.sweep_config(8, 32), gen.sweep_config(8, 64), gen.sweep_config(64, 8), gen.C4]
+            # the batched 8B- and 70B-shaped workloads, and the four points of the sweep around the crossover
+            # from HBM-bound to tensor-bound (136, 264, 520 and 576 rows)
+            todo = [gen.C3, gen.sweep_config(8, 16), gen.sweep_config(8, 32), gen.sweep_config(8, 64), gen.sweep_config(64, 8), gen.C4]
             if not rule:
                 # and the two variants of the acceptance step whose epilogues do more, each right after the
                 # default rule on the same workload: sampled target tokens at C3, the top-K rule at C4

@@ -406,7 +406,7 @@ static aj_status enqueue_project(aj_handle h, const void *h_target, const void *
         UmmaPlan p;
         p.bn = vm_choose_bn(M);
         const CUtensorMap *tw = get_tmap(h, W_lm, V, h->layout == AJ_W_DV ? -1 : 128);
-        const CUtensorMap *th = get_tmap(h, h_target, M, p.bn);
+        const CUtensorMap *th = get_tmap(h, h_target, M, vm_box_rows(M, p.bn));
         const CUtensorMap *tj = fold ? get_tmap(h, h->fold_rows, h->layout == AJ_W_DV ? 8 : JUDGE_FOLD_ROWS, h->layout == AJ_W_DV ? -1 : 128) : tw;
         if (!th || !tw || !tj) return AJ_ERR_CUDA;
         p.tmap_h = *th;

@@ -351,8 +351,9 @@ struct UmmaPlan {
     int bn;              // rows of h per tile
     int grid;
 };
-// tmap_w has a 64 x 128 box and tmap_h a 64 x bn box, bn = vm_choose_bn(M) rows of h per tile.
+// tmap_w has a 64 x 128 box and tmap_h a 64 x vm_box_rows(M, bn) box, bn = vm_choose_bn(M) rows of h per tile.
 int vm_choose_bn(int M);
+int vm_box_rows(int M, int bn);
 cudaError_t umma_vm_prepare();
 cudaError_t launch_umma_vm(const GemmArgs &a, const UmmaPlan &p, cudaStream_t stream);
 const char *umma_vm_path_name(int bn);

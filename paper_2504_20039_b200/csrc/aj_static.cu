@@ -155,7 +155,7 @@ extern "C" aj_status aj_verify_static(const void *h_target, const void *h_draft,
     } else if (dtype == AJ_BF16 && layout == AJ_W_VD && d % 64 == 0) {
         UmmaPlan p;
         p.bn = vm_choose_bn(M);
-        if (!encode_rows(s, &p.tmap_w, W_lm, d, V, 128) || !encode_rows(s, &p.tmap_h, h_target, d, M, p.bn)) return AJ_ERR_CUDA;
+        if (!encode_rows(s, &p.tmap_w, W_lm, d, V, 128) || !encode_rows(s, &p.tmap_h, h_target, d, M, vm_box_rows(M, p.bn))) return AJ_ERR_CUDA;
         const long long tiles = (long long)((M + p.bn - 1) / p.bn) * ((V + 127) / 128);
         p.grid = (int)(tiles < s->num_sms ? tiles : s->num_sms);
         e = launch_umma_vm(g, p, stream);

@@ -58,7 +58,7 @@ template <int BN, bool WDV, int EPI>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 umma_vm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_h,
                const __grid_constant__ CUtensorMap tmap_j, int M, int V, int d, int n_n, int n_v, int fold_tile,
-               int stream_w, int kps, int v_offset, unsigned long long *__restrict__ keys, int *__restrict__ status, const Publish pub,
+               int stream_w, int kps, int box_rows, int v_offset, unsigned long long *__restrict__ keys, int *__restrict__ status, const Publish pub,
                const RankArgs rk, const Noise nz, float *__restrict__ fold_parts, int fold_stride) {
     using C = VCfg<BN>;
     constexpr int STAGES = C::STAGES;
@@ -81,8 +81,12 @@ umma_vm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
     const int num_tiles = n_n * n_v;
     // A stage holds kps k-blocks (1 or 2), each [W | h], in the same ring: with two, the issuing thread tests
     // one barrier and commits once per 8 MMAs instead of per 4.
-    const uint32_t stage_bytes = (uint32_t)kps * C::STAGE_BYTES;
-    const int stages = STAGES / kps;
+    // (and the rows of h per k-block are the rows of the tensor map's box, box_rows <= BN: a batch that fits one
+    // row tile stages only the rows it has, which leaves room for more stages)
+    const uint32_t sub_bytes = A_BYTES + (uint32_t)box_rows * BK * 2;
+    const uint32_t stage_bytes = (uint32_t)kps * sub_bytes;
+    const int fit = (STAGES * C::STAGE_BYTES) / (int)stage_bytes;
+    const int stages = fit < STAGES ? fit : STAGES;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; s++) {
@@ -133,7 +137,7 @@ umma_vm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                     }
                     mbar_expect_tx(full_bar(s), stage_bytes);
                     for (int j = 0; j < kps; j++) {
-                        const uint32_t a_dst = base + s * stage_bytes + j * C::STAGE_BYTES;
+                        const uint32_t a_dst = base + s * stage_bytes + j * sub_bytes;
                         const int kc = (kb + j) * BK;
                         if (WDV) {  // W stored [d, V]: two boxes of 64 entries x 64 k-rows
                             tma_load_2d(a_dst, tw, w_row, kc, full_bar(s), pol_w);
@@ -178,7 +182,7 @@ umma_vm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant
                     }
                     tc_fence_after();
                     for (int j = 0; j < kps; j++) {
-                        const uint32_t a_addr = base + s * stage_bytes + j * C::STAGE_BYTES;
+                        const uint32_t a_addr = base + s * stage_bytes + j * sub_bytes;
                         const unsigned long long adesc = WDV ? smem_desc_sw128_mn(a_addr) : smem_desc_sw128(a_addr);
                         constexpr unsigned long long a_step = WDV ? MN_KSTEP : 2ull;
                         const unsigned long long bdesc = smem_desc_sw128(a_addr + A_BYTES);
@@ -313,7 +317,9 @@ cudaError_t launch_vm(const GemmArgs &a, const UmmaPlan &p, cudaStream_t stream)
     const int stream_w = (n_n == 1) ? 1 : 0;  // W is read by one CTA only: do not keep it in L2
     // two k-blocks per stage where three such stages fit (every width but 256): the issuing thread's barrier
     // test and commit then come once per 8 MMAs
-    const int kps = ((a.d / BK) % 2 == 0 && VCfg<BN>::STAGES / 2 >= 3) ? 2 : 1;
+    const int box_rows = vm_box_rows(a.M, BN);
+    const int ring = VCfg<BN>::STAGES * VCfg<BN>::STAGE_BYTES, sub = A_BYTES + box_rows * BK * 2;
+    const int kps = ((a.d / BK) % 2 == 0 && ring / (2 * sub) >= 3) ? 2 : 1;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)p.grid);
     cfg.blockDim = dim3(NUM_THREADS);
@@ -332,13 +338,17 @@ cudaError_t launch_vm(const GemmArgs &a, const UmmaPlan &p, cudaStream_t stream)
                   : a.rank.thr               ? pick(std::integral_constant<int, EPI_COUNT>{})
                                              : pick(std::integral_constant<int, EPI_PLAIN>{});
     return cudaLaunchKernelEx(&cfg, kernel, p.tmap_w, p.tmap_h, fold ? p.tmap_j : p.tmap_w, a.M, a.V, a.d, n_n, n_v,
-                              fold ? n_v - 1 : -1, stream_w, kps, a.v_offset, a.keys, a.status, a.pub, a.rank, a.noise, a.fold.parts,
+                              fold ? n_v - 1 : -1, stream_w, kps, box_rows, a.v_offset, a.keys, a.status, a.pub, a.rank, a.noise, a.fold.parts,
                               a.fold.stride);
 }
 
 }  // namespace
 
 int vm_choose_bn(int M) { return M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : 256; }
+
+// Rows of h in the tensor map's box (and per staged k-block): the tile width, or, for a batch of one row
+// tile wider than 32, just the batch's rows rounded up to the UMMA N granule of 16.
+int vm_box_rows(int M, int bn) { return (bn > 32 && M <= bn) ? ((M + 15) & ~15) : bn; }
 
 template <int BN> static cudaError_t set_smem() {
     const int bytes = VCfg<BN>::SMEM_BYTES;

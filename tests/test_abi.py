@@ -88,8 +88,11 @@ def test_two_sm_schedule_covers_every_row_once(built):
         assert max(sizes) - min(sizes) <= 1                   # spread evenly
         per_acc = -(-max(sizes) // 2) if s["dual"] else max(sizes)
         assert s["box_rows"] == 8 * per_acc <= 128
-        stage = 16384 + (2 if s["dual"] else 1) * s["box_rows"] * 128
-        assert 4 <= s["stages"] == min(8, (224 * 1024) // stage) and s["stages"] * stage <= 224 * 1024
+        # a stage holds two k-blocks of 64 where three such stages fit in the ring (and d / 64 is even), else one
+        sub = 16384 + (2 if s["dual"] else 1) * s["box_rows"] * 128
+        kps = 2 if ((d // 64) % 2 == 0 and (224 * 1024) // (2 * sub) >= 3) else 1
+        stage = kps * sub
+        assert 3 <= s["stages"] == min(8, (224 * 1024) // stage) and s["stages"] * stage <= 224 * 1024
         groups = [s["g_base"] + (g < s["g_rem"]) for g in range(s["n_groups"])]
         assert sum(groups) == s["n_n"] and min(groups) >= 1 and max(groups) - min(groups) <= 1
         assert max(groups) * (512 if s["dual"] else 256) * d * 2 <= 40 << 20 or max(groups) == 1

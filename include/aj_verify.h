@@ -272,7 +272,8 @@ int aj_last_launch_count(aj_handle h);
  *   [8] 1 if each tile uses two accumulators, each with its own issuing warp, that share the staged
  *       block of W_lm (a tile then holds up to 512 rows; chosen for every batch of more than 256 rows),
  *       else 0 (one tile of at most 256 rows on one accumulator, double-buffered)
- *   [9] depth of the shared-memory ring
+ *   [9] depth of the shared-memory ring, in stages; a stage holds two 64-column blocks of every operand
+ *       where three such stages fit (tiles of up to 320 rows, d / 64 even), else one
  * Errors: AJ_ERR_INVALID_ARG.
  */
 aj_status aj_pair_schedule(int M, int d, int V, int32_t out[10]);
